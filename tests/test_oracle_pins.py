@@ -1,0 +1,451 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU).
+
+Each test names the passage or the textbook fact it checks.  A mistake in the
+oracle (dropped term, wrong sign, transposed operand, wrong index) must fail at
+least one of these before the oracle is trusted as the yardstick of the CUDA path.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import hs_inputs as hi
+import oracle
+
+RNG = np.random.default_rng(1234)
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_round(x):
+    return hi.bf16_to_f32(hi.f32_to_bf16(np.asarray(x, np.float32))).astype(np.float64)
+
+
+# --------------------------------------------------------------------------- components
+def test_matvec_rmsnorm_textbook():
+    W = hi.normal_bf16(37 * 96, 5, 1, 0.5).reshape(37, 96)
+    x = RNG.standard_normal(96)
+    np.testing.assert_allclose(oracle.matvec_bf16(W, x), hi.bf16_to_f32(W).astype(np.float64) @ x, rtol=1e-12, atol=1e-12)
+    w = RNG.uniform(0.5, 1.5, 96).astype(np.float32)
+    got = oracle.rmsnorm(x, w, 1e-5)
+    np.testing.assert_allclose(got, x / np.sqrt((x * x).mean() + 1e-5) * w, rtol=1e-12)
+    # unit weight, eps -> 0: output has unit RMS and is invariant to the input's scale
+    one = np.ones(96, np.float32)
+    assert abs(np.sqrt((oracle.rmsnorm(x, one, 0.0) ** 2).mean()) - 1.0) < 1e-12
+    np.testing.assert_allclose(oracle.rmsnorm(7.5 * x, one, 0.0), oracle.rmsnorm(x, one, 0.0), rtol=1e-12)
+
+
+def test_conv_equals_direct_causal_convolution():
+    # the rolling-window step applied to a sequence == causal convolution with zero left padding
+    T, taps, bias = 11, RNG.uniform(-0.5, 0.5, 4).astype(np.float32), 0.3
+    x = RNG.standard_normal(T)
+    win, got = np.zeros(3), []
+    for t in range(T):
+        o, win = oracle.conv_step(win, x[t], taps, bias)
+        got.append(o)
+    xp = np.concatenate([np.zeros(3), x])
+    want = [bias + sum(float(taps[j]) * xp[t + j] for j in range(4)) for t in range(T)]
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    # the newest input is weighted by the last tap (np.convolve flips the kernel)
+    np.testing.assert_allclose(got, bias + np.convolve(x, taps[::-1].astype(np.float64))[:T], rtol=1e-12, atol=1e-12)
+    np.testing.assert_array_equal(win, x[-3:])
+
+
+def test_ssm_closed_form_constant_inputs():
+    # constant dt, x, B from S_0 = 0: S_t = dt x(x)B (1 - a^t)/(1 - a), a = exp(dt A)
+    P, N, dt, A = 4, 6, 0.3, -1.7
+    x, B, C = RNG.standard_normal(P), RNG.standard_normal(N), RNG.standard_normal(N)
+    S = np.zeros((P, N))
+    a = np.exp(dt * A)
+    for t in range(1, 8):
+        S, y = oracle.ssm_step(S, dt, A, 0.0, x, B, C)
+        np.testing.assert_allclose(S, dt * np.outer(x, B) * (1 - a ** t) / (1 - a), rtol=1e-12)
+        np.testing.assert_allclose(y, S @ C, rtol=1e-12)
+
+
+def test_ssm_no_decay_is_linear_attention_sum_and_C_picks_column():
+    # A -> 0-, dt = 1: S_t = sum_j x_j (x) B_j ; C = e_n reads column n ; D adds D x
+    P, N, T = 3, 5, 6
+    xs, Bs = RNG.standard_normal((T, P)), RNG.standard_normal((T, N))
+    S = np.zeros((P, N))
+    for t in range(T):
+        e = np.zeros(N); e[t % N] = 1.0
+        S, y = oracle.ssm_step(S, 1.0, -0.0, 2.0, xs[t], Bs[t], e)
+        want = sum(np.outer(xs[j], Bs[j]) for j in range(t + 1))
+        np.testing.assert_allclose(S, want, rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(y, want[:, t % N] + 2.0 * xs[t], rtol=1e-12, atol=1e-14)
+
+
+def test_ssm_decay_only():
+    # x = 0: the state only decays by exp(dt A); the state layout is [P][N] (y_p uses row p)
+    S0 = RNG.standard_normal((2, 3))
+    S, y = oracle.ssm_step(S0, 0.5, -2.0, 0.0, np.zeros(2), np.ones(3), np.array([1.0, 0, 0]))
+    np.testing.assert_allclose(S, np.exp(-1.0) * S0, rtol=1e-14)
+    np.testing.assert_allclose(y, np.exp(-1.0) * S0[:, 0], rtol=1e-14)
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 9])
+def test_chunked_ssd_equals_recurrence(T):
+    # one-chunk SSD form == T applications of the recurrence (and T = 1 is the recurrence itself)
+    P, N, A, D = 4, 4, -0.9, 0.7
+    S0 = RNG.standard_normal((P, N))
+    dt = RNG.uniform(0.01, 0.5, T)
+    x, B, C = RNG.standard_normal((T, P)), RNG.standard_normal((T, N)), RNG.standard_normal((T, N))
+    y, snaps = oracle.ssd_chunk(S0, dt, A, D, x, B, C)
+    S = S0
+    for i in range(T):
+        S, yi = oracle.ssm_step(S, dt[i], A, D, x[i], B[i], C[i])
+        np.testing.assert_allclose(snaps[i], S, rtol=1e-5, atol=1e-12)
+        np.testing.assert_allclose(y[i], yi, rtol=1e-5, atol=1e-12)
+
+
+def test_gdn_associative_memory():
+    # alpha = beta = 1, orthonormal keys: after writing (k_i, v_i), S k_j = v_j exactly; rewriting overwrites
+    dk, dv, r = 8, 5, 4
+    Q, _ = np.linalg.qr(RNG.standard_normal((dk, dk)))
+    keys, vals = Q[:, :r].T, RNG.standard_normal((r, dv))
+    S = np.zeros((dv, dk))
+    for i in range(r):
+        S, o = oracle.gdn_step(S, 1.0, 1.0, keys[i], keys[i], vals[i])
+        np.testing.assert_allclose(o, vals[i] / np.sqrt(dk), rtol=1e-10, atol=1e-12)   # o = S q / sqrt(dk), q = k_i
+    for j in range(r):
+        np.testing.assert_allclose(S @ keys[j], vals[j], rtol=1e-10, atol=1e-12)
+    new = RNG.standard_normal(dv)
+    S, _ = oracle.gdn_step(S, 1.0, 1.0, keys[0], keys[1], new)
+    np.testing.assert_allclose(S @ keys[1], new, rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(S @ keys[2], vals[2], rtol=1e-10, atol=1e-12)
+
+
+def test_gdn_gates():
+    dk, dv = 6, 3
+    S0 = RNG.standard_normal((dv, dk))
+    q, k, v = RNG.standard_normal(dk), RNG.standard_normal(dk), RNG.standard_normal(dv)
+    S, _ = oracle.gdn_step(S0, 0.3, 0.0, q, k, v)           # beta = 0: decay only
+    np.testing.assert_allclose(S, 0.3 * S0, rtol=1e-14)
+    S, _ = oracle.gdn_step(S0, 0.0, 0.8, q, k, v)           # alpha = 0: S = beta v k^T
+    np.testing.assert_allclose(S, 0.8 * np.outer(v, k), rtol=1e-14)
+    # general step against the matrix form S' (I - beta k k^T) + beta v k^T
+    S, o = oracle.gdn_step(S0, 0.9, 0.4, q, k, v)
+    want = 0.9 * S0 @ (np.eye(dk) - 0.4 * np.outer(k, k)) + 0.4 * np.outer(v, k)
+    np.testing.assert_allclose(S, want, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(o, want @ q / np.sqrt(dk), rtol=1e-12, atol=1e-14)
+
+
+def test_rope_properties():
+    hd = 16
+    x, y = RNG.standard_normal(hd), RNG.standard_normal(hd)
+    np.testing.assert_array_equal(oracle.rope(x, 0), x)                    # position 0 is the identity
+    d0 = oracle.rope(x, 7) @ oracle.rope(y, 3)
+    np.testing.assert_allclose(oracle.rope(x, 107) @ oracle.rope(y, 103), d0, rtol=1e-9)   # depends on m - n only
+    np.testing.assert_allclose(np.linalg.norm(oracle.rope(x, 12345)), np.linalg.norm(x), rtol=1e-12)
+    # pair (i, i + hd/2) turns by pos * theta^(-2i/hd): check pair 0 (angle = pos) and pair 3
+    e = np.zeros(hd); e[0] = 1.0
+    r = oracle.rope(e, 2)
+    np.testing.assert_allclose([r[0], r[hd // 2]], [np.cos(2.0), np.sin(2.0)], rtol=1e-12)
+    e = np.zeros(hd); e[3] = 1.0
+    r = oracle.rope(e, 5)
+    ang = 5 * 10000.0 ** (-2 * 3 / hd)
+    np.testing.assert_allclose([r[3], r[3 + hd // 2]], [np.cos(ang), np.sin(ang)], rtol=1e-12)
+
+
+def test_attention_special_cases_and_gqa_brute_force():
+    qh, kvh, hd, n = 4, 2, 8, 13
+    q = RNG.standard_normal((qh, hd))
+    K = hi.f32_to_bf16(RNG.standard_normal((n, kvh, hd)).astype(np.float32))
+    V = hi.f32_to_bf16(RNG.standard_normal((n, kvh, hd)).astype(np.float32))
+    Kf, Vf = hi.bf16_to_f32(K).astype(np.float64), hi.bf16_to_f32(V).astype(np.float64)
+    # single key: output = its value row
+    o = oracle.attention(q, K[:1], V[:1], qh, kvh, hd)
+    for h in range(qh):
+        np.testing.assert_allclose(o[h], Vf[0, h // 2], rtol=1e-14)
+    # all keys equal: uniform weights -> mean of V
+    Keq = np.repeat(K[:1], n, axis=0)
+    o = oracle.attention(q, Keq, V, qh, kvh, hd)
+    for h in range(qh):
+        np.testing.assert_allclose(o[h], Vf[:, h // 2].mean(axis=0), rtol=1e-12)
+    # grouped-query result == per-q-head softmax attention with kv heads repeated
+    o = oracle.attention(q, K, V, qh, kvh, hd)
+    for h in range(qh):
+        s = Kf[:, h // (qh // kvh)] @ q[h] / np.sqrt(hd)
+        p = np.exp(s - s.max()); p /= p.sum()
+        np.testing.assert_allclose(o[h], p @ Vf[:, h // (qh // kvh)], rtol=1e-12, atol=1e-14)
+
+
+def test_argmax_tiebreak_and_margin():
+    lg = np.array([0.1, 0.7, 0.7, -1.0, 0.5])
+    i, m = oracle.argmax_margin(lg)
+    assert i == 1 and m == 0.0                       # lowest index wins a tie, margin 0
+    i, m = oracle.argmax_margin(np.array([0.25, -3.0, 1.5, 1.0]))
+    assert i == 2 and m == 0.5
+    # decisions are taken on float32-rounded logits: a difference below float32 resolution is a tie
+    i, m = oracle.argmax_margin(np.array([1.0, 1.0 + 1e-12]))
+    assert i == 0 and m == 0.0
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 5, 8])
+def test_accept_len_brute_force(k):
+    # all match patterns in {0,1}^k: n = number of leading matches (tokens up to the first rejection, Sec. 3.3)
+    for pat in itertools.product([0, 1], repeat=k):
+        g = np.arange(10, 10 + k, dtype=np.int32)
+        d = np.where(np.array(pat) == 1, g, g + 1000).astype(np.int32)
+        want = k if all(pat) else pat.index(0)
+        assert oracle.accept_len(d, g) == want
+
+
+# --------------------------------------------------------------------------- seeded inputs
+def test_word_stream_numpy_equals_c():
+    import ctypes
+    out = np.empty(1000, np.uint64)
+    hi._lib().hsin_words(out.ctypes.data, 1000, 7, 99, 5)
+    np.testing.assert_array_equal(out, hi.words(7, 99, 1000, first=5))
+
+
+def test_weight_statistics():
+    w = hi.bf16_to_f32(hi.normal_bf16(400000, 0, 3, 0.02)).astype(np.float64)
+    assert abs(w.mean()) < 2e-4 and abs(w.std() - 0.02) < 2e-4
+    assert abs((np.abs(w) < 0.02).mean() - 0.6827) < 5e-3
+
+
+def _golden_eq1():
+    rows = [l.split() for l in open(os.path.join(GOLD, "eq1_tokens_per_round.txt")) if not l.startswith("#")]
+    return {int(k): float(v) for k, v in rows}
+
+
+def test_forced_accept_pattern_matches_eq1_numerator():
+    # mean emitted tokens per round of the truncated-geometric pattern -> (1 - a^(k+1))/(1 - a) (Eq. 1)
+    gold = _golden_eq1()
+    for k, want in gold.items():
+        assert abs(hi.expected_tokens_per_round(0.68, k) - want) < 1e-6
+        n = hi.forced_accept(k, 200000, seq=3)
+        assert n.min() >= 0 and n.max() <= k
+        assert abs((n + 1).mean() - want) < 0.012, (k, (n + 1).mean(), want)
+
+
+# --------------------------------------------------------------------------- model-level pins
+@pytest.fixture(scope="module")
+def tiny():
+    s = hi.CONFIGS["cfg1_tiny"]
+    blob, table = hi.make_weights(s, 0, "jitter")
+    return s, blob, table
+
+
+@pytest.fixture(scope="module")
+def tseq():
+    s = hi.CONFIGS["test_seq"]
+    blob, table = hi.make_weights(s, 0, "jitter")
+    return s, blob, table
+
+
+def _decode_spec(model, prompt, k, n_tokens, forced=None):
+    q = model.new_seq(); q.prefill(prompt)
+    out, ns, r = [q.pending], [], 0
+    while len(out) < n_tokens:
+        res = q.round(k, forced_n=-1 if forced is None else int(forced[r]))
+        out += list(res["emitted"]); ns.append(res["n"]); r += 1
+    return np.array(out), ns, q      # may overshoot n_tokens by up to k
+
+
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+@pytest.mark.parametrize("k", [0, 1, 2, 4, 8])
+def test_speculative_equals_plain_greedy(cfg, k, request):
+    # lossless under greedy decoding (Sec. 3.3): token for token identical, bit-exact in the oracle;
+    # k = 0 is ordinary autoregressive decoding
+    s, blob, table = request.getfixturevalue(cfg)
+    m = oracle.Model(s, blob, table, 160)
+    prompt = hi.make_prompt(s.V, s.prompt_len)
+    a = m.new_seq(); a.prefill(prompt)
+    ref = a.greedy(s.gen_tokens)
+    out, ns, _ = _decode_spec(m, prompt, k, s.gen_tokens)
+    np.testing.assert_array_equal(out[: s.gen_tokens], ref)
+    if k >= 2 and cfg == "tiny":
+        assert min(ns) < k and max(ns) == k      # both a rejection and a full accept occur
+
+
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+def test_rollback_equals_recompute(cfg, request):
+    # after rounds, committed state and KV rows == those of re-prefilling the accepted prefix from scratch
+    s, blob, table = request.getfixturevalue(cfg)
+    m = oracle.Model(s, blob, table, 160)
+    prompt = hi.make_prompt(s.V, s.prompt_len)
+    out, ns, q = _decode_spec(m, prompt, 4, 20)
+    q2 = m.new_seq(); q2.reset()
+    consumed = np.concatenate([prompt, out])[: q.len]
+    q2.prefill(consumed)
+    assert q2.len == q.len and q2.pending == q.pending
+    for a, b in ((q.ssm(), q2.ssm()), (q.gdn(), q2.gdn()), (q.conv(), q2.conv())):
+        if a is not None:
+            np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(q.k()[:, : q.len], q2.k()[:, : q.len])
+    np.testing.assert_array_equal(q.v()[:, : q.len], q2.v()[:, : q.len])
+
+
+def test_forced_accept_keeps_state_consistent(tiny):
+    # with a forced accept length the emitted drafts are kept; the state is the full model over what was emitted
+    s, blob, table = tiny
+    m = oracle.Model(s, blob, table, 200)
+    prompt = hi.make_prompt(s.V, 32)
+    forced = hi.forced_accept(4, 16)
+    out, ns, q = _decode_spec(m, prompt, 4, 24, forced=forced)
+    assert ns == list(forced[: len(ns)])
+    q2 = m.new_seq()
+    q2.prefill(np.concatenate([prompt, out])[: q.len])
+    np.testing.assert_array_equal(q.ssm(), q2.ssm())
+    np.testing.assert_array_equal(q.conv(), q2.conv())
+    assert q.pending == q2.pending
+
+
+def test_draft_equals_full_with_attention_output_zeroed(tiny):
+    # Eq. 4: the parallel draft is the full model with the attention output zeroed (here: W_o = 0)
+    s, blob, table = tiny
+    z = blob.copy()
+    for l in range(s.L):
+        hi.tensor_view(z, table, l, hi.T_W_O)[:] = 0
+    m, mz = oracle.Model(s, blob, table, 64), oracle.Model(s, z, table, 64)
+    a, b = m.new_seq(), mz.new_seq()
+    toks = hi.make_prompt(s.V, 12, seq=5)
+    k_before = a.k().copy()
+    for t in toks:
+        np.testing.assert_array_equal(a.step(t, mode=1), b.step(t, mode=0))
+    # the draft touched neither the cache nor the length; the full model's attention does change the logits
+    assert a.len == 0 and np.array_equal(a.k(), k_before)
+    c = m.new_seq()
+    full = [c.step(t, mode=0) for t in toks]
+    assert np.abs(full[-1] - b.step(int(toks[0]), mode=0)).max() > 0
+
+
+def test_sequential_draft_equals_stack_without_attention_layers(tseq):
+    # Eq. 5: attention layers are the identity in the draft (whole layer bypassed by the residual)
+    s, blob, table = tseq
+    m = oracle.Model(s, blob, table, 64)
+    lin = [l for l in range(s.L) if s.layer_type(l) == hi.LAYER_GDN]
+    m_lin = oracle.Model(s, blob, table, 64, layer_ids=lin)
+    a, b = m.new_seq(), m_lin.new_seq()
+    for t in hi.make_prompt(s.V, 10, seq=6):
+        np.testing.assert_array_equal(a.step(t, mode=1), b.step(t, mode=0))
+    assert a.len == 0
+
+
+def _f(blob, table, l, tid):
+    v = hi.tensor_view(blob, table, l, tid)
+    return hi.bf16_to_f32(v).astype(np.float64) if v.dtype == np.uint16 else v.astype(np.float64)
+
+
+def _rms(x, w, eps):
+    return x / np.sqrt((x * x).mean() + eps) * w
+
+
+def test_block_composition_special_cases(tiny):
+    # with the mixers silenced (W_out = W_o = 0) one layer is the textbook pre-norm SwiGLU residual block;
+    # with W_down = 0 as well the stack is the identity and logits = W_lm rmsnorm(E[token])
+    s, blob, table = tiny
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_OUT)[:] = 0
+    hi.tensor_view(b1, table, 0, hi.T_W_O)[:] = 0
+    tok = 77
+    e = _f(b1, table, -1, hi.G_EMBED)[tok]
+    Wlm, wf = _f(b1, table, -1, hi.G_LM_HEAD), _f(b1, table, -1, hi.G_FINAL_NORM)
+    gu, Wd, w2 = _f(b1, table, 0, hi.T_W_GU), _f(b1, table, 0, hi.T_W_DOWN), _f(b1, table, 0, hi.T_NORM2)
+    u = _rms(e, w2, s.eps)
+    g, up = gu[0::2] @ u, gu[1::2] @ u                     # even rows gate, odd rows up
+    h = e + Wd @ (g / (1 + np.exp(-g)) * up)
+    got = oracle.Model(s1, b1, table, 8).new_seq().step(tok)
+    np.testing.assert_allclose(got, Wlm @ _rms(h, wf, s.eps), rtol=1e-10, atol=1e-12)
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    got = oracle.Model(s1, b1, table, 8).new_seq().step(tok)
+    np.testing.assert_allclose(got, Wlm @ _rms(e, wf, s.eps), rtol=1e-10, atol=1e-12)
+
+
+def test_first_token_ssm_branch_closed_form(tiny):
+    # first token from zero state, one layer, attention and MLP silenced: conv sees only the newest tap,
+    # S_1 = dt x(x)B, y = (B.C) dt x + D x ; checks the in-projection row blocks z | x | B | C | dt
+    s, blob, table = tiny
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_O)[:] = 0
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    tok, di, N, H, P = 123, s.d_inner, s.N, s.H, s.P
+    e = _f(b1, table, -1, hi.G_EMBED)[tok]
+    u = _rms(e, _f(b1, table, 0, hi.T_NORM1), s.eps)
+    Win = _f(b1, table, 0, hi.T_W_IN)
+    z, xbc, dtr = Win[:di] @ u, Win[di:2 * di + 2 * N] @ u, Win[2 * di + 2 * N: 2 * di + 2 * N + H] @ u
+    cw, cb = _f(b1, table, 0, hi.T_CONV_W), _f(b1, table, 0, hi.T_CONV_B)
+    pre = cb + cw[:, 3] * xbc
+    act = pre / (1 + np.exp(-pre))
+    x, B, C = act[:di].reshape(H, P), act[di:di + N], act[di + N:]
+    dt = np.log1p(np.exp(dtr + _f(b1, table, 0, hi.T_DT_BIAS)))
+    D = _f(b1, table, 0, hi.T_D)
+    y = ((B @ C) * dt[:, None] * x + D[:, None] * x).reshape(-1)
+    g = y * (z / (1 + np.exp(-z)))
+    h = e + _f(b1, table, 0, hi.T_W_OUT) @ _rms(g, _f(b1, table, 0, hi.T_GNORM), s.eps)
+    want = _f(b1, table, -1, hi.G_LM_HEAD) @ _rms(h, _f(b1, table, -1, hi.G_FINAL_NORM), s.eps)
+    q = oracle.Model(s1, b1, table, 8).new_seq()
+    np.testing.assert_allclose(q.step(tok, mode=1), want, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(q.ssm()[0], dt[:, None, None] * x[:, :, None] * B[None, None, :], rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(q.conv()[0, 2], xbc, rtol=1e-12)            # newest raw input is the last window row
+    assert not q.conv()[0, :2].any()
+
+
+def test_attention_branch_first_two_tokens(tiny):
+    # attention only (W_out = W_down = 0), one layer: token 0 attends to itself -> o = v (bf16-rounded);
+    # checks q | k | v row blocks, RoPE on the cached key, cache layout [position][kv head][dim]
+    s, blob, table = tiny
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_OUT)[:] = 0
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    di, N, H = s.d_inner, s.N, s.H
+    r0 = 2 * di + 2 * N + H
+    Win = _f(b1, table, 0, hi.T_W_IN)
+    Wq, Wk, Wv = Win[r0:r0 + s.qh * s.hd], Win[r0 + s.qh * s.hd: r0 + (s.qh + s.kvh) * s.hd], Win[r0 + (s.qh + s.kvh) * s.hd:]
+    E, Wo = _f(b1, table, -1, hi.G_EMBED), _f(b1, table, 0, hi.T_W_O)
+    Wlm, wf, w1 = _f(b1, table, -1, hi.G_LM_HEAD), _f(b1, table, -1, hi.G_FINAL_NORM), _f(b1, table, 0, hi.T_NORM1)
+    q = oracle.Model(s1, b1, table, 8).new_seq()
+    t0, t1 = 11, 2222
+    u0 = _rms(E[t0], w1, s.eps)
+    v0 = bf16_round(Wv @ u0)
+    o0 = np.repeat(v0.reshape(s.kvh, s.hd), s.qh // s.kvh, axis=0).reshape(-1)
+    np.testing.assert_allclose(q.step(t0), Wlm @ _rms(E[t0] + Wo @ o0, wf, s.eps), rtol=1e-9, atol=1e-11)
+    np.testing.assert_array_equal(hi.bf16_to_f32(q.v()[0, 0]).reshape(-1), v0.astype(np.float32))
+    # second token: two keys, causal; brute-force softmax with RoPE at positions 0 and 1
+    u1 = _rms(E[t1], w1, s.eps)
+    k0 = bf16_round(np.concatenate([oracle.rope(r, 0) for r in (Wk @ u0).reshape(s.kvh, s.hd)]))
+    k1 = bf16_round(np.concatenate([oracle.rope(r, 1) for r in (Wk @ u1).reshape(s.kvh, s.hd)]))
+    v1 = bf16_round(Wv @ u1)
+    qq = np.stack([oracle.rope(r, 1) for r in (Wq @ u1).reshape(s.qh, s.hd)])
+    o = []
+    for h in range(s.qh):
+        kh = h // (s.qh // s.kvh)
+        sc = np.array([qq[h] @ k0.reshape(s.kvh, s.hd)[kh], qq[h] @ k1.reshape(s.kvh, s.hd)[kh]]) / np.sqrt(s.hd)
+        p = np.exp(sc - sc.max()); p /= p.sum()
+        o.append(p[0] * v0.reshape(s.kvh, s.hd)[kh] + p[1] * v1.reshape(s.kvh, s.hd)[kh])
+    want = Wlm @ _rms(E[t1] + Wo @ np.concatenate(o), wf, s.eps)
+    np.testing.assert_allclose(q.step(t1), want, rtol=1e-9, atol=1e-11)
+
+
+def test_gdn_layer_first_token_closed_form(tseq):
+    # one DeltaNet layer from zero state, MLP silenced: S_1 = beta v k^T, o = beta v (k.q)/sqrt(dk)
+    s, blob, table = tseq
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    tok, nk, nv, gh, dk, dv = 99, s.gh * s.gdk, s.gh * s.gdv, s.gh, s.gdk, s.gdv
+    e = _f(b1, table, -1, hi.G_EMBED)[tok]
+    u = _rms(e, _f(b1, table, 0, hi.T_NORM1), s.eps)
+    Win = _f(b1, table, 0, hi.T_W_IN)
+    raw = Win[:2 * nk + nv] @ u
+    z, ga, gb = Win[2 * nk + nv:2 * nk + 2 * nv] @ u, Win[2 * nk + 2 * nv:2 * nk + 2 * nv + gh] @ u, Win[2 * nk + 2 * nv + gh:] @ u
+    pre = _f(b1, table, 0, hi.T_CONV_B) + _f(b1, table, 0, hi.T_CONV_W)[:, 3] * raw
+    act = pre / (1 + np.exp(-pre))
+    qv, kv, vv = act[:nk].reshape(gh, dk), act[nk:2 * nk].reshape(gh, dk), act[2 * nk:].reshape(gh, dv)
+    qn = qv / np.sqrt((qv * qv).sum(1, keepdims=True) + 1e-6)
+    kn = kv / np.sqrt((kv * kv).sum(1, keepdims=True) + 1e-6)
+    beta = 1 / (1 + np.exp(-gb))
+    o = beta[:, None] * vv * (kn * qn).sum(1, keepdims=True) / np.sqrt(dk)
+    wn = _f(b1, table, 0, hi.T_GNORM)
+    o = np.stack([_rms(o[h], wn, s.eps) for h in range(gh)]) * (z / (1 + np.exp(-z))).reshape(gh, dv)
+    h1 = e + _f(b1, table, 0, hi.T_W_OUT) @ o.reshape(-1)
+    want = _f(b1, table, -1, hi.G_LM_HEAD) @ _rms(h1, _f(b1, table, -1, hi.G_FINAL_NORM), s.eps)
+    q = oracle.Model(s1, b1, table, 8).new_seq()
+    np.testing.assert_allclose(q.step(tok, mode=1), want, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(q.gdn()[0], beta[:, None, None] * vv[:, :, None] * kn[:, None, :], rtol=1e-10, atol=1e-14)
