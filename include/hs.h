@@ -1,0 +1,187 @@
+/*
+ * libhs - decode hot path of component-aware self-speculative decoding on hybrid
+ * language models, for one NVIDIA B200 (sm_100a).
+ *
+ * One speculative round (paper Sec. 3.3) is
+ *     hs_draft(k)  ->  hs_verify(k)  ->  hs_accept_rollback()
+ * - draft:  the draft model M_S (paper Eq. 4: attention output zeroed in a parallel hybrid;
+ *   Eq. 5: attention layers are the identity in a sequential hybrid) proposes k tokens
+ *   autoregressively from the committed recurrent state, on scratch state, without touching
+ *   the KV cache;
+ * - verify: the full model M_H (Eq. 2 / Eq. 3) processes the k+1 candidates in one pass, keeps the
+ *   recurrent state after every position and appends k+1 KV rows;
+ * - accept/rollback: greedy rule (Sec. 3.3, T = 0): drafts are kept up to the first position whose
+ *   draft token differs from the full model's argmax; the committed state becomes the snapshot of
+ *   the last accepted position and the KV length is cut to the accepted prefix.
+ *
+ * Conventions
+ * - All functions return HS_OK (0) or a negative hs_status.  Nothing throws, aborts or traps.
+ * - The library allocates NO device memory.  Every device buffer is supplied by the caller in
+ *   hs_buffers (sizes from hs_query_sizes), must be 256-byte aligned and must outlive the handle.
+ *   The library owns only the host-side handle.
+ * - All device work is enqueued on the stream given to hs_init_model.  Calls are asynchronous
+ *   unless they take or return HOST data (documented per call).
+ * - "dev" / "host" in a parameter name says where the pointer must live.
+ * - Sequence b (0 <= b < batch) owns: kv_len[b] consumed tokens (KV rows 0..kv_len-1 and the
+ *   recurrent state reflect them) and a pending token: the full model's greedy choice after those
+ *   tokens, already emitted, not yet consumed.
+ */
+#ifndef HS_H
+#define HS_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HS_OK = 0,
+    HS_ERR_INVALID_ARG = -1,  /* null pointer, bad shape, k out of range, ... */
+    HS_ERR_SIZE = -2,         /* a caller buffer is smaller than hs_query_sizes reports */
+    HS_ERR_CAPACITY = -3,     /* kv_len + k + 1 would exceed kv_capacity */
+    HS_ERR_ORDER = -4,        /* call sequence violated (e.g. accept before verify) */
+    HS_ERR_CUDA = -5,         /* CUDA runtime error; text in hs_last_error */
+    HS_ERR_TIMEOUT = -6,      /* a bounded device-side wait expired */
+    HS_ERR_DEVICE = -7        /* a kernel reported an inconsistency through the status word */
+} hs_status;
+
+enum { HS_ARCH_PARALLEL = 0, HS_ARCH_SEQUENTIAL = 1 };
+/* layer kinds: parallel block (Mamba-2 + attention summed, Eq. 2); Gated DeltaNet layer and
+ * attention layer of a sequential hybrid (Eq. 3; layer l is attention iff l % 4 == 3) */
+enum { HS_LAYER_PAR = 0, HS_LAYER_GDN = 1, HS_LAYER_ATT = 2 };
+
+typedef struct hs_config {
+    int32_t arch;              /* HS_ARCH_* */
+    int32_t L, d, V;           /* layers, model width, vocabulary */
+    int32_t H, P, N;           /* Mamba-2 heads, head dim, state dim (one B/C group); parallel arch */
+    int32_t conv_w;            /* causal depthwise conv width; must be 4 */
+    int32_t qh, kvh, hd;       /* attention: query heads, KV heads, head dim */
+    int32_t ff;                /* SwiGLU width */
+    int32_t gh, gdk, gdv;      /* Gated DeltaNet heads, key dim, value dim; sequential arch */
+    int32_t max_batch;         /* sequences resident at once */
+    int32_t max_k;             /* largest draft length (<= 8) */
+    int32_t kv_capacity;       /* KV rows per sequence */
+    float rope_theta;          /* 10000 */
+    float eps;                 /* RMSNorm epsilon */
+    int32_t flags;             /* HS_FLAG_* */
+} hs_config;
+
+enum {
+    HS_FLAG_GRAPHS = 1         /* replay each (mode, k, batch) step as a captured CUDA graph */
+};
+
+/* Bytes the caller must provide (each buffer 256-byte aligned). */
+typedef struct hs_sizes {
+    int64_t weights;           /* weight blob, format below */
+    int64_t snap;              /* recurrent-state snapshots [rec layer][seq][max_k+1][state] fp32 */
+    int64_t dstate;            /* draft scratch state       [rec layer][seq][state] fp32 */
+    int64_t conv;              /* conv windows: committed, per-position history, draft ping-pong, fp32 */
+    int64_t kv;                /* K then V: [attn layer][seq][kv head][kv_capacity][hd] bf16 each */
+    int64_t work;              /* activations, logits, split-KV partials, RoPE table, control block */
+} hs_sizes;
+
+typedef struct hs_buffers {    /* DEVICE pointers */
+    const void *weights;
+    void *snap, *dstate, *conv, *kv, *work;
+} hs_buffers;
+
+typedef struct hs_model hs_model;
+
+/*
+ * Weight blob format (all offsets multiples of 256 bytes; bf16 matrices are row-major [out, in]).
+ * Globals, in order: EMBED [V,d] bf16, LM_HEAD [V,d] bf16, FINAL_NORM [d] f32.
+ * Then per layer, the tensors its kind has, in id order:
+ *   0 NORM1 [d] f32
+ *   1 W_IN  bf16, row blocks:  parallel: z[di] x[di] B[N] C[N] dt[H] q[qh*hd] k[kvh*hd] v[kvh*hd]
+ *                              DeltaNet: q[gh*gdk] k[gh*gdk] v[gh*gdv] z[gh*gdv] a[gh] b[gh]
+ *                              attention: q k v
+ *   2 CONV_W [channels,4] f32 (tap 3 weights the newest input), 3 CONV_B [channels] f32
+ *   4 A_LOG [H], 5 D [H], 6 DT_BIAS [H] f32                        (parallel only)
+ *   7 GNORM f32: gated-norm weight [di] (parallel) / per-head output-norm weight [gdv] (DeltaNet)
+ *   8 W_OUT [d, di] or [d, gh*gdv] bf16, 9 W_O [d, qh*hd] bf16
+ *   10 NORM2 [d] f32, 11 W_GU [2*ff, d] bf16 (row 2i = gate_i, row 2i+1 = up_i), 12 W_DOWN [d, ff] bf16
+ * hs_weight_offset returns the byte offset of (layer, tensor id), layer = -1 for the globals
+ * (ids 0..2), or -1 if the layer has no such tensor.
+ */
+enum { HS_T_NORM1 = 0, HS_T_W_IN, HS_T_CONV_W, HS_T_CONV_B, HS_T_A_LOG, HS_T_D, HS_T_DT_BIAS, HS_T_GNORM,
+       HS_T_W_OUT, HS_T_W_O, HS_T_NORM2, HS_T_W_GU, HS_T_W_DOWN, HS_T_COUNT };
+enum { HS_G_EMBED = 0, HS_G_LM_HEAD = 1, HS_G_FINAL_NORM = 2 };
+
+/* Sizes of the caller's buffers for this configuration.  Host only, no CUDA call.
+ * HS_ERR_INVALID_ARG if the shape is unsupported (see hs_init_model). */
+int hs_query_sizes(const hs_config *cfg, hs_sizes *out);
+int64_t hs_weight_offset(const hs_config *cfg, int layer, int tensor);
+
+/* Build the host handle.  Requirements: conv_w == 4; d, ff, di, qh*hd, gh*gdv multiples of 256;
+ * P and gdv multiples of 16; N in {64,128,256}; hd in {64,128}; gdk == 64; qh % kvh == 0;
+ * (qh/kvh)*(max_k+1) <= 48; max_k <= 8.  Enqueues (on `stream`, a cudaStream_t) the RoPE table
+ * upload and the zeroing of the control block; does not read the other buffers.
+ * The weights must already be in `bufs->weights` in the blob format. */
+int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs_model **out);
+
+/* Zero every sequence: recurrent state, conv windows, kv_len = 0, no pending token.  Async. */
+int hs_reset(hs_model *m);
+
+/* Consume prompts with the full model (paper Sec. 3.3 prefix x_{1:t}).  tokens_host: the prompts
+ * back to back (sequence b starts at sum(lens_host[0..b-1])); lens_host[b] >= 1.  Sets the batch
+ * size for the following rounds.  Afterwards kv_len[b] = lens[b] and pending[b] = the greedy choice
+ * after the last prompt token (generated token #1).  Runs as repeated verify passes over chunks of
+ * max_k+1 tokens with every candidate accepted.  Synchronises the stream before returning. */
+int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host, int batch);
+
+/* Draft phase: k draft-mode steps for every sequence; candidates cand[b][0..k] = [pending, d_1..d_k]
+ * stay on the device.  0 <= k <= max_k; k = 0 does nothing.  Async. */
+int hs_draft(hs_model *m, int k);
+
+/* Verification phase over k+1 candidates per sequence at positions kv_len[b]..kv_len[b]+k.
+ * cand_dev: NULL to verify the candidates of the preceding hs_draft(k) (HS_ERR_ORDER if there was
+ * none with this k, except k = 0), or int32 [batch][k+1] candidates to verify instead (cand[b][0]
+ * replaces the pending token).  Produces g[b][i] = argmax of the logits after candidate i
+ * (lowest id on ties), the top-2 margin, state snapshots and KV rows.  Async.
+ * HS_ERR_CAPACITY if a sequence could exceed kv_capacity. */
+int hs_verify(hs_model *m, int k, const int32_t *cand_dev);
+
+/* Greedy acceptance + rollback after hs_verify.  Per sequence: n = number of leading drafts with
+ * cand[i+1] == g[i]; emitted = cand[1..n], g[n]; committed state <- snapshot n; kv_len += n+1;
+ * pending <- g[n].  forced_n_dev (int32 [batch] on the device, or NULL) overrides n (0 <= n <= k) with
+ * everything else unchanged; forced_next_dev (int32 [batch], entries < 0 ignored, or NULL) overrides
+ * the next pending token.  n_acc_host [batch] / emitted_host [batch][k+1] (unused slots -1): if
+ * either is non-NULL the results are copied to HOST memory and the stream is synchronised. */
+int hs_accept_rollback(hs_model *m, const int32_t *forced_n_dev, const int32_t *forced_next_dev,
+                       int32_t *n_acc_host, int32_t *emitted_host);
+
+/* One whole round with HOST buffers: uploads forced_n_host / forced_next_host (either may be NULL),
+ * runs draft(k), verify(k), accept/rollback, downloads n_acc_host [batch] and
+ * emitted_host [batch][k+1] (either may be NULL) and synchronises. */
+int hs_round_host(hs_model *m, int k, const int32_t *forced_n_host, const int32_t *forced_next_host,
+                  int32_t *n_acc_host, int32_t *emitted_host);
+
+/* ---- test and injection hooks (synchronous, host buffers) ---- */
+enum { HS_STATE_SSM = 0,   /* f32 [H][P][N] committed Mamba-2 state of (layer, seq) */
+       HS_STATE_CONV = 1,  /* f32 [3][channels] committed conv window (oldest row first) */
+       HS_STATE_GDN = 2,   /* f32 [gh][gdv][gdk] committed DeltaNet state */
+       HS_STATE_K = 3,     /* bf16 [rows][kvh][hd], rows = bytes / (kvh*hd*2), from row 0 */
+       HS_STATE_V = 4,
+       HS_STATE_DRAFT = 5  /* f32 draft scratch state after the last hs_draft (export only) */ };
+int hs_export_state(hs_model *m, int layer, int seq, int kind, void *host, int64_t bytes);
+int hs_import_state(hs_model *m, int layer, int seq, int kind, const void *host, int64_t bytes);
+/* Declare sequence `seq` to hold kv_len consumed tokens and the given pending token (after imports);
+ * batch = number of sequences that take part in the following rounds. */
+int hs_set_context(hs_model *m, int seq, int kv_len, int pending);
+int hs_set_batch(hs_model *m, int batch);
+int hs_get_context(hs_model *m, int seq, int32_t *kv_len, int32_t *pending);
+/* Logits [rows][V] f32 of the last pass (verify: row b*(k+1)+i; draft: last step, row b). */
+int hs_get_logits(hs_model *m, float *host, int rows);
+/* cand / g int32 [batch][k+1] and margin f32 [batch][k+1] of the last verify (any may be NULL). */
+int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin_host);
+/* Number of kernels the library has launched (including those replayed inside graphs) so far. */
+int64_t hs_launch_count(const hs_model *m);
+/* Device status word: 0, or the first hs_status a kernel recorded.  Synchronises. */
+int hs_device_status(hs_model *m);
+const char *hs_last_error(const hs_model *m);
+int hs_destroy(hs_model *m);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,634 @@
+// C-ABI of libhs: buffer layout, the fixed kernel sequence of a draft step and of a verify pass,
+// CUDA-graph replay of those sequences, and the test / injection hooks.  See include/hs.h.
+#include "hs_internal.h"
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+namespace {
+
+constexpr int64_t ALIGN = 256;
+inline int64_t up(int64_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+int layer_type(const hs_config &c, int l) {
+    if (c.arch == HS_ARCH_PARALLEL) return HS_LAYER_PAR;
+    return (l % 4 == 3) ? HS_LAYER_ATT : HS_LAYER_GDN;
+}
+int d_inner(const hs_config &c) { return c.H * c.P; }
+int conv_channels(const hs_config &c) {
+    return c.arch == HS_ARCH_PARALLEL ? c.H * c.P + 2 * c.N : 2 * c.gh * c.gdk + c.gh * c.gdv;
+}
+int attn_rows(const hs_config &c) { return (c.qh + 2 * c.kvh) * c.hd; }
+int in_rows(const hs_config &c, int type, bool draft) {
+    if (type == HS_LAYER_PAR) return 2 * d_inner(c) + 2 * c.N + c.H + (draft ? 0 : attn_rows(c));
+    if (type == HS_LAYER_GDN) return 2 * c.gh * c.gdk + 2 * c.gh * c.gdv + 2 * c.gh;
+    return attn_rows(c);
+}
+
+struct TensorDesc { int id; int64_t elems; int esize; };
+
+int layer_tensors(const hs_config &c, int type, TensorDesc *out) {
+    int n = 0;
+    const int64_t d = c.d, di = d_inner(c), cd = conv_channels(c);
+    out[n++] = {HS_T_NORM1, d, 4};
+    out[n++] = {HS_T_W_IN, (int64_t)in_rows(c, type, false) * d, 2};
+    if (type == HS_LAYER_PAR) {
+        out[n++] = {HS_T_CONV_W, cd * 4, 4}; out[n++] = {HS_T_CONV_B, cd, 4};
+        out[n++] = {HS_T_A_LOG, c.H, 4}; out[n++] = {HS_T_D, c.H, 4}; out[n++] = {HS_T_DT_BIAS, c.H, 4};
+        out[n++] = {HS_T_GNORM, di, 4};
+        out[n++] = {HS_T_W_OUT, d * di, 2}; out[n++] = {HS_T_W_O, d * c.qh * c.hd, 2};
+    } else if (type == HS_LAYER_GDN) {
+        out[n++] = {HS_T_CONV_W, cd * 4, 4}; out[n++] = {HS_T_CONV_B, cd, 4};
+        out[n++] = {HS_T_GNORM, c.gdv, 4};
+        out[n++] = {HS_T_W_OUT, d * c.gh * c.gdv, 2};
+    } else {
+        out[n++] = {HS_T_W_O, d * c.qh * c.hd, 2};
+    }
+    out[n++] = {HS_T_NORM2, d, 4};
+    out[n++] = {HS_T_W_GU, (int64_t)2 * c.ff * d, 2};
+    out[n++] = {HS_T_W_DOWN, d * c.ff, 2};
+    return n;
+}
+
+// byte offset of (layer, tensor) in the blob, or the total size when layer == L
+int64_t blob_offset(const hs_config &c, int layer, int tensor) {
+    int64_t off = 0;
+    const int64_t g[3] = {(int64_t)c.V * c.d * 2, (int64_t)c.V * c.d * 2, (int64_t)c.d * 4};
+    for (int t = 0; t < 3; ++t) {
+        if (layer == -1 && tensor == t) return off;
+        off = up(off + g[t]);
+    }
+    if (layer == -1) return -1;
+    TensorDesc td[HS_T_COUNT];
+    for (int l = 0; l < c.L; ++l) {
+        int n = layer_tensors(c, layer_type(c, l), td);
+        for (int i = 0; i < n; ++i) {
+            if (l == layer && td[i].id == tensor) return off;
+            off = up(off + td[i].elems * td[i].esize);
+        }
+        if (l == layer) return -1;
+    }
+    return off;   // layer == L: total
+}
+
+bool valid_config(const hs_config &c) {
+    if (c.L < 1 || c.d < 256 || (c.d & 255) || c.V < 2 || (c.ff & 255) || c.ff < 256) return false;
+    if (c.conv_w != 4 || c.max_k < 0 || c.max_k > HS_MAX_K || c.max_batch < 1 || c.kv_capacity < 1) return false;
+    if (c.hd != 64 && c.hd != 128) return false;
+    if (c.qh < 1 || c.kvh < 1 || c.qh % c.kvh) return false;
+    if ((c.qh / c.kvh) * (c.max_k + 1) > HS_MAX_GT) return false;
+    if ((c.qh * c.hd) & 255) return false;
+    if (c.arch == HS_ARCH_PARALLEL) {
+        if (c.H < 1 || c.P < 16 || (c.P & 15)) return false;
+        if (c.N != 64 && c.N != 128 && c.N != 256) return false;
+        if ((c.H * c.P) & 255) return false;
+        if ((2 * c.H * c.P + 2 * c.N + c.H) & 3) return false;   // attention rows must start 16-byte aligned
+    } else if (c.arch == HS_ARCH_SEQUENTIAL) {
+        if (c.gh < 1 || c.gdk != 64 || c.gdv < 16 || c.gdv > 64 || (c.gdv & 15)) return false;
+        if ((c.gh * c.gdv) & 255) return false;
+    } else return false;
+    return true;
+}
+
+struct Derived {
+    int B, Tm, R, n_rl, n_al, convd, gw, in_rows_max, att_chunk, att_nch;
+    int64_t state_elems;
+};
+
+Derived derive(const hs_config &c) {
+    Derived v;
+    v.B = c.max_batch; v.Tm = c.max_k + 1; v.R = v.B * v.Tm;
+    v.n_rl = v.n_al = 0; v.in_rows_max = 0;
+    for (int l = 0; l < c.L; ++l) {
+        int t = layer_type(c, l);
+        if (t != HS_LAYER_ATT) ++v.n_rl;
+        if (t != HS_LAYER_GDN) ++v.n_al;
+        int r = in_rows(c, t, false);
+        if (r > v.in_rows_max) v.in_rows_max = r;
+    }
+    v.convd = conv_channels(c);
+    v.gw = c.arch == HS_ARCH_PARALLEL ? d_inner(c) : c.gh * c.gdv;
+    v.state_elems = c.arch == HS_ARCH_PARALLEL ? (int64_t)c.H * c.P * c.N : (int64_t)c.gh * c.gdv * c.gdk;
+    int chunk = 256;
+    while (chunk > 64 && (int64_t)c.max_batch * c.kvh * ((c.kv_capacity + chunk - 1) / chunk) < 296) chunk >>= 1;
+    v.att_chunk = chunk;
+    v.att_nch = (c.kv_capacity + chunk - 1) / chunk;
+    return v;
+}
+
+// layout of the work buffer; base may be null to only measure
+struct WorkLayout {
+    int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters;
+    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, total;
+};
+
+WorkLayout work_layout(const hs_config &c, const Derived &v) {
+    WorkLayout w; int64_t off = 0;
+    auto take = [&](int64_t bytes) { int64_t o = off; off = up(off + bytes); return o; };
+    w.kv_len = take(4 * v.B); w.slot = take(4 * v.B);
+    w.cand = take(4 * v.R); w.g = take(4 * v.R); w.margin = take(4 * v.R);
+    w.n_acc = take(4 * v.B); w.emitted = take(4 * v.R);
+    w.stage_n = take(4 * v.B); w.stage_next = take(4 * v.B);
+    w.status = take(4); w.counters = take((int64_t)4 * v.B * c.kvh);
+    w.rope = take((int64_t)c.kv_capacity * (c.hd / 2) * 8);
+    w.h = take((int64_t)4 * v.R * c.d);
+    w.zx = take((int64_t)4 * v.R * v.in_rows_max);
+    w.gbuf = take((int64_t)4 * v.R * v.gw);
+    w.obuf = take((int64_t)4 * v.R * c.qh * c.hd);
+    w.abuf = take((int64_t)4 * v.R * c.ff);
+    w.logits = take((int64_t)4 * v.R * c.V);
+    w.att_acc = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * c.hd);
+    w.att_ml = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * 2);
+    w.total = off;
+    return w;
+}
+
+int fail(hs_model *m, int code, const char *msg) {
+    if (m) m->err = msg;
+    return code;
+}
+int cuda_fail(hs_model *m, cudaError_t e, const char *where) {
+    if (m) { m->err = std::string(where) + ": " + cudaGetErrorString(e); }
+    return HS_ERR_CUDA;
+}
+#define CK(call, where) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return cuda_fail(m, e__, where); } while (0)
+
+// ------------------------------------------------------------------------------------------------
+// one pass of the model over T positions per sequence (sequences b0 .. b0+nb-1)
+//   draft = false: full model M_H (verify);  draft = true: draft model M_S, one position,
+//   reading candidate column `col` and, for step > 0, the scratch state of the previous step.
+// ------------------------------------------------------------------------------------------------
+int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
+    const hs_config &c = m->c;
+    cudaStream_t s = m->stream;
+    const int rows = nb * T, d = c.d;
+    const int64_t se = m->state_elems;
+    CK(launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->h, s), "embed");
+    ++m->launches;
+    for (int l = 0; l < c.L; ++l) {
+        const HsLayer &ly = m->layers[l];
+        if (draft && ly.type == HS_LAYER_ATT) continue;           // Eq. 5: identity in the draft
+        const bool with_attn = !draft && ly.type != HS_LAYER_GDN;
+        const int inr = draft ? ly.in_rows_draft : ly.in_rows_full;
+        // (1) RMSNorm + in-projection (verify: Mamba rows and q|k|v rows in one pass over u)
+        GemvArgs ga{};
+        ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->h; ga.ldx0 = d; ga.norm_w = ly.norm1; ga.eps = c.eps;
+        ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
+        CK(launch_gemv(ga, s, &m->launches), "in_proj");
+        // (2) recurrent mixer
+        if (ly.type != HS_LAYER_ATT) {
+            const size_t lrB = (size_t)ly.rl * m->B;
+            const float *win_in; float *win_out = nullptr, *hist = nullptr;
+            if (!draft) { win_in = m->cw + lrB * 3 * m->convd; hist = m->hist + lrB * m->Tm * m->convd; }
+            else {
+                const size_t half = (size_t)m->n_rl * m->B * 3 * m->convd;
+                win_in = step == 0 ? m->cw + lrB * 3 * m->convd : m->dcw + ((step - 1) & 1) * half + lrB * 3 * m->convd;
+                win_out = m->dcw + (step & 1) * half + lrB * 3 * m->convd;
+            }
+            const float *st_in; int64_t in_seq, in_slot; float *st_out; int64_t out_seq, out_slot;
+            float *snap_l = m->snap + lrB * m->Tm * se, *dst_l = m->dstate + lrB * se;
+            if (!draft) { st_in = snap_l; in_seq = m->Tm * se; in_slot = se; st_out = snap_l; out_seq = m->Tm * se; out_slot = se; }
+            else if (step == 0) { st_in = snap_l; in_seq = m->Tm * se; in_slot = se; st_out = dst_l; out_seq = se; out_slot = 0; }
+            else { st_in = dst_l; in_seq = se; in_slot = 0; st_out = dst_l; out_seq = se; out_slot = 0; }
+            if (ly.type == HS_LAYER_PAR) {
+                SsmArgs sa{};
+                sa.H = c.H; sa.P = c.P; sa.N = c.N; sa.di = m->di; sa.convd = m->convd; sa.in_ld = m->in_rows_max;
+                sa.zx = m->zx; sa.conv_w = ly.conv_w; sa.conv_b = ly.conv_b; sa.A_log = ly.A_log; sa.D = ly.D; sa.dt_bias = ly.dt_bias;
+                sa.win_in = win_in; sa.win_out = win_out; sa.hist = hist;
+                sa.state_in = st_in; sa.in_seq_stride = in_seq; sa.in_slot_stride = in_slot;
+                sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
+                sa.slot = m->ctrl.slot; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
+                CK(launch_ssm(sa, s), "ssm");
+            } else {
+                GdnArgs gd{};
+                gd.gh = c.gh; gd.dk = c.gdk; gd.dv = c.gdv; gd.convd = m->convd; gd.in_ld = m->in_rows_max;
+                gd.zx = m->zx; gd.conv_w = ly.conv_w; gd.conv_b = ly.conv_b; gd.onorm = ly.gnorm; gd.eps = c.eps;
+                gd.win_in = win_in; gd.win_out = win_out; gd.hist = hist;
+                gd.state_in = st_in; gd.in_seq_stride = in_seq; gd.in_slot_stride = in_slot;
+                gd.state_out = st_out; gd.out_seq_stride = out_seq; gd.out_slot_stride = out_slot;
+                gd.slot = m->ctrl.slot; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
+                CK(launch_gdn(gd, s), "gdn");
+            }
+            ++m->launches;
+        }
+        // (3) attention over the cache + the new rows (full model only)
+        if (with_attn) {
+            AttnArgs aa{};
+            aa.qh = c.qh; aa.kvh = c.kvh; aa.hd = c.hd; aa.in_ld = m->in_rows_max;
+            aa.q_off = ly.type == HS_LAYER_PAR ? ly.in_rows_draft : 0;
+            aa.k_off = aa.q_off + c.qh * c.hd; aa.v_off = aa.k_off + c.kvh * c.hd;
+            aa.zx = m->zx; aa.rope = m->rope;
+            const size_t per_layer = (size_t)m->B * c.kvh * c.kv_capacity * c.hd;
+            aa.Kc = m->Kc + ly.al * per_layer; aa.Vc = m->Vc + ly.al * per_layer; aa.cap = c.kv_capacity;
+            aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
+            aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
+            aa.chunk = m->att_chunk; aa.nch = m->att_nch; aa.T = T; aa.b0 = b0; aa.nb = nb;
+            CK(launch_attn(aa, s), "attention");
+            ++m->launches;
+        }
+        // (4) out-projection(s) + residual:  h += W_out rmsnorm_gated(g)  (+ W_o o)
+        GemvArgs go{};
+        go.O = d; go.out = m->h; go.ldo = d; go.resid = m->h; go.nrows = rows; go.epi = EPI_RESID;
+        if (ly.type == HS_LAYER_PAR) {
+            go.W0 = ly.W_out; go.ldw0 = m->di; go.K0 = m->di; go.x0 = m->gbuf; go.ldx0 = m->di; go.norm_w = ly.gnorm; go.eps = c.eps;
+            if (with_attn) { go.W1 = ly.W_o; go.ldw1 = c.qh * c.hd; go.K1 = c.qh * c.hd; go.x1 = m->obuf; go.ldx1 = c.qh * c.hd; }
+        } else if (ly.type == HS_LAYER_GDN) {
+            go.W0 = ly.W_out; go.ldw0 = m->gw; go.K0 = m->gw; go.x0 = m->gbuf; go.ldx0 = m->gw;
+        } else {
+            go.W0 = ly.W_o; go.ldw0 = c.qh * c.hd; go.K0 = c.qh * c.hd; go.x0 = m->obuf; go.ldx0 = c.qh * c.hd;
+        }
+        CK(launch_gemv(go, s, &m->launches), "out_proj");
+        // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
+        GemvArgs gu{};
+        gu.W0 = ly.W_gu; gu.ldw0 = d; gu.K0 = d; gu.x0 = m->h; gu.ldx0 = d; gu.norm_w = ly.norm2; gu.eps = c.eps;
+        gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
+        CK(launch_gemv(gu, s, &m->launches), "gate_up");
+        GemvArgs gdn{};
+        gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff;
+        gdn.O = d; gdn.out = m->h; gdn.ldo = d; gdn.resid = m->h; gdn.nrows = rows; gdn.epi = EPI_RESID;
+        CK(launch_gemv(gdn, s, &m->launches), "down");
+    }
+    // final norm + LM head, then greedy argmax
+    GemvArgs lm{};
+    lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->h; lm.ldx0 = d; lm.norm_w = m->final_norm; lm.eps = c.eps;
+    lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
+    CK(launch_gemv(lm, s, &m->launches), "lm_head");
+    if (draft) CK(launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
+    else CK(launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");
+    ++m->launches;
+    m->last_rows = rows;
+    return HS_OK;
+}
+
+int enqueue_draft(hs_model *m, int k, int b0, int nb) {
+    for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb); if (rc) return rc; }
+    return HS_OK;
+}
+
+int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const int32_t *fx) {
+    AcceptArgs a{};
+    a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd;
+    a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist;
+    CK(launch_accept(a, m->stream), "accept");
+    ++m->launches;
+    return HS_OK;
+}
+
+// Run `body` directly, or (HS_FLAG_GRAPHS) capture it once per key and replay the graph.
+template <class F>
+int run_maybe_graph(hs_model *m, uint64_t key, F body) {
+    if (!(m->c.flags & HS_FLAG_GRAPHS)) return body();
+    auto it = m->graphs.find(key);
+    if (it == m->graphs.end()) {
+        int64_t before = m->launches;
+        CK(cudaStreamBeginCapture(m->stream, cudaStreamCaptureModeThreadLocal), "begin capture");
+        int rc = body();
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(m->stream, &graph);
+        if (rc != HS_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+        if (e != cudaSuccess) return cuda_fail(m, e, "end capture");
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) return cuda_fail(m, e, "graph instantiate");
+        m->graphs[key] = exec;
+        m->graph_launches[key] = (int)(m->launches - before);
+        m->launches = before;
+        it = m->graphs.find(key);
+    }
+    CK(cudaGraphLaunch(it->second, m->stream), "graph launch");
+    m->launches += m->graph_launches[key];
+    return HS_OK;
+}
+
+int check_capacity(hs_model *m, int T, int b0, int nb) {
+    for (int b = b0; b < b0 + nb; ++b)
+        if (m->kv_upper[b] + T > m->c.kv_capacity) return fail(m, HS_ERR_CAPACITY, "kv_len + k + 1 exceeds kv_capacity");
+    return HS_OK;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+int hs_query_sizes(const hs_config *cfg, hs_sizes *out) {
+    if (!cfg || !out || !valid_config(*cfg)) return HS_ERR_INVALID_ARG;
+    const hs_config &c = *cfg;
+    Derived v = derive(c);
+    out->weights = blob_offset(c, c.L, 0);
+    out->snap = up((int64_t)4 * v.n_rl * v.B * v.Tm * v.state_elems);
+    out->dstate = up((int64_t)4 * v.n_rl * v.B * v.state_elems);
+    out->conv = up((int64_t)4 * v.n_rl * v.B * v.convd * (3 + v.Tm + 6));
+    out->kv = up((int64_t)2 * 2 * v.n_al * v.B * c.kvh * c.kv_capacity * c.hd);
+    out->work = work_layout(c, v).total;
+    return HS_OK;
+}
+
+int64_t hs_weight_offset(const hs_config *cfg, int layer, int tensor) {
+    if (!cfg || !valid_config(*cfg) || layer < -1 || layer >= cfg->L) return -1;
+    return blob_offset(*cfg, layer, tensor);
+}
+
+int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs_model **out) {
+    if (!cfg || !bufs || !out || !valid_config(*cfg)) return HS_ERR_INVALID_ARG;
+    const void *ptrs[6] = {bufs->weights, bufs->snap, bufs->dstate, bufs->conv, bufs->kv, bufs->work};
+    for (int i = 0; i < 6; ++i) if (!ptrs[i] || ((uintptr_t)ptrs[i] & (ALIGN - 1))) return HS_ERR_INVALID_ARG;
+    hs_model *m = new hs_model();
+    m->c = *cfg; m->bufs = *bufs; m->stream = (cudaStream_t)stream;
+    const hs_config &c = m->c;
+    Derived v = derive(c);
+    m->B = v.B; m->Tm = v.Tm; m->batch = 0; m->di = d_inner(c); m->convd = v.convd; m->gw = v.gw;
+    m->n_rl = v.n_rl; m->n_al = v.n_al; m->state_elems = v.state_elems; m->in_rows_max = v.in_rows_max;
+    m->att_chunk = v.att_chunk; m->att_nch = v.att_nch;
+    m->phase = 0; m->last_k = -1; m->last_rows = 0; m->launches = 0; m->capturing = false;
+    m->kv_upper.assign(v.B, 0);
+    const char *wb = (const char *)bufs->weights;
+    auto f32 = [&](int l, int t) { int64_t o = blob_offset(c, l, t); return o < 0 ? nullptr : (const float *)(wb + o); };
+    auto b16 = [&](int l, int t) { int64_t o = blob_offset(c, l, t); return o < 0 ? nullptr : (const __nv_bfloat16 *)(wb + o); };
+    m->embed = b16(-1, HS_G_EMBED); m->lm_head = b16(-1, HS_G_LM_HEAD); m->final_norm = f32(-1, HS_G_FINAL_NORM);
+    int rl = 0, al = 0;
+    for (int l = 0; l < c.L; ++l) {
+        HsLayer ly{};
+        ly.type = layer_type(c, l);
+        ly.rl = ly.type != HS_LAYER_ATT ? rl++ : -1;
+        ly.al = ly.type != HS_LAYER_GDN ? al++ : -1;
+        ly.norm1 = f32(l, HS_T_NORM1); ly.conv_w = f32(l, HS_T_CONV_W); ly.conv_b = f32(l, HS_T_CONV_B);
+        ly.A_log = f32(l, HS_T_A_LOG); ly.D = f32(l, HS_T_D); ly.dt_bias = f32(l, HS_T_DT_BIAS);
+        ly.gnorm = f32(l, HS_T_GNORM); ly.norm2 = f32(l, HS_T_NORM2);
+        ly.W_in = b16(l, HS_T_W_IN); ly.W_out = b16(l, HS_T_W_OUT); ly.W_o = b16(l, HS_T_W_O);
+        ly.W_gu = b16(l, HS_T_W_GU); ly.W_down = b16(l, HS_T_W_DOWN);
+        ly.in_rows_full = in_rows(c, ly.type, false); ly.in_rows_draft = in_rows(c, ly.type, true);
+        m->layers.push_back(ly);
+    }
+    // carve the work buffer
+    char *w = (char *)bufs->work;
+    WorkLayout wl = work_layout(c, v);
+    m->ctrl.kv_len = (int32_t *)(w + wl.kv_len); m->ctrl.slot = (int32_t *)(w + wl.slot);
+    m->ctrl.cand = (int32_t *)(w + wl.cand); m->ctrl.g = (int32_t *)(w + wl.g); m->ctrl.margin = (float *)(w + wl.margin);
+    m->ctrl.n_acc = (int32_t *)(w + wl.n_acc); m->ctrl.emitted = (int32_t *)(w + wl.emitted);
+    m->ctrl.stage_n = (int32_t *)(w + wl.stage_n); m->ctrl.stage_next = (int32_t *)(w + wl.stage_next);
+    m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters);
+    m->rope = (float2 *)(w + wl.rope);
+    m->h = (float *)(w + wl.h); m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
+    m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits);
+    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml);
+    // conv buffer: committed windows | verify history | draft ping-pong
+    float *cv = (float *)bufs->conv;
+    const size_t win = (size_t)v.n_rl * v.B * 3 * v.convd;
+    m->cw = cv; m->hist = cv + win; m->dcw = m->hist + (size_t)v.n_rl * v.B * v.Tm * v.convd;
+    m->Kc = (__nv_bfloat16 *)bufs->kv;
+    m->Vc = m->Kc + (size_t)v.n_al * v.B * c.kvh * c.kv_capacity * c.hd;
+    m->snap = (float *)bufs->snap; m->dstate = (float *)bufs->dstate;
+    *out = m;
+    CK(configure_gemv(), "configure gemv");
+    CK(configure_attn(), "configure attention");
+    // RoPE table (rotate-half pairing: pair (e, e + hd/2) turns by pos * theta^(-2e/hd)), computed in double
+    std::vector<float2> tab((size_t)c.kv_capacity * (c.hd / 2));
+    for (int e = 0; e < c.hd / 2; ++e) {
+        const double f = std::pow((double)c.rope_theta, -2.0 * e / c.hd);
+        for (int p = 0; p < c.kv_capacity; ++p) {
+            const double ang = (double)p * f;
+            tab[(size_t)p * (c.hd / 2) + e] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+        }
+    }
+    CK(cudaMemcpyAsync(m->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, m->stream), "rope upload");
+    CK(cudaMemsetAsync(w, 0, wl.rope, m->stream), "ctrl clear");
+    CK(cudaStreamSynchronize(m->stream), "init sync");
+    return HS_OK;
+}
+
+int hs_reset(hs_model *m) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    hs_sizes sz; hs_query_sizes(&m->c, &sz);
+    CK(cudaMemsetAsync(m->snap, 0, sz.snap, m->stream), "reset snap");
+    CK(cudaMemsetAsync(m->dstate, 0, sz.dstate, m->stream), "reset dstate");
+    CK(cudaMemsetAsync(m->bufs.conv, 0, sz.conv, m->stream), "reset conv");
+    CK(cudaMemsetAsync(m->bufs.work, 0, (char *)m->rope - (char *)m->bufs.work, m->stream), "reset ctrl");
+    std::fill(m->kv_upper.begin(), m->kv_upper.end(), 0);
+    m->phase = 0; m->batch = 0;
+    return HS_OK;
+}
+
+int hs_set_batch(hs_model *m, int batch) {
+    if (!m || batch < 1 || batch > m->B) return HS_ERR_INVALID_ARG;
+    m->batch = batch; m->phase = 0;
+    return HS_OK;
+}
+
+int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host, int batch) {
+    if (!m || !tokens_host || !lens_host || batch < 1 || batch > m->B) return HS_ERR_INVALID_ARG;
+    int64_t off = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (lens_host[b] < 1) return fail(m, HS_ERR_INVALID_ARG, "empty prompt");
+        if (m->kv_upper[b] + lens_host[b] > m->c.kv_capacity) return fail(m, HS_ERR_CAPACITY, "prompt exceeds kv_capacity");
+    }
+    for (int b = 0; b < batch; ++b) {
+        const int len = lens_host[b];
+        for (int p = 0; p < len; p += m->Tm) {
+            const int T = std::min(m->Tm, len - p);
+            CK(cudaMemcpyAsync(m->ctrl.cand + b * m->Tm, tokens_host + off + p, sizeof(int32_t) * T,
+                               cudaMemcpyHostToDevice, m->stream), "prefill tokens");
+            CK(cudaMemsetAsync(m->ctrl.stage_n + b, 0, 4, m->stream), "prefill stage");
+            int32_t n = T - 1;
+            CK(cudaMemcpyAsync(m->ctrl.stage_n + b, &n, 4, cudaMemcpyHostToDevice, m->stream), "prefill n");
+            int rc = model_pass(m, false, T, 0, b, 1);
+            if (rc) return rc;
+            rc = enqueue_accept(m, T - 1, b, 1, m->ctrl.stage_n, nullptr);
+            if (rc) return rc;
+            CK(cudaStreamSynchronize(m->stream), "prefill sync");   // `n` and the token slice are host temporaries
+        }
+        m->kv_upper[b] += len;
+        off += len;
+    }
+    m->batch = batch; m->phase = 0;
+    return hs_device_status(m);
+}
+
+int hs_draft(hs_model *m, int k) {
+    if (!m || k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
+    if (m->batch < 1) return fail(m, HS_ERR_ORDER, "no active sequences: prefill or set_context first");
+    if (k > 0) {
+        const int nb = m->batch;
+        int rc = run_maybe_graph(m, (1ull << 40) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
+        if (rc) return rc;
+    }
+    m->phase = 1; m->last_k = k;
+    return HS_OK;
+}
+
+int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
+    if (!m || k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
+    if (m->batch < 1) return fail(m, HS_ERR_ORDER, "no active sequences: prefill or set_context first");
+    if (!cand_dev && k > 0 && !(m->phase == 1 && m->last_k == k)) return fail(m, HS_ERR_ORDER, "verify(k) needs a preceding draft(k) or explicit candidates");
+    const int nb = m->batch, T = k + 1;
+    int rc = check_capacity(m, T, 0, nb);
+    if (rc) return rc;
+    if (cand_dev)
+        CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
+                             cudaMemcpyDeviceToDevice, m->stream), "candidates");
+    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
+    if (rc) return rc;
+    m->phase = 2; m->last_k = k;
+    return HS_OK;
+}
+
+int hs_accept_rollback(hs_model *m, const int32_t *forced_n_dev, const int32_t *forced_next_dev,
+                       int32_t *n_acc_host, int32_t *emitted_host) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    if (m->phase != 2) return fail(m, HS_ERR_ORDER, "accept_rollback needs a preceding verify");
+    const int k = m->last_k, nb = m->batch, T = k + 1;
+    int rc = enqueue_accept(m, k, 0, nb, forced_n_dev, forced_next_dev);
+    if (rc) return rc;
+    m->phase = 0;
+    for (int b = 0; b < nb; ++b) m->kv_upper[b] += T;
+    if (n_acc_host || emitted_host) {
+        std::vector<int32_t> n(nb);
+        CK(cudaMemcpyAsync(n.data(), m->ctrl.n_acc, 4 * nb, cudaMemcpyDeviceToHost, m->stream), "n_acc readback");
+        if (emitted_host)
+            CK(cudaMemcpy2DAsync(emitted_host, 4 * T, m->ctrl.emitted, 4 * m->Tm, 4 * T, nb, cudaMemcpyDeviceToHost, m->stream), "emitted readback");
+        CK(cudaStreamSynchronize(m->stream), "accept sync");
+        for (int b = 0; b < nb; ++b) { m->kv_upper[b] += n[b] + 1 - T; if (n_acc_host) n_acc_host[b] = n[b]; }
+    }
+    return HS_OK;
+}
+
+int hs_round_host(hs_model *m, int k, const int32_t *forced_n_host, const int32_t *forced_next_host,
+                  int32_t *n_acc_host, int32_t *emitted_host) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    const int nb = m->batch;
+    if (nb < 1) return fail(m, HS_ERR_ORDER, "no active sequences");
+    if (forced_n_host) CK(cudaMemcpyAsync(m->ctrl.stage_n, forced_n_host, 4 * nb, cudaMemcpyHostToDevice, m->stream), "forced_n upload");
+    if (forced_next_host) CK(cudaMemcpyAsync(m->ctrl.stage_next, forced_next_host, 4 * nb, cudaMemcpyHostToDevice, m->stream), "forced_next upload");
+    int rc = hs_draft(m, k);
+    if (rc) return rc;
+    rc = hs_verify(m, k, nullptr);
+    if (rc) return rc;
+    rc = hs_accept_rollback(m, forced_n_host ? m->ctrl.stage_n : nullptr, forced_next_host ? m->ctrl.stage_next : nullptr,
+                            n_acc_host, emitted_host);
+    if (rc) return rc;
+    if (!n_acc_host && !emitted_host) CK(cudaStreamSynchronize(m->stream), "round sync");
+    return HS_OK;
+}
+
+// ---- hooks ----------------------------------------------------------------------------------
+static int state_xfer(hs_model *m, int layer, int seq, int kind, void *host, int64_t bytes, bool to_host) {
+    if (!m || !host || layer < 0 || layer >= m->c.L || seq < 0 || seq >= m->B) return HS_ERR_INVALID_ARG;
+    const hs_config &c = m->c;
+    const HsLayer &ly = m->layers[layer];
+    const cudaMemcpyKind dir = to_host ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    if (kind == HS_STATE_SSM || kind == HS_STATE_GDN || kind == HS_STATE_DRAFT) {
+        if (ly.rl < 0) return fail(m, HS_ERR_INVALID_ARG, "layer has no recurrent state");
+        if (kind == HS_STATE_SSM && ly.type != HS_LAYER_PAR) return HS_ERR_INVALID_ARG;
+        if (kind == HS_STATE_GDN && ly.type != HS_LAYER_GDN) return HS_ERR_INVALID_ARG;
+        if (bytes != 4 * m->state_elems) return fail(m, HS_ERR_SIZE, "state size mismatch");
+        float *dev;
+        if (kind == HS_STATE_DRAFT) {
+            if (!to_host) return HS_ERR_INVALID_ARG;
+            dev = m->dstate + ((size_t)ly.rl * m->B + seq) * m->state_elems;
+        } else {
+            int32_t slot = 0;
+            if (to_host) CK(cudaMemcpy(&slot, m->ctrl.slot + seq, 4, cudaMemcpyDeviceToHost), "slot read");
+            else CK(cudaMemcpy(m->ctrl.slot + seq, &slot, 4, cudaMemcpyHostToDevice), "slot write");
+            dev = m->snap + (((size_t)ly.rl * m->B + seq) * m->Tm + slot) * m->state_elems;
+        }
+        CK(to_host ? cudaMemcpy(host, dev, bytes, dir) : cudaMemcpy(dev, host, bytes, dir), "state copy");
+        return HS_OK;
+    }
+    if (kind == HS_STATE_CONV) {
+        if (ly.rl < 0) return fail(m, HS_ERR_INVALID_ARG, "layer has no conv window");
+        if (bytes != (int64_t)4 * 3 * m->convd) return fail(m, HS_ERR_SIZE, "conv window size mismatch");
+        float *dev = m->cw + ((size_t)ly.rl * m->B + seq) * 3 * m->convd;
+        CK(to_host ? cudaMemcpy(host, dev, bytes, dir) : cudaMemcpy(dev, host, bytes, dir), "conv copy");
+        return HS_OK;
+    }
+    if (kind == HS_STATE_K || kind == HS_STATE_V) {
+        if (ly.al < 0) return fail(m, HS_ERR_INVALID_ARG, "layer has no KV cache");
+        const int64_t rowb = (int64_t)c.kvh * c.hd * 2;
+        if (bytes <= 0 || bytes % rowb) return fail(m, HS_ERR_SIZE, "KV bytes must be whole rows");
+        const int64_t rows = bytes / rowb;
+        if (rows > c.kv_capacity) return fail(m, HS_ERR_SIZE, "more rows than kv_capacity");
+        __nv_bfloat16 *base = (kind == HS_STATE_K ? m->Kc : m->Vc) + ((size_t)ly.al * m->B + seq) * c.kvh * c.kv_capacity * c.hd;
+        // device [kvh][cap][hd]  <->  host [rows][kvh][hd]
+        for (int h = 0; h < c.kvh; ++h) {
+            __nv_bfloat16 *dev = base + (size_t)h * c.kv_capacity * c.hd;
+            char *hp = (char *)host + (size_t)h * c.hd * 2;
+            if (to_host) CK(cudaMemcpy2D(hp, rowb, dev, c.hd * 2, c.hd * 2, rows, dir), "kv export");
+            else CK(cudaMemcpy2D(dev, c.hd * 2, hp, rowb, c.hd * 2, rows, dir), "kv import");
+        }
+        return HS_OK;
+    }
+    return HS_ERR_INVALID_ARG;
+}
+
+int hs_export_state(hs_model *m, int layer, int seq, int kind, void *host, int64_t bytes) {
+    return state_xfer(m, layer, seq, kind, host, bytes, true);
+}
+int hs_import_state(hs_model *m, int layer, int seq, int kind, const void *host, int64_t bytes) {
+    return state_xfer(m, layer, seq, kind, const_cast<void *>(host), bytes, false);
+}
+
+int hs_set_context(hs_model *m, int seq, int kv_len, int pending) {
+    if (!m || seq < 0 || seq >= m->B || kv_len < 0 || kv_len > m->c.kv_capacity || pending < 0 || pending >= m->c.V)
+        return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    int32_t v = kv_len, p = pending;
+    CK(cudaMemcpy(m->ctrl.kv_len + seq, &v, 4, cudaMemcpyHostToDevice), "set kv_len");
+    CK(cudaMemcpy(m->ctrl.cand + seq * m->Tm, &p, 4, cudaMemcpyHostToDevice), "set pending");
+    m->kv_upper[seq] = kv_len;
+    if (m->batch < seq + 1) m->batch = seq + 1;
+    m->phase = 0;
+    return HS_OK;
+}
+
+int hs_get_context(hs_model *m, int seq, int32_t *kv_len, int32_t *pending) {
+    if (!m || seq < 0 || seq >= m->B) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    int32_t v = 0, p = 0;
+    CK(cudaMemcpy(&v, m->ctrl.kv_len + seq, 4, cudaMemcpyDeviceToHost), "get kv_len");
+    CK(cudaMemcpy(&p, m->ctrl.cand + seq * m->Tm, 4, cudaMemcpyDeviceToHost), "get pending");
+    if (m->phase == 0) m->kv_upper[seq] = v;
+    if (kv_len) *kv_len = v;
+    if (pending) *pending = p;
+    return HS_OK;
+}
+
+int hs_get_logits(hs_model *m, float *host, int rows) {
+    if (!m || !host || rows < 1 || rows > m->last_rows) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    CK(cudaMemcpy(host, m->logits, (size_t)4 * rows * m->c.V, cudaMemcpyDeviceToHost), "logits");
+    return HS_OK;
+}
+
+int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin_host) {
+    if (!m || m->last_k < 0 || m->batch < 1) return HS_ERR_INVALID_ARG;
+    const int T = m->last_k + 1, nb = m->batch;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    if (cand_host) CK(cudaMemcpy2D(cand_host, 4 * T, m->ctrl.cand, 4 * m->Tm, 4 * T, nb, cudaMemcpyDeviceToHost), "cand");
+    if (g_host) CK(cudaMemcpy2D(g_host, 4 * T, m->ctrl.g, 4 * m->Tm, 4 * T, nb, cudaMemcpyDeviceToHost), "g");
+    if (margin_host) CK(cudaMemcpy2D(margin_host, 4 * T, m->ctrl.margin, 4 * m->Tm, 4 * T, nb, cudaMemcpyDeviceToHost), "margin");
+    return HS_OK;
+}
+
+int64_t hs_launch_count(const hs_model *m) { return m ? m->launches : -1; }
+
+int hs_device_status(hs_model *m) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "status sync");
+    int32_t st = 0;
+    CK(cudaMemcpy(&st, m->ctrl.status, 4, cudaMemcpyDeviceToHost), "status read");
+    if (st != 0) { m->err = "a kernel recorded an error in the device status word"; return st; }
+    return HS_OK;
+}
+
+const char *hs_last_error(const hs_model *m) { return m ? m->err.c_str() : "null handle"; }
+
+int hs_destroy(hs_model *m) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);
+    delete m;
+    return HS_OK;
+}
+
+}  // extern "C"

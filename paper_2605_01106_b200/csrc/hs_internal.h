@@ -1,0 +1,153 @@
+// Internal declarations shared by the translation units of libhs (host orchestration + kernels).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string>
+#include <vector>
+#include <map>
+#include "../../include/hs.h"
+
+#define HS_MAX_K 8
+#define HS_MAX_T (HS_MAX_K + 1)
+#define HS_MAX_GT 48          // (q heads per kv head) * (k+1) upper bound of the attention kernel
+
+// ---------------------------------------------------------------------------------------------
+// Control block in device memory (part of the caller's work buffer).  Everything a captured graph
+// needs that changes from round to round lives here, so the graphs themselves never change.
+// ---------------------------------------------------------------------------------------------
+struct HsCtrl {
+    int32_t *kv_len;      // [B]   consumed tokens per sequence
+    int32_t *slot;        // [B]   snapshot index that holds the committed recurrent state
+    int32_t *cand;        // [B][Tm] candidates of the current round; cand[b][0] = pending token
+    int32_t *g;           // [B][Tm] full-model argmax after candidate i
+    float *margin;        // [B][Tm] top1 - top2 of those logits
+    int32_t *n_acc;       // [B]
+    int32_t *emitted;     // [B][Tm]
+    int32_t *stage_n;     // [B]   staging for host-supplied forced accept lengths
+    int32_t *stage_next;  // [B]
+    int32_t *status;      // [1]   first error a kernel recorded
+    int32_t *counters;    // [B][kvh] split-KV arrival tickets (zero between launches)
+};
+
+struct HsLayer {
+    int type;                 // HS_LAYER_*
+    int rl;                   // ordinal among recurrent layers (PAR / GDN), else -1
+    int al;                   // ordinal among layers with a KV cache (PAR / ATT), else -1
+    const float *norm1, *conv_w, *conv_b, *A_log, *D, *dt_bias, *gnorm, *norm2;
+    const __nv_bfloat16 *W_in, *W_out, *W_o, *W_gu, *W_down;
+    int in_rows_full;         // rows of W_IN used in verify mode
+    int in_rows_draft;        // rows used in draft mode (attention rows dropped)
+};
+
+struct hs_model {
+    hs_config c;
+    hs_buffers bufs;
+    cudaStream_t stream;
+    int B, Tm;                // max_batch, max_k + 1
+    int batch;                // active sequences
+    int di, convd, gw;        // d_inner, conv channels, width of the gated mixer output
+    int n_rl, n_al;           // recurrent layers, KV layers
+    int64_t state_elems;      // floats of one (layer, seq) recurrent state
+    int in_rows_max;
+    int att_chunk, att_nch;   // keys per split, max splits
+    std::vector<HsLayer> layers;
+    const __nv_bfloat16 *embed, *lm_head;
+    const float *final_norm;
+    // carved out of bufs.work
+    HsCtrl ctrl;
+    float2 *rope;             // [cap][hd/2] (cos, sin)
+    float *h, *zx, *gbuf, *obuf, *abuf, *logits;
+    float *att_acc, *att_ml;
+    // conv buffers
+    float *cw, *hist, *dcw;
+    __nv_bfloat16 *Kc, *Vc;
+    float *snap, *dstate;
+    // host bookkeeping
+    std::vector<int> kv_upper; // upper bound of kv_len per sequence (exact after a host readback)
+    int phase;                 // 0 idle, 1 drafted, 2 verified
+    int last_k;                // k of the last draft / verify
+    int last_rows;             // rows of logits of the last pass
+    int64_t launches;
+    std::string err;
+    bool capturing;
+    std::map<uint64_t, cudaGraphExec_t> graphs;
+    std::map<uint64_t, int> graph_launches;
+};
+
+// ---------------------------------------------------------------------------------------------
+// kernel launchers (each returns the cudaError_t of the launch)
+// ---------------------------------------------------------------------------------------------
+enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
+
+struct GemvArgs {
+    // segment 0 (optionally RMS-normalised by norm_w) and optional segment 1, summed
+    const __nv_bfloat16 *W0; int ldw0; int K0; const float *x0; int ldx0; const float *norm_w; float eps;
+    const __nv_bfloat16 *W1; int ldw1; int K1; const float *x1; int ldx1;
+    int O;                    // output rows of W (for SWIGLU: 2 * outputs)
+    float *out; int ldo;      // [nrows][ldo]
+    const float *resid;       // EPI_RESID: same layout as out (may alias)
+    int nrows;                // activation rows (batch * T)
+    int epi;
+};
+cudaError_t launch_gemv(const GemvArgs &a, cudaStream_t s, int64_t *launches);
+cudaError_t configure_gemv();   // one-time kernel attributes; call outside stream capture
+cudaError_t configure_attn();
+
+cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
+                         int b0, int nb, float *h, cudaStream_t s);
+
+struct SsmArgs {
+    int H, P, N, di, convd, in_ld;      // in_ld = row stride of zx
+    const float *zx;                    // [rows][in_ld]: z | x B C | dt (| q k v)
+    const float *conv_w, *conv_b, *A_log, *D, *dt_bias;
+    const float *win_in;                // [B][3][convd] window the conv starts from
+    float *win_out;                     // draft: [B][3][convd] shifted window; verify: NULL
+    float *hist;                        // verify: [B][Tm][convd] raw inputs; draft: NULL
+    const float *state_in;              // base of the state to read; per-seq stride + optional slot
+    int64_t in_seq_stride, in_slot_stride;   // slot stride 0 => no slot indexing
+    float *state_out;                   // verify: snapshots (slot i at i*out_slot_stride); draft: scratch
+    int64_t out_seq_stride, out_slot_stride;
+    const int32_t *slot;                // [B] committed slot (used when in_slot_stride != 0)
+    float *g;                           // [rows][di] gated output y * silu(z)
+    int T, Tm, b0, nb;
+};
+cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s);
+
+struct GdnArgs {
+    int gh, dk, dv, convd, in_ld;
+    const float *zx;                    // [rows][in_ld]: q | k | v | z | a | b
+    const float *conv_w, *conv_b, *onorm; float eps;
+    const float *win_in; float *win_out; float *hist;
+    const float *state_in; int64_t in_seq_stride, in_slot_stride;
+    float *state_out; int64_t out_seq_stride, out_slot_stride;
+    const int32_t *slot;
+    float *g;                           // [rows][gh*dv]
+    int T, Tm, b0, nb;
+};
+cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s);
+
+struct AttnArgs {
+    int qh, kvh, hd, in_ld, q_off, k_off, v_off;
+    const float *zx;
+    const float2 *rope;                 // [cap][hd/2]
+    __nv_bfloat16 *Kc, *Vc;             // this layer: [B][kvh][cap][hd]
+    int cap;
+    const int32_t *kv_len;
+    float *o;                           // [rows][qh*hd]
+    float *part_acc, *part_ml; int32_t *counters; int32_t *status;
+    int chunk, nch;
+    int T, b0, nb;
+};
+cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);
+
+cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
+                          int32_t *tok_out, int tok_col0, float *margin_out, cudaStream_t s);
+
+struct AcceptArgs {
+    int k, Tm, b0, nb, n_rl, B, convd;
+    HsCtrl ctrl;
+    const int32_t *forced_n, *forced_next;
+    float *cw; const float *hist;       // [n_rl][B][3][convd], [n_rl][B][Tm][convd]
+};
+cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s);

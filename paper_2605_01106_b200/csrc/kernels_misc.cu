@@ -1,0 +1,134 @@
+// Small kernels of the round: token embedding gather, greedy argmax with top-2 margin, and the
+// accept / rollback step (paper Sec. 3.3, greedy rule).
+#include "hs_internal.h"
+
+namespace {
+
+// h[row(b,i)][:] = E[cand[b][col0 + i]]
+__global__ void embed_kernel(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
+                             int b0, float *h) {
+    const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
+    const int tok = cand[b * Tm + col0 + i];
+    const uint4 *src = reinterpret_cast<const uint4 *>(E + (size_t)tok * d);
+    float *dst = h + (size_t)(lb * T + i) * d;
+    for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
+        uint4 w = src[c];
+        float4 lo = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u),
+                                __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u));
+        float4 hi = make_float4(__uint_as_float(w.z << 16), __uint_as_float(w.z & 0xffff0000u),
+                                __uint_as_float(w.w << 16), __uint_as_float(w.w & 0xffff0000u));
+        reinterpret_cast<float4 *>(dst)[2 * c] = lo;
+        reinterpret_cast<float4 *>(dst)[2 * c + 1] = hi;
+    }
+}
+
+struct Top2 { float v1; int i1; float v2; };
+
+__device__ __forceinline__ Top2 top2_merge(const Top2 &a, const Top2 &b) {
+    // lowest index wins a tie for first place; an equal runner-up makes the margin zero
+    Top2 r;
+    if (a.v1 > b.v1 || (a.v1 == b.v1 && a.i1 < b.i1)) { r.v1 = a.v1; r.i1 = a.i1; r.v2 = fmaxf(a.v2, b.v1); }
+    else { r.v1 = b.v1; r.i1 = b.i1; r.v2 = fmaxf(b.v2, a.v1); }
+    return r;
+}
+
+// one block per logits row: token = argmax (lowest id on ties), margin = top1 - top2
+__global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V, int T, int b0, int Tm,
+                                                      int32_t *tok_out, int tok_col0, float *margin_out) {
+    const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
+    const float *row = logits + (size_t)(lb * T + i) * V;
+    Top2 t = {-INFINITY, 0x7fffffff, -INFINITY};
+    for (int j = threadIdx.x; j < V; j += blockDim.x) {
+        float v = row[j];
+        if (v > t.v1) { t.v2 = t.v1; t.v1 = v; t.i1 = j; }
+        else if (v > t.v2) t.v2 = v;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        Top2 u;
+        u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t = top2_merge(t, u);
+    }
+    __shared__ Top2 s[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    if (lane == 0) s[warp] = t;
+    __syncthreads();
+    if (warp == 0) {
+        t = lane < nw ? s[lane] : Top2{-INFINITY, 0x7fffffff, -INFINITY};
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            Top2 u;
+            u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+            u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+            u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+            t = top2_merge(t, u);
+        }
+        if (lane == 0) {
+            tok_out[b * Tm + tok_col0 + i] = t.i1;
+            if (margin_out) margin_out[b * Tm + i] = t.v1 - t.v2;
+        }
+    }
+}
+
+// Greedy acceptance and rollback.  grid = (channel chunks, max(n_rl,1), nb).
+//   n = forced_n[b], or the number of leading drafts cand[b][i+1] == g[b][i]
+//   committed conv window <- the three raw inputs that end at accepted position n
+//   block (0,0,b) also updates the control words: slot, kv_len, pending (= cand[b][0]), outputs.
+__global__ void accept_kernel(AcceptArgs a) {
+    const int lb = blockIdx.z, b = a.b0 + lb, rl = blockIdx.y;
+    const int k = a.k, Tm = a.Tm;
+    const int32_t *cand = a.ctrl.cand + b * Tm, *g = a.ctrl.g + b * Tm;
+    int n;
+    if (a.forced_n) n = min(max(a.forced_n[b], 0), k);
+    else { n = 0; while (n < k && cand[n + 1] == g[n]) ++n; }
+    int next = g[n];
+    if (a.forced_next && a.forced_next[b] >= 0) next = a.forced_next[b];
+    // conv windows: sequence of raw inputs = [w0 w1 w2 | hist_0 .. hist_k]; new window = entries n+1..n+3
+    if (rl < a.n_rl) {
+        float *cw = a.cw + ((size_t)rl * a.B + b) * 3 * a.convd;
+        const float *hist = a.hist + ((size_t)rl * a.B + b) * Tm * a.convd;
+        for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < a.convd; c += gridDim.x * blockDim.x) {
+            float v[3];
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                int e = n + 1 + j;
+                v[j] = e < 3 ? cw[e * a.convd + c] : hist[(e - 3) * a.convd + c];
+            }
+#pragma unroll
+            for (int j = 0; j < 3; ++j) cw[j * a.convd + c] = v[j];
+        }
+    }
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        int32_t *em = a.ctrl.emitted + b * Tm;
+        int d[HS_MAX_T];
+        for (int i = 0; i < k; ++i) d[i] = cand[i + 1];
+        for (int i = 0; i <= k; ++i) em[i] = i < n ? d[i] : (i == n ? next : -1);
+        a.ctrl.n_acc[b] = n;
+        a.ctrl.slot[b] = n;
+        a.ctrl.kv_len[b] += n + 1;
+        a.ctrl.cand[b * Tm] = next;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
+                         int b0, int nb, float *h, cudaStream_t s) {
+    embed_kernel<<<dim3(T, nb), 128, 0, s>>>(E, d, cand, Tm, col0, T, b0, h);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
+                          int32_t *tok_out, int tok_col0, float *margin_out, cudaStream_t s) {
+    argmax_kernel<<<dim3(T, nb), 1024, 0, s>>>(logits, V, T, b0, Tm, tok_out, tok_col0, margin_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s) {
+    int chunks = (a.convd + 255) / 256;
+    if (chunks < 1) chunks = 1;
+    accept_kernel<<<dim3(chunks, a.n_rl > 0 ? a.n_rl : 1, a.nb), 256, 0, s>>>(a);
+    return cudaGetLastError();
+}

@@ -1,0 +1,233 @@
+// Recurrent mixers of the hybrid block, for T = 1 (draft step) or T = k+1 (verify) positions:
+//   * Mamba-2 branch: causal conv (width 4) + SiLU on x|B|C, softplus(dt), the state recurrence
+//       S <- exp(dt A) S + dt x (x) B ,  y = S C + D x ,  then the gate y * silu(z)
+//   * Gated DeltaNet layer: conv + SiLU on q|k|v, L2-normalised q,k, the delta rule
+//       S <- a S ; S <- S + b (v - S k) k^T ; o = S q / sqrt(dk), per-head RMSNorm and gate.
+// The state of a (sequence, head, row strip) lives in registers for the whole kernel: it is read
+// once with 128-bit loads, advanced T times, and written after every position (verify: one
+// snapshot per position, so that rollback is an index; draft: the scratch copy).  Reductions over
+// the state dimension are warp shuffles in a fixed order.
+#include "hs_internal.h"
+#include "hs_device.cuh"
+
+namespace {
+using namespace hsd;
+
+constexpr int SSM_PR = 16;       // state rows (of P) per block
+constexpr int SSM_THREADS = 128; // 4 warps x 4 rows
+
+template <int EPL>               // floats of one state row held by a lane; N = 32 * EPL
+__global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
+    constexpr int N = 32 * EPL;
+    constexpr int VW = EPL < 4 ? EPL : 4;       // vector width of the state loads
+    constexpr int NVEC = EPL / VW;
+    constexpr int RPW = SSM_PR / (SSM_THREADS / 32);
+    __shared__ __align__(16) float Bs[HS_MAX_T][N], Cs[HS_MAX_T][N];
+    __shared__ float xs[HS_MAX_T][SSM_PR], dt_s[HS_MAX_T], a_s[HS_MAX_T];
+
+    const int p0 = blockIdx.x * SSM_PR, h = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, T = a.T;
+    const int rowbase = lb * T;
+
+    // ---- issue the state loads first: they do not depend on anything computed here
+    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
+                        (a.in_slot_stride ? (size_t)a.slot[b] * a.in_slot_stride : 0) +
+                        ((size_t)h * a.P + p0 + warp * RPW) * N;
+    float s[RPW][EPL];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v) {
+            const float *src = sin_ + r * N + v * (32 * VW) + lane * VW;
+            if (VW == 4) { float4 t = *reinterpret_cast<const float4 *>(src); s[r][v * 4] = t.x; s[r][v * 4 + 1] = t.y; s[r][v * 4 + 2] = t.z; s[r][v * 4 + 3] = t.w; }
+            else { float2 t = *reinterpret_cast<const float2 *>(src); s[r][0] = t.x; s[r][1] = t.y; }
+        }
+
+    // ---- causal conv + SiLU for the channels this block needs: its x strip, all of B and C
+    const int nch = SSM_PR + 2 * N;
+    const bool owner = (blockIdx.x == 0 && blockIdx.y == 0);   // writes the shared B|C channels' history
+    for (int c = threadIdx.x; c < nch; c += SSM_THREADS) {
+        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+        const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
+        const float bias = a.conv_b[gc];
+        const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
+        float w0 = win[0], w1 = win[a.convd], w2 = win[2 * a.convd];
+        const bool wr = c < SSM_PR || owner;
+        for (int i = 0; i < T; ++i) {
+            const float raw = a.zx[(size_t)(rowbase + i) * a.in_ld + a.di + gc];
+            const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
+            w0 = w1; w1 = w2; w2 = raw;
+            if (c < SSM_PR) xs[i][c] = act;
+            else if (c < SSM_PR + N) Bs[i][c - SSM_PR] = act;
+            else Cs[i][c - SSM_PR - N] = act;
+            if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+        }
+        if (wr && a.win_out) {
+            float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
+            wo[0] = w0; wo[a.convd] = w1; wo[2 * a.convd] = w2;
+        }
+    }
+    if (threadIdx.x < T) {
+        const float dt = softplus_f(a.zx[(size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h] + a.dt_bias[h]);
+        dt_s[threadIdx.x] = dt;
+        a_s[threadIdx.x] = expf(-dt * expf(a.A_log[h]));
+    }
+    __syncthreads();
+
+    // ---- recurrence over the T positions
+    const float Dh = a.D[h];
+    float *sout = a.state_out + (size_t)b * a.out_seq_stride + ((size_t)h * a.P + p0 + warp * RPW) * N;
+    for (int i = 0; i < T; ++i) {
+        const float dec = a_s[i], dt = dt_s[i];
+        float Bv[EPL], Cv[EPL];
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v)
+#pragma unroll
+            for (int j = 0; j < VW; ++j) {
+                Bv[v * VW + j] = Bs[i][v * (32 * VW) + lane * VW + j];
+                Cv[v * VW + j] = Cs[i][v * (32 * VW) + lane * VW + j];
+            }
+        float acc[RPW];
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const float dtx = dt * xs[i][warp * RPW + r];
+            float t = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                s[r][e] = fmaf(dec, s[r][e], dtx * Bv[e]);
+                t = fmaf(s[r][e], Cv[e], t);
+            }
+            acc[r] = t;
+        }
+        const float y = xreduce<RPW>(acc, lane);           // lanes l with l / (32/RPW) == r hold row r
+        constexpr int LPV = 32 / RPW;
+        if ((lane & (LPV - 1)) == 0) {
+            const int r = lane / LPV, col = h * a.P + p0 + warp * RPW + r;
+            const float z = a.zx[(size_t)(rowbase + i) * a.in_ld + col];
+            a.g[(size_t)(rowbase + i) * a.di + col] = (y + Dh * xs[i][warp * RPW + r]) * silu_f(z);
+        }
+        // state after position i (verify: snapshot i; draft: the scratch state)
+        float *dst = sout + (size_t)i * a.out_slot_stride;
+#pragma unroll
+        for (int r = 0; r < RPW; ++r)
+#pragma unroll
+            for (int v = 0; v < NVEC; ++v) {
+                float *p = dst + r * N + v * (32 * VW) + lane * VW;
+                if (VW == 4) *reinterpret_cast<float4 *>(p) = make_float4(s[r][v * 4], s[r][v * 4 + 1], s[r][v * 4 + 2], s[r][v * 4 + 3]);
+                else *reinterpret_cast<float2 *>(p) = make_float2(s[r][0], s[r][1]);
+            }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+constexpr int GDN_THREADS = 256;   // 8 warps x 8 value rows; key dim 64 = 32 lanes x 2
+
+__global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
+    constexpr int DK = 64, RPW = 8;
+    __shared__ __align__(16) float qs[HS_MAX_T][DK], ks[HS_MAX_T][DK];
+    __shared__ float vs[HS_MAX_T][64], os[HS_MAX_T][64], al[HS_MAX_T], be[HS_MAX_T];
+    const int h = blockIdx.x, lb = blockIdx.y, b = a.b0 + lb, T = a.T, dv = a.dv;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, rowbase = lb * T;
+    const int nk = a.gh * DK, nv = a.gh * dv;
+
+    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
+                        (a.in_slot_stride ? (size_t)a.slot[b] * a.in_slot_stride : 0) + (size_t)h * dv * DK;
+    float s[RPW][2];
+    const bool rows_ok = warp * RPW < dv;
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+        float2 t = rows_ok ? *reinterpret_cast<const float2 *>(sin_ + (warp * RPW + r) * DK + 2 * lane) : make_float2(0.f, 0.f);
+        s[r][0] = t.x; s[r][1] = t.y;
+    }
+    // conv + SiLU on this head's q, k, v channels
+    for (int c = threadIdx.x; c < 2 * DK + dv; c += GDN_THREADS) {
+        const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
+        const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
+        const float bias = a.conv_b[gc];
+        const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
+        float w0 = win[0], w1 = win[a.convd], w2 = win[2 * a.convd];
+        for (int i = 0; i < T; ++i) {
+            const float raw = a.zx[(size_t)(rowbase + i) * a.in_ld + gc];
+            const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
+            w0 = w1; w1 = w2; w2 = raw;
+            if (c < DK) qs[i][c] = act; else if (c < 2 * DK) ks[i][c - DK] = act; else vs[i][c - 2 * DK] = act;
+            if (a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+        }
+        if (a.win_out) {
+            float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
+            wo[0] = w0; wo[a.convd] = w1; wo[2 * a.convd] = w2;
+        }
+    }
+    if (threadIdx.x < T) {
+        const float *row = a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld;
+        al[threadIdx.x] = sigmoid_f(row[2 * nk + 2 * nv + h]);
+        be[threadIdx.x] = sigmoid_f(row[2 * nk + 2 * nv + a.gh + h]);
+    }
+    __syncthreads();
+    // L2-normalise q and k of every position (one warp per vector)
+    for (int t = warp; t < 2 * T; t += GDN_THREADS / 32) {
+        float *vec = t < T ? qs[t] : ks[t - T];
+        float x0 = vec[2 * lane], x1 = vec[2 * lane + 1];
+        float inv = rsqrtf(warp_sum(x0 * x0 + x1 * x1) + 1e-6f);
+        vec[2 * lane] = x0 * inv; vec[2 * lane + 1] = x1 * inv;
+    }
+    __syncthreads();
+
+    float *sout = a.state_out + (size_t)b * a.out_seq_stride + (size_t)h * dv * DK;
+    constexpr int LPV = 32 / RPW;
+    for (int i = 0; i < T; ++i) {
+        const float alpha = al[i], beta = be[i];
+        const float k0 = ks[i][2 * lane], k1 = ks[i][2 * lane + 1], q0 = qs[i][2 * lane], q1 = qs[i][2 * lane + 1];
+        float part[RPW];
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            s[r][0] *= alpha; s[r][1] *= alpha;
+            part[r] = fmaf(s[r][0], k0, s[r][1] * k1);
+        }
+        const float rk = xreduce<RPW>(part, lane);          // S' k for row lane / LPV
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const float rr = __shfl_sync(0xffffffffu, rk, r * LPV);
+            const float u = beta * ((rows_ok ? vs[i][warp * RPW + r] : 0.f) - rr);
+            s[r][0] = fmaf(u, k0, s[r][0]); s[r][1] = fmaf(u, k1, s[r][1]);
+            part[r] = fmaf(s[r][0], q0, s[r][1] * q1);
+        }
+        const float o = xreduce<RPW>(part, lane);
+        if (rows_ok && (lane & (LPV - 1)) == 0) os[i][warp * RPW + lane / LPV] = o * 0.125f;   // 1/sqrt(64)
+        if (rows_ok) {
+            float *dst = sout + (size_t)i * a.out_slot_stride;
+#pragma unroll
+            for (int r = 0; r < RPW; ++r)
+                *reinterpret_cast<float2 *>(dst + (warp * RPW + r) * DK + 2 * lane) = make_float2(s[r][0], s[r][1]);
+        }
+    }
+    __syncthreads();
+    // per-head RMSNorm over dv, then the output gate silu(z)
+    for (int i = warp; i < T; i += GDN_THREADS / 32) {
+        float ss = 0.f;
+        for (int j = lane; j < dv; j += 32) ss = fmaf(os[i][j], os[i][j], ss);
+        const float rstd = rsqrtf(warp_sum(ss) / (float)dv + a.eps);
+        const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
+        for (int j = lane; j < dv; j += 32) {
+            const float z = row[2 * nk + nv + h * dv + j];
+            a.g[(size_t)(rowbase + i) * nv + h * dv + j] = os[i][j] * rstd * a.onorm[j] * silu_f(z);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
+    dim3 grid(a.P / SSM_PR, a.H, a.nb);
+    if (a.N == 64) ssm_kernel<2><<<grid, SSM_THREADS, 0, s>>>(a);
+    else if (a.N == 128) ssm_kernel<4><<<grid, SSM_THREADS, 0, s>>>(a);
+    else if (a.N == 256) ssm_kernel<8><<<grid, SSM_THREADS, 0, s>>>(a);
+    else return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s) {
+    if (a.dk != 64 || a.dv > 64 || (a.dv & 7)) return cudaErrorInvalidValue;
+    gdn_kernel<<<dim3(a.gh, a.nb), GDN_THREADS, 0, s>>>(a);
+    return cudaGetLastError();
+}

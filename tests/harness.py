@@ -1,0 +1,142 @@
+"""Round-by-round comparison of the CUDA library with the CPU oracle on the same seeded inputs.
+
+Tolerances (from the benchmark spec): token ids, accept lengths and KV/state indices bit-exact wherever the
+oracle's top-2 logit margin exceeds 1e-2 (narrower positions are listed, and the GPU is re-synchronised to
+the oracle there); logits within 2e-2 absolute; recurrent states within 1e-3 of the state's magnitude.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+import hs_inputs as hi
+import oracle
+from paper_2605_01106_b200 import binding as hs
+
+MARGIN = 1e-2
+LOGIT_TOL = 2e-2
+STATE_TOL = 1e-3
+
+
+class Report:
+    def __init__(self):
+        self.listed = []          # (round, seq, phase, position, margin)
+        self.n_hist = {}
+        self.max_logit_err = 0.0
+        self.max_state_err = 0.0
+        self.rounds = 0
+        self.tokens = 0
+
+    def __repr__(self):
+        return "Report(rounds=%d tokens=%d listed=%d n_hist=%s max_logit_err=%.2e max_state_err=%.2e)" % (
+            self.rounds, self.tokens, len(self.listed), dict(sorted(self.n_hist.items())), self.max_logit_err,
+            self.max_state_err)
+
+
+def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
+    """Committed recurrent state, conv window and KV rows of every sequence against the oracle."""
+    worst = 0.0
+    for b, o in enumerate(seqs):
+        kv_len, pending = eng.get_context(b)
+        assert kv_len == o.len, ("kv_len", b, kv_len, o.len)
+        assert pending == o.pending, ("pending", b, pending, o.pending)
+        ssm, gdn, conv = o.ssm(), o.gdn(), o.conv()
+        for l in range(shape.L):
+            t = shape.layer_type(l)
+            if t != hi.LAYER_ATT:
+                want = ssm[l] if t == hi.LAYER_PAR else gdn[l]      # the oracle indexes its arrays by layer
+                got = eng.export_state(l, b, hs.STATE_SSM if t == hi.LAYER_PAR else hs.STATE_GDN)
+                err = np.abs(got - want).max() / max(np.abs(want).max(), 1e-30)
+                assert err <= STATE_TOL, ("state", l, b, err)
+                worst = max(worst, err)
+                gotc = eng.export_state(l, b, hs.STATE_CONV)
+                errc = np.abs(gotc - conv[l]).max() / max(np.abs(conv[l]).max(), 1e-30)
+                assert errc <= STATE_TOL, ("conv", l, b, errc)
+        n = o.len if kv_rows is None else min(kv_rows, o.len)
+        for l in range(shape.L):
+            if shape.layer_type(l) == hi.LAYER_GDN or n == 0:
+                continue
+            for kind, ref in ((hs.STATE_K, o.k()), (hs.STATE_V, o.v())):
+                got = hi.bf16_to_f32(eng.export_state(l, b, kind, rows=o.len)[-n:]).astype(np.float64)
+                want = hi.bf16_to_f32(ref[l, o.len - n:o.len]).astype(np.float64)
+                # bf16 rows: equal up to one rounding step of the larger magnitude
+                assert (np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-3).all(), ("kv", l, b, kind)
+                assert (got == want).mean() > 0.9, ("kv exact fraction", l, b, kind, (got == want).mean())
+    if rep is not None:
+        rep.max_state_err = max(rep.max_state_err, worst)
+    return worst
+
+
+def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_every=1, check_logits=True,
+               torch=None):
+    """seqs: oracle sequences, one per active GPU sequence, already holding the same context.
+    forced: None (real acceptance) or int array [batch][rounds] of forced accept lengths."""
+    import torch as _torch
+    torch = torch or _torch
+    rep = rep or Report()
+    B, T, V = len(seqs), k + 1, shape.V
+    dev = eng.device
+    for r in range(rounds):
+        # ---- oracle: draft (with logits, for the margins), then the whole round on those candidates
+        ora = []
+        for b, o in enumerate(seqs):
+            if k > 0:
+                d, dlg = o.draft_only(k, want_logits=True)
+                dm = np.array([oracle.argmax_margin(dlg[i])[1] for i in range(k)])
+            else:
+                d, dm = np.zeros(0, np.int32), np.zeros(0)
+            cand = np.concatenate([[o.pending], d]).astype(np.int32)
+            fn = -1 if forced is None else int(forced[b][r])
+            res = o.round(k, cand_in=cand, forced_n=fn, want_logits=check_logits)
+            res["draft_margin"] = dm
+            ora.append(res)
+        # ---- GPU draft; candidates must agree where the oracle's draft margin is wide
+        eng.draft(k)
+        eng.last_k = k
+        # get_round reads cand before verify: phase is 'drafted'
+        gc, _, _ = eng.get_round(k)
+        resync = False
+        for b in range(B):
+            for i in range(T):
+                if gc[b, i] != ora[b]["cand"][i]:
+                    m = ora[b]["draft_margin"][i - 1] if i > 0 else np.inf
+                    assert m <= MARGIN, ("draft token differs at a wide margin", r, b, i, m, gc[b], ora[b]["cand"])
+                    rep.listed.append((r, b, "draft", i, float(m)))
+                    resync = True
+                    break
+        cand_all = np.stack([o["cand"] for o in ora]).astype(np.int32)
+        eng.verify(k, torch.from_numpy(cand_all).to(dev) if resync else None)
+        gc, gg, gm = eng.get_round(k)
+        assert np.array_equal(gc, cand_all)
+        force_accept = resync
+        for b in range(B):
+            for i in range(T):
+                if gg[b, i] != ora[b]["g"][i]:
+                    m = ora[b]["margin"][i]
+                    assert m <= MARGIN, ("verify argmax differs at a wide margin", r, b, i, m)
+                    rep.listed.append((r, b, "verify", i, float(m)))
+                    force_accept = True
+        if check_logits:
+            lg = eng.get_logits(B * T).reshape(B, T, V)
+            for b in range(B):
+                err = np.abs(lg[b] - ora[b]["logits"]).max()
+                assert err <= LOGIT_TOL, ("logits", r, b, err)
+                rep.max_logit_err = max(rep.max_logit_err, float(err))
+        # ---- accept / rollback (forced to the oracle's decision when the pattern is forced or a listed
+        #      narrow-margin position made the GPU's own decision differ)
+        fn_dev = fx_dev = None
+        if forced is not None or force_accept:
+            fn_dev = torch.tensor([o["n"] for o in ora], dtype=torch.int32, device=dev)
+        if force_accept:
+            fx_dev = torch.tensor([int(o["emitted"][-1]) for o in ora], dtype=torch.int32, device=dev)
+        n, em = eng.accept_rollback(fn_dev, fx_dev, readback=True)
+        for b in range(B):
+            assert n[b] == ora[b]["n"], ("accept length", r, b, n[b], ora[b]["n"])
+            want = ora[b]["emitted"]
+            assert np.array_equal(em[b, : n[b] + 1], want), ("emitted", r, b, em[b], want)
+            assert (em[b, n[b] + 1:] == -1).all()
+            rep.n_hist[int(n[b])] = rep.n_hist.get(int(n[b]), 0) + 1
+            rep.tokens += int(n[b]) + 1
+        rep.rounds += 1
+        if check_states_every and (r % check_states_every == 0 or r == rounds - 1):
+            compare_states(eng, seqs, shape, rep, kv_rows=2 * T + 2)
+    return rep
