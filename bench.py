@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative decode round (draft k steps -> verify k+1 -> accept/rollback).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME] [--k K]
+
+A step is one round over the synthetic workload (default: the 0.5B-class parallel hybrid, batch 1,
+512-token prompt, seeded geometric accept pattern with per-token success 0.68).  Rank 0 prints one
+JSON line.  With N > 1 every rank runs an independent replica (sequences are independent; there is
+no collective on the data path) and the value is the sum over replicas divided by the slowest.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import hs_inputs as hi  # noqa: E402
+
+METRIC = "decode tokens/s at k=2 (seeded accept)"
+UNIT = "tokens/s"
+ALPHA = 0.68
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic bytes of one step: every used weight once, recurrent state read + written once,
+# KV rows read once + T rows appended, logits written (snapshot copies beyond the first are overhead)
+# ------------------------------------------------------------------------------------------------
+def step_bytes(s, draft: bool, T: int, kv_len: float, batch: int = 1) -> float:
+    w = 0.0          # weight bytes, shared by the batch
+    per_seq = 0.0
+    for l in range(s.L):
+        t = s.layer_type(l)
+        if draft and t == hi.LAYER_ATT:
+            continue
+        attn_rows = (s.qh + 2 * s.kvh) * s.hd
+        mlp = 3 * s.ff * s.d
+        if t == hi.LAYER_PAR:
+            rows = 2 * s.d_inner + 2 * s.N + s.H + (0 if draft else attn_rows)
+            w += 2 * (rows * s.d + s.d * s.d_inner + (0 if draft else s.d * s.qh * s.hd) + mlp)
+            w += 4 * (2 * s.d + s.convd * 5 + 3 * s.H + s.d_inner)
+            per_seq += 2 * 4 * s.H * s.P * s.N + 2 * 4 * 3 * s.convd
+        elif t == hi.LAYER_GDN:
+            rows = 2 * s.gh * s.gdk + 2 * s.gh * s.gdv + 2 * s.gh
+            w += 2 * (rows * s.d + s.d * s.gh * s.gdv + mlp) + 4 * (2 * s.d + s.convd * 5 + s.gdv)
+            per_seq += 2 * 4 * s.gh * s.gdv * s.gdk + 2 * 4 * 3 * s.convd
+        else:
+            w += 2 * (attn_rows * s.d + s.d * s.qh * s.hd + mlp) + 4 * 2 * s.d
+        if not draft and t != hi.LAYER_GDN:
+            per_seq += 2 * 2 * s.kvh * s.hd * (kv_len + T)          # K and V rows read + appended
+    w += 2 * s.V * s.d + 4 * s.d                                      # LM head + final norm
+    per_seq += T * (2 * s.d + 4 * s.V)                                # embedding rows, logits
+    return w + batch * per_seq
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx, self.rows, self.proc = gpu_index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------------
+def cpu_oracle_rate(s, blob, table, k, budget_s=15.0, max_rounds=24, prompt_len=32):
+    """tokens/s of the oracle, as it stands, on the host cores, on a bounded sample."""
+    import oracle
+    model = oracle.Model(s, blob, table, prompt_len + (max_rounds + 2) * (k + 1) + 8)
+    q = model.new_seq()
+    q.prefill(hi.make_prompt(s.V, prompt_len))
+    forced = hi.forced_accept(k, max_rounds + 1)
+    q.round(k, forced_n=int(forced[0]))                  # warm-up round
+    t0 = time.perf_counter(); toks = 0; r = 0
+    while r < max_rounds and (time.perf_counter() - t0 < budget_s or r < 2):
+        res = q.round(k, forced_n=int(forced[r + 1]))
+        toks += res["n"] + 1; r += 1
+    dt = time.perf_counter() - t0
+    return toks / dt, r, dt, prompt_len
+
+
+def run_reference(args):
+    """The reference arm of this build is the CPU oracle, timed as it stands on the host cores."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    s = hi.CONFIGS[args.config]
+    blob, table = hi.make_weights(s, 0, "unit")
+    import oracle
+    k, plen = args.k, 32
+    model = oracle.Model(s, blob, table, plen + (args.steps + args.warmup + 2) * (k + 1) + 8)
+    q = model.new_seq()
+    q.prefill(hi.make_prompt(s.V, plen))
+    forced = hi.forced_accept(k, args.steps + args.warmup)
+    for r in range(args.warmup):
+        q.round(k, forced_n=int(forced[r]))
+    t0 = time.perf_counter(); toks = 0
+    for r in range(args.steps):
+        toks += q.round(k, forced_n=int(forced[args.warmup + r]))["n"] + 1
+    dt = time.perf_counter() - t0
+    val = toks / dt
+    cores = len(os.sched_getaffinity(0))
+    sample = "%s shape, batch 1, %d-token prompt, %d rounds at k=%d, forced accept pattern" % (s.name, plen, args.steps, k)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC.replace("k=2", "k=%d" % k), "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": s.name, "k": k, "batch": 1, "prompt_len": plen, "alpha": ALPHA},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    from paper_2605_01106_b200 import binding as hs
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    s = hi.CONFIGS[args.config]
+    B = s.batch if args.batch is None else args.batch
+    ks = [args.k] + [k for k in s.ks if k != args.k and args.all_k]
+    max_k = max(max(ks), 1)
+    blob, table = hi.make_weights(s, 0, "unit")
+    steps, warm = args.steps, max(args.warmup, 3)
+    cap = s.prompt_len + (steps + warm + 4) * (max_k + 1) * 2 + 64
+    eng = hs.Engine(s, blob, max_batch=B, max_k=max_k, kv_capacity=cap, flags=hs.HS_FLAG_GRAPHS, device=str(dev))
+    prompts = [hi.make_prompt(s.V, s.prompt_len, seq=b) for b in range(B)]
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def fresh_context():
+        eng.reset()
+        eng.prefill(prompts)
+
+    def timed_rounds(k):
+        """Device-resident loop: W warm-up + K timed rounds; returns dict of timings."""
+        fresh_context()
+        forced = np.stack([hi.forced_accept(k, warm + steps, seq=b) for b in range(B)], axis=1)   # [rounds][B]
+        f_dev = torch.from_numpy(np.ascontiguousarray(forced)).to(dev)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        for r in range(warm):
+            eng.draft(k); eng.verify(k); eng.accept_rollback(f_dev[r], wait=False)
+        barrier()
+        l0 = eng.launch_count()
+        for r in range(steps):
+            e = ev[r]
+            e[0].record(eng.stream)
+            eng.draft(k)
+            e[1].record(eng.stream)
+            eng.verify(k)
+            e[2].record(eng.stream)
+            eng.accept_rollback(f_dev[warm + r], wait=False)
+            e[3].record(eng.stream)
+        barrier()
+        total_ms = ev[0][0].elapsed_time(ev[-1][3])
+        d_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / steps
+        v_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+        a_ms = sum(e[2].elapsed_time(e[3]) for e in ev) / steps
+        toks = int((forced[warm:] + 1).sum())
+        assert eng.device_status() == 0
+        kv_mid = s.prompt_len + float((forced + 1).sum(axis=0).mean()) * (warm + steps / 2) / (warm + steps)
+        return dict(total_ms=total_ms, draft_ms=d_ms, verify_ms=v_ms, accept_ms=a_ms, tokens=toks,
+                    launches=eng.launch_count() - l0, kv_mid=kv_mid)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    results = {k: timed_rounds(k) for k in ks}
+    clocks = sampler.stop() if rank == 0 else None
+    main = results[args.k]
+    total_ms = max_over_ranks(main["total_ms"])
+    value = world * main["tokens"] / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (H2D of the accept pattern, D2H of results)
+    k = args.k
+    fresh_context()
+    forced = np.stack([hi.forced_accept(k, warm + steps, seq=b) for b in range(B)], axis=1).astype(np.int32)
+    pinned = torch.from_numpy(np.ascontiguousarray(forced)).pin_memory().numpy()
+    for r in range(warm):
+        eng.round_host(k, forced_n=pinned[r])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(eng.stream)
+    toks_e2e = 0
+    for r in range(steps):
+        n, em = eng.round_host(k, forced_n=pinned[warm + r])
+        toks_e2e += int(n.sum()) + B
+    e1.record(eng.stream)
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    e2e_val = world * toks_e2e / (e2e_ms * 1e-3)
+
+    # ---- dominant kernel (projection GEMV family): live event timing of every launch
+    fresh_context()
+    f_dev = torch.from_numpy(np.ascontiguousarray(forced)).to(dev)
+    eng.profile(True)
+    for r in range(min(steps, 10)):
+        eng.draft(k); eng.verify(k); eng.accept_rollback(f_dev[r])
+    prof = eng.profile_read()
+    eng.profile(False)
+    peak, peak_src = measured_peak()
+    g_ms, g_n, g_bytes = prof["gemv"]
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "gemv_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get("dram_bytes_per_launch")
+        except Exception:
+            traffic = None
+    achieved = (g_bytes / g_n) / (g_ms / g_n * 1e-3) / 1e9 if g_n else 0.0
+    roofline = {"bound": "hbm", "kernel": "gemv_kernel (all projections)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": traffic,
+                "launches_timed": g_n, "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
+                "algorithmic_bytes_per_launch": g_bytes / max(g_n, 1),
+                "time_share": {kk: v[0] for kk, v in prof.items()}}
+
+    if rank != 0:
+        return
+    # ---- step-level roofline: algorithmic bytes / event time
+    step_roof = {}
+    for kk, r in results.items():
+        db, vb = step_bytes(s, True, 1, 0, B), step_bytes(s, False, kk + 1, r["kv_mid"], B)
+        d_step_ms = r["draft_ms"] / max(kk, 1)
+        step_roof[str(kk)] = {
+            "tokens_per_s": world * r["tokens"] / (r["total_ms"] * 1e-3), "ms_per_round": r["total_ms"] / steps,
+            "draft_step_ms": d_step_ms, "verify_step_ms": r["verify_ms"], "accept_ms": r["accept_ms"],
+            "draft_step_GBps": db / (d_step_ms * 1e-3) / 1e9 if kk else None, "verify_step_GBps": vb / (r["verify_ms"] * 1e-3) / 1e9,
+            "draft_frac_of_measured_peak": db / (d_step_ms * 1e-3) / 1e9 / peak if kk else None,
+            "verify_frac_of_measured_peak": vb / (r["verify_ms"] * 1e-3) / 1e9 / peak,
+            "draft_bytes": db, "verify_bytes": vb}
+    out = {
+        "metric": METRIC.replace("k=2", "k=%d" % args.k), "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": s.name, "k": args.k, "batch": B, "prompt_len": s.prompt_len, "alpha": ALPHA,
+                   "weights": "bf16", "state": "f32", "kv": "bf16", "cuda_graphs": True,
+                   "l2": "inputs larger than L2 (every step streams %.2f GB of weights)" % (step_bytes(s, True, 1, 0, B) / 1e9),
+                   "parallelism": "replicas x%d (no collective)" % world},
+        "clocks": clocks,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 4 * B, "d2h_bytes_per_step": 4 * B * (k + 2),
+                "ms_per_step": e2e_ms / steps},
+        "gpu_launches": int(main["launches"]),
+        "roofline": roofline,
+        "by_k": step_roof,
+    }
+    if world == 1 and not args.no_cpu:
+        val, rounds, dt, plen = cpu_oracle_rate(s, blob, table, args.k)
+        out["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                               "sample": "%s shape, batch 1, %d-token prompt, %d rounds at k=%d (%.1f s), forced accept pattern"
+                                         % (s.name, plen, rounds, args.k, dt)}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2_0p5b", choices=sorted(hi.CONFIGS))
+    ap.add_argument("--k", type=int, default=2)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--all-k", dest="all_k", action="store_true", default=True)
+    ap.add_argument("--one-k", dest="all_k", action="store_false")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

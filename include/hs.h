@@ -176,6 +176,15 @@ int hs_get_logits(hs_model *m, float *host, int rows);
 int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin_host);
 /* Number of kernels the library has launched (including those replayed inside graphs) so far. */
 int64_t hs_launch_count(const hs_model *m);
+/* Measurement hook.  hs_profile(m, 1) brackets every following kernel launch with two CUDA events on
+ * the launching stream (graph replay is bypassed while it is on); hs_profile_read synchronises and
+ * returns, per category, the summed device time in ms, the number of launches and the algorithmic
+ * bytes the library attributes to them (projections: weights once + activations in + outputs;
+ * 0 for the other categories).  Arrays have HS_PROF_COUNT entries.  hs_profile(m, 0) switches it
+ * off and drops the records. */
+enum { HS_PROF_GEMV = 0, HS_PROF_MIXER, HS_PROF_ATTN, HS_PROF_ARGMAX, HS_PROF_EMBED, HS_PROF_ACCEPT, HS_PROF_COUNT };
+int hs_profile(hs_model *m, int enable);
+int hs_profile_read(hs_model *m, double *ms, int64_t *launches, double *bytes);
 /* Device status word: 0, or the first hs_status a kernel recorded.  Synchronises. */
 int hs_device_status(hs_model *m);
 const char *hs_last_error(const hs_model *m);

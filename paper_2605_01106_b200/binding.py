@@ -19,7 +19,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_device_status", "hs_last_error", "hs_destroy"]
+           "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy"]
 
 
 class HsError(RuntimeError):
@@ -71,6 +71,8 @@ def load_library(path: str | None = None):
     L.hs_get_round.argtypes = [vp, vp, vp, vp]
     L.hs_launch_count.restype = i64
     L.hs_launch_count.argtypes = [vp]
+    L.hs_profile.argtypes = [vp, ctypes.c_int]
+    L.hs_profile_read.argtypes = [vp, vp, vp, vp]
     L.hs_device_status.argtypes = [vp]
     L.hs_last_error.restype = ctypes.c_char_p
     L.hs_last_error.argtypes = [vp]
@@ -174,14 +176,18 @@ class Engine:
         if any(t is not None for t in tensors):
             self.stream.wait_stream(self.torch.cuda.current_stream(self.device))
 
-    def verify(self, k, cand_dev=None):
-        self._after_torch(cand_dev)
+    def verify(self, k, cand_dev=None, wait=True):
+        if wait:
+            self._after_torch(cand_dev)
         self._ck(lib().hs_verify(self.h, k, _ptr(cand_dev)))
         self.last_k = k
 
-    def accept_rollback(self, forced_n_dev=None, forced_next_dev=None, readback=False):
-        """Returns (n_acc [batch], emitted [batch][k+1]) as numpy when readback, else None."""
-        self._after_torch(forced_n_dev, forced_next_dev)
+    def accept_rollback(self, forced_n_dev=None, forced_next_dev=None, readback=False, wait=True):
+        """Returns (n_acc [batch], emitted [batch][k+1]) as numpy when readback, else None.
+        wait=False skips the stream dependency on torch's current stream (the caller guarantees that
+        the device tensors are complete)."""
+        if wait:
+            self._after_torch(forced_n_dev, forced_next_dev)
         if not readback:
             self._ck(lib().hs_accept_rollback(self.h, _ptr(forced_n_dev), _ptr(forced_next_dev), None, None))
             return None
@@ -257,6 +263,18 @@ class Engine:
         c, g, m = np.empty((self.batch, T), np.int32), np.empty((self.batch, T), np.int32), np.empty((self.batch, T), np.float32)
         self._ck(lib().hs_get_round(self.h, _ptr(c), _ptr(g), _ptr(m)))
         return c, g, m
+
+    PROF_NAMES = ("gemv", "mixer", "attention", "argmax", "embed", "accept")
+
+    def profile(self, enable):
+        self._ck(lib().hs_profile(self.h, int(enable)))
+
+    def profile_read(self):
+        """{category: (ms, launches, algorithmic bytes)} accumulated since profile(True)."""
+        n = len(self.PROF_NAMES)
+        ms, cnt, by = np.zeros(n), np.zeros(n, np.int64), np.zeros(n)
+        self._ck(lib().hs_profile_read(self.h, _ptr(ms), _ptr(cnt), _ptr(by)))
+        return {k: (float(ms[i]), int(cnt[i]), float(by[i])) for i, k in enumerate(self.PROF_NAMES)}
 
     def launch_count(self):
         return lib().hs_launch_count(self.h)

@@ -153,6 +153,24 @@ int cuda_fail(hs_model *m, cudaError_t e, const char *where) {
 }
 #define CK(call, where) do { cudaError_t e__ = (call); if (e__ != cudaSuccess) return cuda_fail(m, e__, where); } while (0)
 
+// Per-kernel timing (measurement hook): when enabled, every launch is bracketed by two events on the
+// launching stream; hs_profile_read sums the elapsed times per category.
+void prof_mark(hs_model *m, int cat, bool begin, double bytes) {
+    if (!m->prof) return;
+    cudaEvent_t ev;
+    if (cudaEventCreate(&ev) != cudaSuccess) return;
+    cudaEventRecord(ev, m->stream);
+    if (begin) m->prof_events.push_back({cat, ev, nullptr, 0.0});
+    else { m->prof_events.back().stop = ev; m->prof_events.back().bytes = bytes; }
+}
+#define PROF(cat, bytes, call, where) do { prof_mark(m, cat, true, 0); CK(call, where); prof_mark(m, cat, false, bytes); } while (0)
+
+double gemv_bytes(const GemvArgs &a) {
+    // weights once (bf16) + activation rows in (fp32) + outputs (fp32; residual read as well)
+    const double Kt = (double)a.K0 + a.K1, outs = a.epi == EPI_SWIGLU ? a.O / 2 : a.O;
+    return (double)a.O * Kt * 2 + (double)a.nrows * Kt * 4 + (double)a.nrows * outs * 4 * (a.epi == EPI_RESID ? 2 : 1);
+}
+
 // ------------------------------------------------------------------------------------------------
 // one pass of the model over T positions per sequence (sequences b0 .. b0+nb-1)
 //   draft = false: full model M_H (verify);  draft = true: draft model M_S, one position,
@@ -163,7 +181,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
-    CK(launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->h, s), "embed");
+    PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->h, s), "embed");
     ++m->launches;
     for (int l = 0; l < c.L; ++l) {
         const HsLayer &ly = m->layers[l];
@@ -174,7 +192,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         GemvArgs ga{};
         ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->h; ga.ldx0 = d; ga.norm_w = ly.norm1; ga.eps = c.eps;
         ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
-        CK(launch_gemv(ga, s, &m->launches), "in_proj");
+        PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, s, &m->launches), "in_proj");
         // (2) recurrent mixer
         if (ly.type != HS_LAYER_ATT) {
             const size_t lrB = (size_t)ly.rl * m->B;
@@ -198,7 +216,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
                 sa.state_in = st_in; sa.in_seq_stride = in_seq; sa.in_slot_stride = in_slot;
                 sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
                 sa.slot = m->ctrl.slot; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
-                CK(launch_ssm(sa, s), "ssm");
+                PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
             } else {
                 GdnArgs gd{};
                 gd.gh = c.gh; gd.dk = c.gdk; gd.dv = c.gdv; gd.convd = m->convd; gd.in_ld = m->in_rows_max;
@@ -207,7 +225,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
                 gd.state_in = st_in; gd.in_seq_stride = in_seq; gd.in_slot_stride = in_slot;
                 gd.state_out = st_out; gd.out_seq_stride = out_seq; gd.out_slot_stride = out_slot;
                 gd.slot = m->ctrl.slot; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
-                CK(launch_gdn(gd, s), "gdn");
+                PROF(HS_PROF_MIXER, 0, launch_gdn(gd, s), "gdn");
             }
             ++m->launches;
         }
@@ -223,7 +241,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
             aa.chunk = m->att_chunk; aa.nch = m->att_nch; aa.T = T; aa.b0 = b0; aa.nb = nb;
-            CK(launch_attn(aa, s), "attention");
+            PROF(HS_PROF_ATTN, 0, launch_attn(aa, s), "attention");
             ++m->launches;
         }
         // (4) out-projection(s) + residual:  h += W_out rmsnorm_gated(g)  (+ W_o o)
@@ -237,24 +255,24 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         } else {
             go.W0 = ly.W_o; go.ldw0 = c.qh * c.hd; go.K0 = c.qh * c.hd; go.x0 = m->obuf; go.ldx0 = c.qh * c.hd;
         }
-        CK(launch_gemv(go, s, &m->launches), "out_proj");
+        PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, s, &m->launches), "out_proj");
         // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
         GemvArgs gu{};
         gu.W0 = ly.W_gu; gu.ldw0 = d; gu.K0 = d; gu.x0 = m->h; gu.ldx0 = d; gu.norm_w = ly.norm2; gu.eps = c.eps;
         gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
-        CK(launch_gemv(gu, s, &m->launches), "gate_up");
+        PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, s, &m->launches), "gate_up");
         GemvArgs gdn{};
         gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff;
         gdn.O = d; gdn.out = m->h; gdn.ldo = d; gdn.resid = m->h; gdn.nrows = rows; gdn.epi = EPI_RESID;
-        CK(launch_gemv(gdn, s, &m->launches), "down");
+        PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, s, &m->launches), "down");
     }
     // final norm + LM head, then greedy argmax
     GemvArgs lm{};
     lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->h; lm.ldx0 = d; lm.norm_w = m->final_norm; lm.eps = c.eps;
     lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
-    CK(launch_gemv(lm, s, &m->launches), "lm_head");
-    if (draft) CK(launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
-    else CK(launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");
+    PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, s, &m->launches), "lm_head");
+    if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
+    else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");
     ++m->launches;
     m->last_rows = rows;
     return HS_OK;
@@ -269,7 +287,7 @@ int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const 
     AcceptArgs a{};
     a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd;
     a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist;
-    CK(launch_accept(a, m->stream), "accept");
+    PROF(HS_PROF_ACCEPT, 0, launch_accept(a, m->stream), "accept");
     ++m->launches;
     return HS_OK;
 }
@@ -277,7 +295,7 @@ int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const 
 // Run `body` directly, or (HS_FLAG_GRAPHS) capture it once per key and replay the graph.
 template <class F>
 int run_maybe_graph(hs_model *m, uint64_t key, F body) {
-    if (!(m->c.flags & HS_FLAG_GRAPHS)) return body();
+    if (!(m->c.flags & HS_FLAG_GRAPHS) || m->prof) return body();
     auto it = m->graphs.find(key);
     if (it == m->graphs.end()) {
         int64_t before = m->launches;
@@ -341,7 +359,7 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     m->B = v.B; m->Tm = v.Tm; m->batch = 0; m->di = d_inner(c); m->convd = v.convd; m->gw = v.gw;
     m->n_rl = v.n_rl; m->n_al = v.n_al; m->state_elems = v.state_elems; m->in_rows_max = v.in_rows_max;
     m->att_chunk = v.att_chunk; m->att_nch = v.att_nch;
-    m->phase = 0; m->last_k = -1; m->last_rows = 0; m->launches = 0; m->capturing = false;
+    m->phase = 0; m->last_k = -1; m->last_rows = 0; m->launches = 0; m->prof = false;
     m->kv_upper.assign(v.B, 0);
     const char *wb = (const char *)bufs->weights;
     auto f32 = [&](int l, int t) { int64_t o = blob_offset(c, l, t); return o < 0 ? nullptr : (const float *)(wb + o); };
@@ -613,6 +631,28 @@ int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin
 
 int64_t hs_launch_count(const hs_model *m) { return m ? m->launches : -1; }
 
+int hs_profile(hs_model *m, int enable) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "profile sync");
+    for (auto &e : m->prof_events) { cudaEventDestroy(e.start); if (e.stop) cudaEventDestroy(e.stop); }
+    m->prof_events.clear();
+    m->prof = enable != 0;
+    return HS_OK;
+}
+
+int hs_profile_read(hs_model *m, double *ms, int64_t *launches, double *bytes) {
+    if (!m || !ms || !launches || !bytes) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "profile sync");
+    for (int i = 0; i < HS_PROF_COUNT; ++i) { ms[i] = 0; launches[i] = 0; bytes[i] = 0; }
+    for (auto &e : m->prof_events) {
+        if (!e.stop) continue;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, e.start, e.stop) != cudaSuccess) continue;
+        ms[e.cat] += t; launches[e.cat] += 1; bytes[e.cat] += e.bytes;
+    }
+    return HS_OK;
+}
+
 int hs_device_status(hs_model *m) {
     if (!m) return HS_ERR_INVALID_ARG;
     CK(cudaStreamSynchronize(m->stream), "status sync");
@@ -627,6 +667,7 @@ const char *hs_last_error(const hs_model *m) { return m ? m->err.c_str() : "null
 int hs_destroy(hs_model *m) {
     if (!m) return HS_ERR_INVALID_ARG;
     for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);
+    for (auto &e : m->prof_events) { cudaEventDestroy(e.start); if (e.stop) cudaEventDestroy(e.stop); }
     delete m;
     return HS_OK;
 }

@@ -70,7 +70,9 @@ struct hs_model {
     int last_rows;             // rows of logits of the last pass
     int64_t launches;
     std::string err;
-    bool capturing;
+    bool prof;                 // per-kernel event timing enabled
+    struct ProfEvent { int cat; cudaEvent_t start, stop; double bytes; };
+    std::vector<ProfEvent> prof_events;
     std::map<uint64_t, cudaGraphExec_t> graphs;
     std::map<uint64_t, int> graph_launches;
 };
