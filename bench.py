@@ -179,6 +179,8 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     s = hi.CONFIGS[args.config]
+    if args.prompt_len is not None:
+        s = s.replace(prompt_len=args.prompt_len)
     B = s.batch if args.batch is None else args.batch
     ks = [args.k] + [k for k in s.ks if k != args.k and args.all_k]
     max_k = max(max(ks), 1)
@@ -335,6 +337,7 @@ def main():
     ap.add_argument("--config", default="cfg2_0p5b", choices=sorted(hi.CONFIGS))
     ap.add_argument("--k", type=int, default=2)
     ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (profiling runs)")
     ap.add_argument("--all-k", dest="all_k", action="store_true", default=True)
     ap.add_argument("--one-k", dest="all_k", action="store_false")
     ap.add_argument("--no-cpu", action="store_true")

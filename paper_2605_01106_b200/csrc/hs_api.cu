@@ -131,7 +131,7 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.stage_n = take(4 * v.B); w.stage_next = take(4 * v.B);
     w.status = take(4); w.counters = take((int64_t)4 * v.B * c.kvh);
     w.rope = take((int64_t)c.kv_capacity * (c.hd / 2) * 8);
-    w.h = take((int64_t)4 * v.R * c.d);
+    w.h = take((int64_t)4 * 2 * HS_H_PARTS * v.R * c.d);
     w.zx = take((int64_t)4 * v.R * v.in_rows_max);
     w.gbuf = take((int64_t)4 * v.R * v.gw);
     w.obuf = take((int64_t)4 * v.R * c.qh * c.hd);
@@ -181,7 +181,12 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
-    PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->h, s), "embed");
+    // the residual stream ping-pongs between two buffers; a projection that splits its reduction
+    // leaves it as `hparts` partial sums, which every consumer adds in order
+    int cur = 0, hparts = 1;
+    const int64_t hps = (int64_t)m->B * m->Tm * d;
+    int32_t *st_w = m->ctrl.status;
+    PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->hbuf[0], s), "embed");
     ++m->launches;
     for (int l = 0; l < c.L; ++l) {
         const HsLayer &ly = m->layers[l];
@@ -190,9 +195,10 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         const int inr = draft ? ly.in_rows_draft : ly.in_rows_full;
         // (1) RMSNorm + in-projection (verify: Mamba rows and q|k|v rows in one pass over u)
         GemvArgs ga{};
-        ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->h; ga.ldx0 = d; ga.norm_w = ly.norm1; ga.eps = c.eps;
+        ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->hbuf[cur]; ga.ldx0 = d; ga.xparts = hparts; ga.xpstride = hps;
+        ga.norm_w = ly.norm1; ga.eps = c.eps;
         ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
-        PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, s, &m->launches), "in_proj");
+        PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, st_w, s, &m->launches, nullptr), "in_proj");
         // (2) recurrent mixer
         if (ly.type != HS_LAYER_ATT) {
             const size_t lrB = (size_t)ly.rl * m->B;
@@ -246,7 +252,8 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         }
         // (4) out-projection(s) + residual:  h += W_out rmsnorm_gated(g)  (+ W_o o)
         GemvArgs go{};
-        go.O = d; go.out = m->h; go.ldo = d; go.resid = m->h; go.nrows = rows; go.epi = EPI_RESID;
+        go.O = d; go.out = m->hbuf[cur ^ 1]; go.ldo = d; go.opstride = hps; go.max_oparts = HS_H_PARTS;
+        go.resid = m->hbuf[cur]; go.rparts = hparts; go.rpstride = hps; go.nrows = rows; go.epi = EPI_RESID; go.xparts = 1;
         if (ly.type == HS_LAYER_PAR) {
             go.W0 = ly.W_out; go.ldw0 = m->di; go.K0 = m->di; go.x0 = m->gbuf; go.ldx0 = m->di; go.norm_w = ly.gnorm; go.eps = c.eps;
             if (with_attn) { go.W1 = ly.W_o; go.ldw1 = c.qh * c.hd; go.K1 = c.qh * c.hd; go.x1 = m->obuf; go.ldx1 = c.qh * c.hd; }
@@ -255,22 +262,27 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         } else {
             go.W0 = ly.W_o; go.ldw0 = c.qh * c.hd; go.K0 = c.qh * c.hd; go.x0 = m->obuf; go.ldx0 = c.qh * c.hd;
         }
-        PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, s, &m->launches), "out_proj");
+        PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, st_w, s, &m->launches, &hparts), "out_proj");
+        cur ^= 1;
         // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
         GemvArgs gu{};
-        gu.W0 = ly.W_gu; gu.ldw0 = d; gu.K0 = d; gu.x0 = m->h; gu.ldx0 = d; gu.norm_w = ly.norm2; gu.eps = c.eps;
+        gu.W0 = ly.W_gu; gu.ldw0 = d; gu.K0 = d; gu.x0 = m->hbuf[cur]; gu.ldx0 = d; gu.xparts = hparts; gu.xpstride = hps;
+        gu.norm_w = ly.norm2; gu.eps = c.eps;
         gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
-        PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, s, &m->launches), "gate_up");
+        PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, st_w, s, &m->launches, nullptr), "gate_up");
         GemvArgs gdn{};
-        gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff;
-        gdn.O = d; gdn.out = m->h; gdn.ldo = d; gdn.resid = m->h; gdn.nrows = rows; gdn.epi = EPI_RESID;
-        PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, s, &m->launches), "down");
+        gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff; gdn.xparts = 1;
+        gdn.O = d; gdn.out = m->hbuf[cur ^ 1]; gdn.ldo = d; gdn.opstride = hps; gdn.max_oparts = HS_H_PARTS;
+        gdn.resid = m->hbuf[cur]; gdn.rparts = hparts; gdn.rpstride = hps; gdn.nrows = rows; gdn.epi = EPI_RESID;
+        PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, st_w, s, &m->launches, &hparts), "down");
+        cur ^= 1;
     }
     // final norm + LM head, then greedy argmax
     GemvArgs lm{};
-    lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->h; lm.ldx0 = d; lm.norm_w = m->final_norm; lm.eps = c.eps;
+    lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->hbuf[cur]; lm.ldx0 = d; lm.xparts = hparts; lm.xpstride = hps;
+    lm.norm_w = m->final_norm; lm.eps = c.eps;
     lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
-    PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, s, &m->launches), "lm_head");
+    PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
     if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
     else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");
     ++m->launches;
@@ -388,7 +400,7 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     m->ctrl.stage_n = (int32_t *)(w + wl.stage_n); m->ctrl.stage_next = (int32_t *)(w + wl.stage_next);
     m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters);
     m->rope = (float2 *)(w + wl.rope);
-    m->h = (float *)(w + wl.h); m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
+    m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
     m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits);
     m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml);
     // conv buffer: committed windows | verify history | draft ping-pong

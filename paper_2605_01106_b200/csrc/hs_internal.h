@@ -10,6 +10,7 @@
 
 #define HS_MAX_K 8
 #define HS_MAX_T (HS_MAX_K + 1)
+#define HS_H_PARTS 4          // a projection may leave the residual stream as up to 4 partial sums
 #define HS_MAX_GT 48          // (q heads per kv head) * (k+1) upper bound of the attention kernel
 
 // ---------------------------------------------------------------------------------------------
@@ -57,7 +58,8 @@ struct hs_model {
     // carved out of bufs.work
     HsCtrl ctrl;
     float2 *rope;             // [cap][hd/2] (cos, sin)
-    float *h, *zx, *gbuf, *obuf, *abuf, *logits;
+    float *hbuf[2];            // residual stream, ping-pong; each [HS_H_PARTS][B*Tm][d] partial sums
+    float *zx, *gbuf, *obuf, *abuf, *logits;
     float *att_acc, *att_ml;
     // conv buffers
     float *cw, *hist, *dcw;
@@ -80,19 +82,39 @@ struct hs_model {
 // ---------------------------------------------------------------------------------------------
 // kernel launchers (each returns the cudaError_t of the launch)
 // ---------------------------------------------------------------------------------------------
+// Every kernel of a step is launched with programmatic stream serialization: it may start while its
+// predecessor still runs and synchronises with griddepcontrol.wait (see hs_device.cuh).
+extern bool g_hs_pdl;
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = g_hs_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 
 struct GemvArgs {
-    // segment 0 (optionally RMS-normalised by norm_w) and optional segment 1, summed
-    const __nv_bfloat16 *W0; int ldw0; int K0; const float *x0; int ldx0; const float *norm_w; float eps;
+    // out[r][o] = sum_j W0[o][j] x0[r][j] (+ sum_j W1[o][j] x1[r][j]); x0 optionally RMS-normalised by norm_w.
+    // x0 may be given as `xparts` partial sums (part p at x0 + p * xpstride), added in order.
+    const __nv_bfloat16 *W0; int ldw0; int K0; const float *x0; int ldx0; int xparts; int64_t xpstride;
+    const float *norm_w; float eps;
     const __nv_bfloat16 *W1; int ldw1; int K1; const float *x1; int ldx1;
     int O;                    // output rows of W (for SWIGLU: 2 * outputs)
-    float *out; int ldo;      // [nrows][ldo]
-    const float *resid;       // EPI_RESID: same layout as out (may alias)
-    int nrows;                // activation rows (batch * T)
+    float *out; int ldo;      // [nrows][ldo]; EPI_RESID may write several parts, opstride floats apart
+    int64_t opstride; int max_oparts;
+    const float *resid; int rparts; int64_t rpstride;   // EPI_RESID: residual = sum of rparts parts, laid out like out
+    int nrows;                // activation rows (batch * T), at most 16 per launch
     int epi;
+    const void *pf_ptr; int64_t pf_bytes;   // optional: weights of the next projection, prefetched into L2
+    int early_trigger;        // 1: let the next kernel start before this one has waited for its predecessor
+                              // (allowed only if that kernel touches nothing but weights before its own wait)
 };
-cudaError_t launch_gemv(const GemvArgs &a, cudaStream_t s, int64_t *launches);
+// *oparts receives the number of parts written to `out` (1 unless EPI_RESID split the reduction).
+cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
 cudaError_t configure_gemv();   // one-time kernel attributes; call outside stream capture
 cudaError_t configure_attn();
 

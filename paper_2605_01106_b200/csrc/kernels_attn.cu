@@ -36,7 +36,9 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(AttnArgs a) {
 
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int len = a.kv_len[b];
+    pdl_wait();
+    pdl_trigger();
+    const int len = __ldcg(a.kv_len + b);
     const int nch = max(1, (len + a.chunk - 1) / a.chunk);
     if (split >= nch) return;
     if (len + T > a.cap) {             // never write past the cache; the host reports the status word
@@ -53,7 +55,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(AttnArgs a) {
         const int gq = qi / T, i = qi - gq * T;
         const float *src = a.zx + (size_t)(rowbase + i) * a.in_ld + a.q_off + (kh * G + gq) * HD;
         const float2 cs = a.rope[(size_t)(len + i) * (HD / 2) + e];
-        const float x0 = src[e], x1 = src[e + HD / 2];
+        const float x0 = __ldcg(src + e), x1 = __ldcg(src + e + HD / 2);
         q_s[qi * HD + e] = (x0 * cs.x - x1 * cs.y) * scale;
         q_s[qi * HD + e + HD / 2] = (x1 * cs.x + x0 * cs.y) * scale;
     }
@@ -66,11 +68,11 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(AttnArgs a) {
             const int i = idx / (HD / 2), e = idx - i * (HD / 2);
             const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
             const float2 cs = a.rope[(size_t)(len + i) * (HD / 2) + e];
-            const float x0 = row[a.k_off + kh * HD + e], x1 = row[a.k_off + kh * HD + e + HD / 2];
+            const float x0 = __ldcg(row + a.k_off + kh * HD + e), x1 = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
             const __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * cs.x - x1 * cs.y);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(row[a.v_off + kh * HD + e]);
-            const __nv_bfloat16 v1 = __float2bfloat16_rn(row[a.v_off + kh * HD + e + HD / 2]);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
+            const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
             Kn_s[i * KSTR + e] = k0; Kn_s[i * KSTR + e + HD / 2] = k1;
             Vn_s[i * KSTR + e] = v0; Vn_s[i * KSTR + e + HD / 2] = v1;
             Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
@@ -209,8 +211,7 @@ cudaError_t configure_attn() {
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     dim3 grid(a.nch, a.kvh, a.nb);
-    if (a.hd == 128) attn_kernel<128><<<grid, AT_THREADS, attn_smem<128>(), s>>>(a);
-    else if (a.hd == 64) attn_kernel<64><<<grid, AT_THREADS, attn_smem<64>(), s>>>(a);
-    else return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    if (a.hd == 128) return launch_pdl(attn_kernel<128>, grid, dim3(AT_THREADS), attn_smem<128>(), s, a);
+    if (a.hd == 64) return launch_pdl(attn_kernel<64>, grid, dim3(AT_THREADS), attn_smem<64>(), s, a);
+    return cudaErrorInvalidValue;
 }

@@ -1,17 +1,45 @@
-// Skinny projection kernels: out[r][o] = sum_j W[o][j] * x[r][j] for a handful of activation rows r
-// (batch * (k+1)), bf16 weights streamed once from HBM, fp32 activations and accumulation.
+// Skinny projection kernel (CUDA cores): out[r][o] = sum_j W[o][j] * x[r][j] for a handful of
+// activation rows r (batch * (k+1) <= 16), bf16 weights streamed exactly once from HBM, fp32
+// activations and accumulation.  Every weight byte is used only `rows` times, so the kernel is
+// HBM-bound and its job is to keep the weight stream running through the dependency stalls of a
+// decode step:
 //
-// The work is HBM-bound (every weight byte is used R <= 9 times), so it runs on the CUDA cores:
-// a warp owns WR consecutive weight rows and walks the K dimension with 128-bit streaming loads;
-// the R activation rows (after an optional fused RMSNorm) sit in shared memory and are re-used by
-// all WR rows; the WR*R partial sums of a lane are combined with a transposing shuffle reduction
-// (WR*R - 1 shuffles instead of 5 per value, fixed order -> bit-reproducible).
-// Epilogues: plain store, residual add, SwiGLU over interleaved gate/up rows.
+//  * The weight matrix is cut into one tile per CTA - a contiguous range of output rows times a
+//    range of the reduction dimension (a "K split"; only the residual epilogue may split K, its
+//    partial sums are written as separate parts that the consumer adds in a fixed order, so the
+//    result is bit-reproducible and needs no atomics).  grid = one CTA per SM.
+//  * A CTA streams its tile through a ring of shared-memory stages filled by bulk asynchronous
+//    copies (one per weight row, completion counted on an mbarrier).  The first stages are issued
+//    BEFORE the programmatic-dependent-launch wait: they depend on nothing the previous kernel
+//    computes, so the next kernel's weights are already on their way into shared memory while the
+//    current kernel is still running.
+//  * After the wait the activation rows are staged in shared memory (summing the parts of the
+//    producer, with the optional RMSNorm weight folded in; the 1/rms factor is a per-row scalar and
+//    is applied in the epilogue), and 8 warps consume the stages: a warp owns 8 weight rows and an
+//    interleaved set of 256-column blocks, keeps 8*R accumulators, and reduces them with one
+//    transposing shuffle reduction.
+// Epilogues: plain store, residual add (with K split), SwiGLU over interleaved gate/up rows.
 #include "hs_internal.h"
 #include "hs_device.cuh"
 
 namespace {
 using namespace hsd;
+
+constexpr int GV_WARPS = 8;
+constexpr int GV_THREADS = GV_WARPS * 32;
+constexpr int GV_MAXROWS = 16;      // activation rows per launch
+constexpr int GV_MAXDEPTH = 4;
+
+struct GemvGeo {
+    int S0, S1;          // K splits of segment 0 / 1
+    int kr0, kr1;        // nominal K-range width per split (multiple of 256; the last may be shorter)
+    int NR;              // row ranges; grid = NR * (S0 + S1)
+    int unit;            // row ranges start on multiples of this (2 for the SwiGLU epilogue)
+    int kc;              // columns per tile (multiple of 256): a K range is walked in chunks of kc
+    int D;               // tiles in flight per warp (depth of each warp's private ring)
+    int krmax;           // max(kr0, kr1): row stride of the staged activations
+    int off_x, off_ring; // shared-memory carve-up (bytes)
+};
 
 __device__ __forceinline__ float dot8(const uint4 &w, const float4 &a, const float4 &b, float acc) {
     acc = fmaf(bf_lo(w.x), a.x, acc); acc = fmaf(bf_hi(w.x), a.y, acc);
@@ -21,151 +49,291 @@ __device__ __forceinline__ float dot8(const uint4 &w, const float4 &a, const flo
     return acc;
 }
 
-template <int R, int WR>
-__global__ void __launch_bounds__(256) gemv_kernel(GemvArgs a) {
-    constexpr int NV = pow2_ge(R * WR);
-    extern __shared__ __align__(16) float smem[];
-    const int Kt = a.K0 + a.K1;
-    const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float *x_s = smem;                    // [R][Kt]
-    float *res_s = smem + R * Kt;         // [nw][32]
-    float *rstd_s = res_s + nw * 32;      // [R]
+// Position of activation column c (a multiple of 4) inside its staged row.  Within every block of 256
+// columns the lane that owns columns 8l..8l+7 finds its first four floats at 4l and the next four at
+// 128 + 4l, so that both 128-bit reads of a warp are contiguous (no bank conflicts).
+__device__ __forceinline__ int xs_pos(int c) {
+    const int within = c & 255;
+    return (c & ~255) + ((within >> 2) & 1) * 128 + (within >> 3) * 4;
+}
 
-    for (int rb = 0; rb < a.nrows; rb += R) {
-        const int nr = min(R, a.nrows - rb);
-        // ---- stage the activation rows (zero rows beyond nr)
-        const int q4 = Kt >> 2, q0 = a.K0 >> 2;
-        for (int idx = threadIdx.x; idx < R * q4; idx += blockDim.x) {
-            int r = idx / q4, c = idx - r * q4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (r < nr) {
-                if (c < q0) v = *reinterpret_cast<const float4 *>(a.x0 + (size_t)(rb + r) * a.ldx0 + 4 * c);
-                else v = *reinterpret_cast<const float4 *>(a.x1 + (size_t)(rb + r) * a.ldx1 + 4 * (c - q0));
-            }
-            *reinterpret_cast<float4 *>(x_s + r * Kt + 4 * c) = v;
-        }
-        __syncthreads();
-        if (a.norm_w) {
-            // fused RMSNorm of segment 0: x <- x * rsqrt(mean(x^2) + eps) * w
-            for (int r = warp; r < R; r += nw) {
-                float ss = 0.f;
-                for (int j = lane; j < a.K0; j += 32) { float t = x_s[r * Kt + j]; ss = fmaf(t, t, ss); }
+// R activation rows per pass in registers, WR weight rows per warp tile.
+// A tile is WR weight rows x kc columns; warp w owns the row groups w, w + 8, ... of the CTA's row
+// range and walks each group's K chunks in order through a private ring of D tile buffers, so the
+// main loop needs no block-wide synchronisation.
+template <int R, int WR>
+__global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
+    constexpr int NV = pow2_ge(WR * R);
+    constexpr int LPV = 32 / NV;
+    extern __shared__ __align__(128) unsigned char smraw[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smraw);                 // [8][D]
+    float *rstd_s = reinterpret_cast<float *>(smraw + 256);               // [16]
+    float *ss_s = rstd_s + GV_MAXROWS;                                    // [8][16]
+    float *x_s = reinterpret_cast<float *>(smraw + g.off_x);              // [nrows][krmax]
+    __nv_bfloat16 *ring = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_ring);   // [8][D][WR][kc]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int S = g.S0 + g.S1;
+    const int ri = blockIdx.x / S, si = blockIdx.x - ri * S;
+    const bool seg1 = si >= g.S0;
+    const __nv_bfloat16 *W = seg1 ? a.W1 : a.W0;
+    const int ld = seg1 ? a.ldw1 : a.ldw0, Kseg = seg1 ? a.K1 : a.K0;
+    const int krn = seg1 ? g.kr1 : g.kr0;
+    const int k0 = (seg1 ? si - g.S0 : si) * krn;
+    const int kr = min(krn, Kseg - k0);
+    const int units = a.O / g.unit;
+    const int r0 = (int)((long long)ri * units / g.NR) * g.unit;
+    const int r1 = (int)((long long)(ri + 1) * units / g.NR) * g.unit;
+    const int nrow = r1 - r0;
+    const int kc = g.kc, D = g.D, krmax = g.krmax;
+    const int nch = (kr + kc - 1) / kc;
+    const int ngrp = (nrow + WR - 1) / WR;
+    const int mygrps = warp < ngrp ? (ngrp - warp + GV_WARPS - 1) / GV_WARPS : 0;
+    const int ntile = mygrps * nch;
+    uint64_t *mybar = bars + warp * D;
+    __nv_bfloat16 *mybuf = ring + (size_t)warp * D * WR * kc;
+
+    auto issue_tile = [&](int t) {         // whole warp
+        const int gi = t / nch, ch = t - gi * nch;
+        const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
+        const int rows_in = min(WR, r1 - row0);
+        const int cw = min(kc, kr - ch * kc);
+        const int buf = t % D;
+        if (lane == 0) mbar_expect_tx(&mybar[buf], (uint32_t)rows_in * cw * 2);
+        __syncwarp();
+        if (lane < rows_in)
+            bulk_g2s(mybuf + ((size_t)buf * WR + lane) * kc, W + (size_t)(row0 + lane) * ld + k0 + ch * kc,
+                     (uint32_t)cw * 2, &mybar[buf]);
+    };
+
+    // ---- prologue, independent of the previous kernel: start the weight stream
+    if (a.early_trigger) pdl_trigger();
+    if (tid < GV_WARPS * D) { mbar_init(&bars[tid], 1); mbar_fence_init(); }
+    __syncthreads();
+    {
+        const int pre = min(D, ntile);
+        for (int t = 0; t < pre; ++t) issue_tile(t);
+    }
+    // pull the next projection's weights towards L2: by the time its own kernel asks for them the
+    // HBM latency is already paid
+    if (a.pf_bytes > 0 && warp == GV_WARPS - 1) {
+        const long long per = ((a.pf_bytes / gridDim.x) + 15) & ~15ll;
+        const long long lo = (long long)blockIdx.x * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+        for (long long o = lo + (long long)lane * 8192; o < hi; o += 32 * 8192)
+            prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
+    }
+    pdl_wait();
+    if (!a.early_trigger) pdl_trigger();
+
+    // ---- stage the activation rows of this K range (parts summed, norm weight folded in)
+    const bool normed = a.norm_w != nullptr && !seg1;
+    const int nrows = a.nrows;
+    {
+        const float *xsrc = seg1 ? a.x1 : a.x0;
+        const int ldx = seg1 ? a.ldx1 : a.ldx0;
+        const int parts = seg1 ? 1 : a.xparts;
+        const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
+        for (int rbase = 0; rbase < nrows; rbase += 4) {
+            float ss[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
+                float4 v[4];
 #pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                if (lane == 0) rstd_s[r] = rsqrtf(ss / (float)a.K0 + a.eps);
+                for (int j = 0; j < 4; ++j) {              // all loads of the four rows are in flight together
+                    v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (rbase + j < nrows) {
+                        const float *p = xsrc + (size_t)(rbase + j) * ldx + c;
+                        v[j] = __ldcg(reinterpret_cast<const float4 *>(p));
+                        for (int q = 1; q < parts; ++q) {
+                            const float4 u = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
+                            v[j].x += u.x; v[j].y += u.y; v[j].z += u.z; v[j].w += u.w;
+                        }
+                    }
+                }
+                const bool inside = c >= k0 && c < k0 + kr;
+                float4 nw = make_float4(1.f, 1.f, 1.f, 1.f);
+                if (normed && inside) nw = *reinterpret_cast<const float4 *>(a.norm_w + c);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (rbase + j >= nrows) continue;
+                    ss[j] = fmaf(v[j].x, v[j].x, fmaf(v[j].y, v[j].y, fmaf(v[j].z, v[j].z, fmaf(v[j].w, v[j].w, ss[j]))));
+                    if (inside)
+                        *reinterpret_cast<float4 *>(x_s + (size_t)(rbase + j) * krmax + xs_pos(c - k0)) =
+                            make_float4(v[j].x * nw.x, v[j].y * nw.y, v[j].z * nw.z, v[j].w * nw.w);
+                }
             }
-            __syncthreads();
-            for (int idx = threadIdx.x; idx < R * a.K0; idx += blockDim.x) {
-                int r = idx / a.K0, j = idx - r * a.K0;
-                x_s[r * Kt + j] *= rstd_s[r] * a.norm_w[j];
+            if (normed) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float t = warp_sum(ss[j]);
+                    if (lane == 0 && rbase + j < nrows) ss_s[warp * GV_MAXROWS + rbase + j] = t;
+                }
             }
-            __syncthreads();
         }
-        // ---- stream the weights
-        for (int og = (blockIdx.x * nw + warp) * WR; og < a.O; og += gridDim.x * nw * WR) {
+    }
+    __syncthreads();
+
+    // which result this lane holds after the transposing reduction: value v = (r, w)
+    const int vidx = lane / LPV, vr = vidx / WR, vw = vidx - vr * WR;
+    const bool holder = (lane & (LPV - 1)) == 0 && vidx < WR * R;
+    bool bad = false;
+    for (int gi = 0; gi < mygrps; ++gi) {
+        const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
+        const int rows_in = min(WR, r1 - row0);
+        for (int p0 = 0; p0 < nrows; p0 += R) {
+            // residual of the value this lane will own: in flight while the tile is reduced
+            float res = 0.f;
+            const bool live = holder && p0 + vr < nrows && vw < rows_in;
+            const size_t oi = (size_t)(p0 + vr) * a.ldo + row0 + vw;
+            if (a.epi == EPI_RESID && si == 0 && live)
+                for (int q = 0; q < a.rparts; ++q) res += __ldcg(a.resid + (size_t)q * a.rpstride + oi);
             float acc[NV];
 #pragma unroll
             for (int i = 0; i < NV; ++i) acc[i] = 0.f;
-#pragma unroll
-            for (int seg = 0; seg < 2; ++seg) {
-                const __nv_bfloat16 *W = seg ? a.W1 : a.W0;
-                const int K = seg ? a.K1 : a.K0, ld = seg ? a.ldw1 : a.ldw0, koff = seg ? a.K0 : 0;
-                if (K == 0) continue;
-                const __nv_bfloat16 *wrow[WR];
-#pragma unroll
-                for (int w = 0; w < WR; ++w) wrow[w] = W + (size_t)min(og + w, a.O - 1) * ld;
-#pragma unroll 2
-                for (int kc = lane * 8; kc < K; kc += 256) {
+            for (int ch = 0; ch < nch; ++ch) {
+                const int t = gi * nch + ch, buf = t % D;
+                if (p0 == 0 && !__all_sync(0xffffffffu, mbar_wait(&mybar[buf], (uint32_t)(t / D) & 1u))) { bad = true; break; }
+                const __nv_bfloat16 *tile = mybuf + (size_t)buf * WR * kc;
+                const int nb = min(kc, kr - ch * kc) >> 8;
+                for (int blk = 0; blk < nb; ++blk) {
+                    const int col = (blk << 8) + lane * 8;
                     uint4 wv[WR];
 #pragma unroll
-                    for (int w = 0; w < WR; ++w) wv[w] = ldg_stream(wrow[w] + kc);
+                    for (int w = 0; w < WR; ++w) wv[w] = *reinterpret_cast<const uint4 *>(tile + (size_t)w * kc + col);
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        const float4 xa = *reinterpret_cast<const float4 *>(x_s + r * Kt + koff + kc);
-                        const float4 xb = *reinterpret_cast<const float4 *>(x_s + r * Kt + koff + kc + 4);
+                        const float *xr = x_s + (size_t)min(p0 + r, nrows - 1) * krmax + ch * kc + (blk << 8) + lane * 4;
+                        const float4 xa = *reinterpret_cast<const float4 *>(xr);
+                        const float4 xb = *reinterpret_cast<const float4 *>(xr + 128);
 #pragma unroll
                         for (int w = 0; w < WR; ++w) acc[r * WR + w] = dot8(wv[w], xa, xb, acc[r * WR + w]);
                     }
                 }
+                // last pass over the activation rows: this buffer is free, refill it D tiles ahead
+                if (p0 + R >= nrows) {
+                    __syncwarp();
+                    if (t + D < ntile) issue_tile(t + D);
+                }
             }
-            const float tot = xreduce<NV>(acc, lane);
-            constexpr int LPV = 32 / NV;                     // lanes that hold each value
-            if ((lane & (LPV - 1)) == 0) res_s[warp * 32 + lane / LPV] = tot;
-            __syncwarp();
-            // ---- epilogue: value index = r * WR + w
+            if (bad) break;
+            float tot = xreduce<NV>(acc, lane);
+            if (normed) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < GV_WARPS; ++w) t += ss_s[w * GV_MAXROWS + min(p0 + vr, nrows - 1)];
+                tot *= rsqrtf(t / (float)Kseg + a.eps);
+            }
             if (a.epi == EPI_SWIGLU) {
-                if (lane < nr * (WR / 2)) {
-                    int r = lane / (WR / 2), p = lane - r * (WR / 2);
-                    int o = og + 2 * p;
-                    if (o + 1 < a.O) {
-                        float gt = res_s[warp * 32 + r * WR + 2 * p], up = res_s[warp * 32 + r * WR + 2 * p + 1];
-                        a.out[(size_t)(rb + r) * a.ldo + (o >> 1)] = silu_f(gt) * up;
-                    }
-                }
-            } else {
-                if (lane < nr * WR) {
-                    int r = lane / WR, w = lane - r * WR;
-                    int o = og + w;
-                    if (o < a.O) {
-                        float v = res_s[warp * 32 + r * WR + w];
-                        size_t oi = (size_t)(rb + r) * a.ldo + o;
-                        if (a.epi == EPI_RESID) v += a.resid[oi];
-                        a.out[oi] = v;
-                    }
-                }
+                const float up = __shfl_down_sync(0xffffffffu, tot, LPV);    // value v + 1 = the up row of the pair
+                if (live && !(vw & 1)) a.out[(size_t)(p0 + vr) * a.ldo + ((row0 + vw) >> 1)] = silu_f(tot) * up;
+            } else if (live) {
+                if (a.epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = tot + res;
+                else a.out[oi] = tot;
             }
-            __syncwarp();
         }
-        __syncthreads();
+        if (bad) break;
     }
+    if (bad) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);     // a copy never landed
 }
 
-constexpr size_t GEMV_SMEM_MAX = 201 * 1024;
-
-template <int R, int WR>
-cudaError_t launch_t(const GemvArgs &a, int nw, int grid, size_t smem, cudaStream_t s) {
-    gemv_kernel<R, WR><<<grid, nw * 32, smem, s>>>(a);
-    return cudaGetLastError();
-}
+int g_sms = 148;
+constexpr size_t GV_SMEM_MAX = 200 * 1024;
+constexpr size_t GV_SMEM_PAIR = 127 * 1024;   // below this the CTA of the next kernel fits beside it
 
 template <int R, int WR>
-cudaError_t configure_t() {
-    return cudaFuncSetAttribute(gemv_kernel<R, WR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMV_SMEM_MAX);
+cudaError_t launch_rw(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
+    return launch_pdl(gemv_kernel<R, WR>, dim3(g.NR * (g.S0 + g.S1)), dim3(GV_THREADS), smem, s, a, g, status);
 }
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 }  // namespace
 
-// Opt every instantiation into large dynamic shared memory once, outside any stream capture.
 cudaError_t configure_gemv() {
-    cudaError_t e = cudaSuccess;
-#define CFG(r, w) if (e == cudaSuccess) e = configure_t<r, w>()
-    CFG(1, 2); CFG(2, 2); CFG(3, 2); CFG(4, 2); CFG(5, 2); CFG(9, 2);
-    CFG(1, 4); CFG(2, 4); CFG(3, 4); CFG(4, 4); CFG(5, 4);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (g_sms < 1) g_sms = 148;
+    // every kernel asks for the largest shared-memory carve-out, so that an SM never has to drain to
+    // re-partition L1/shared memory before a CTA of the next kernel can join the running one
+#define CFG(r, w) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<r, w>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<r, w>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+    CFG(1, 4); CFG(2, 4); CFG(3, 4); CFG(4, 4); CFG(1, 8); CFG(2, 8); CFG(3, 8); CFG(4, 8);
 #undef CFG
     return e;
 }
 
-cudaError_t launch_gemv(const GemvArgs &a, cudaStream_t s, int64_t *launches) {
-    const int Kt = a.K0 + a.K1;
-    if ((a.K0 & 255) || (a.K1 & 255) || a.O < 2 || a.nrows < 1) return cudaErrorInvalidValue;
-    // rows per pass: must fit shared memory; fewest passes, then smallest R
-    static const int cand[6] = {1, 2, 3, 4, 5, 9};
-    int R = 1, best_pass = 1 << 30;
-    for (int i = 0; i < 6; ++i) {
-        size_t bytes = (size_t)cand[i] * Kt * 4 + 8 * 32 * 4 + 64;
-        if (bytes > 200 * 1024) continue;
-        int pass = (a.nrows + cand[i] - 1) / cand[i];
-        if (pass < best_pass) { best_pass = pass; R = cand[i]; }
+// Launches the projection.  a.max_oparts > 1 allows a K split for the residual epilogue; the number
+// of parts written is returned in *oparts (1 for the other epilogues).
+cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts) {
+    // More than four activation rows are walked in passes over tiles that stay resident; when a K range
+    // is too wide for that (more than one chunk), the rows go in launches of four.
+    if (a.nrows > 4 && a.nrows <= GV_MAXROWS) {
+        const int K = a.K0 > a.K1 ? a.K0 : a.K1;
+        const bool splittable = a.epi == EPI_RESID && a.max_oparts > 1;
+        const int kr = splittable ? 1280 : K;
+        if ((splittable ? (a.K0 + a.K1 + 3) / 4 : K) > 1280 && kr > 0) {
+            for (int r = 0; r < a.nrows; r += 4) {
+                GemvArgs b = a;
+                b.nrows = a.nrows - r < 4 ? a.nrows - r : 4;
+                b.x0 = a.x0 + (size_t)r * a.ldx0;
+                if (a.x1) b.x1 = a.x1 + (size_t)r * a.ldx1;
+                b.out = a.out + (size_t)r * a.ldo;
+                if (a.resid) b.resid = a.resid + (size_t)r * a.ldo;
+                cudaError_t e = launch_gemv(b, status, s, launches, oparts);
+                if (e != cudaSuccess) return e;
+            }
+            return cudaSuccess;
+        }
     }
-    int WR = (R * 4 <= 32 && a.O >= 4096) ? 4 : 2;
-    int nw = (a.O / WR >= 148 * 8) ? 8 : 4;
-    int grid = (a.O + nw * WR - 1) / (nw * WR);
-    if (grid > 148 * 8) grid = 148 * 8;
-    size_t smem = (size_t)R * Kt * 4 + nw * 32 * 4 + 64;
+    if ((a.K0 & 255) || (a.K1 & 255) || a.K0 < 256 || a.O < 2 || a.nrows < 1 || a.nrows > GV_MAXROWS) return cudaErrorInvalidValue;
+    GemvGeo g{};
+    g.unit = a.epi == EPI_SWIGLU ? 2 : 1;
+    if (a.O % g.unit) return cudaErrorInvalidValue;
+    const int maxp = (a.epi == EPI_RESID && a.max_oparts > 1) ? (a.max_oparts < 4 ? a.max_oparts : 4) : 1;
+    // K split: ranges of about 1024 columns, at most maxp in total, aligned to the segment boundary
+    if (maxp == 1) {
+        if (a.K1) return cudaErrorInvalidValue;               // two segments need at least two parts
+        g.S0 = 1; g.S1 = 0;
+    } else {
+        for (int krt = 1024;; krt += 256) {
+            g.S0 = ceil_div(a.K0, krt); g.S1 = a.K1 ? ceil_div(a.K1, krt) : 0;
+            if (g.S0 + g.S1 <= maxp) break;
+        }
+    }
+    g.kr0 = ceil_div(ceil_div(a.K0, g.S0), 256) * 256;
+    g.kr1 = g.S1 ? ceil_div(ceil_div(a.K1, g.S1), 256) * 256 : 0;
+    g.S0 = ceil_div(a.K0, g.kr0);
+    if (g.S1) g.S1 = ceil_div(a.K1, g.kr1);
+    g.krmax = g.kr0 > g.kr1 ? g.kr0 : g.kr1;
+    const int S = g.S0 + g.S1;
+    const int units = a.O / g.unit;
+    g.NR = g_sms / S;
+    if (g.NR < 1) g.NR = 1;
+    if (g.NR > units) g.NR = units;
+    const int nrow_max = ceil_div(units, g.NR) * g.unit;
+    // tile: 4 weight rows per warp when that already gives every warp a tile, else 8
+    const int WR = nrow_max <= 4 * GV_WARPS ? 4 : 8;
+    // chunk of at most 1280 columns, as even as possible
+    const int nch = ceil_div(g.krmax, 1280);
+    g.kc = ceil_div(ceil_div(g.krmax, nch), 256) * 256;
+    const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * ceil_div(g.krmax, g.kc);
+    const size_t tile = (size_t)WR * g.kc * 2;
+    const size_t xs = (size_t)a.nrows * g.krmax * 4;
+    g.off_x = 1024;
+    g.off_ring = (int)((g.off_x + xs + 127) / 128 * 128);
+    int D = 1;
+    while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= GV_SMEM_PAIR) ++D;
+    g.D = D;
+    const int ring_warps = ceil_div(nrow_max, WR) < GV_WARPS ? ceil_div(nrow_max, WR) : GV_WARPS;
+    const size_t smem = g.off_ring + tile * ring_warps * D;
+    if (smem > GV_SMEM_MAX) return cudaErrorInvalidValue;
+    if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
     if (launches) ++*launches;
-#define CASE(r, w) if (R == r && WR == w) return launch_t<r, w>(a, nw, grid, smem, s)
-    CASE(1, 2); CASE(2, 2); CASE(3, 2); CASE(4, 2); CASE(5, 2); CASE(9, 2);
-    CASE(1, 4); CASE(2, 4); CASE(3, 4); CASE(4, 4); CASE(5, 4);
+    // rows held in registers per pass: as even as possible over ceil(nrows / 4) passes
+    const int npass = ceil_div(a.nrows, 4), R = ceil_div(a.nrows, npass);
+#define CASE(r, w) if (R == r && WR == w) return launch_rw<r, w>(a, g, smem, status, s)
+    CASE(1, 4); CASE(2, 4); CASE(3, 4); CASE(4, 4); CASE(1, 8); CASE(2, 8); CASE(3, 8); CASE(4, 8);
 #undef CASE
     return cudaErrorInvalidValue;
 }

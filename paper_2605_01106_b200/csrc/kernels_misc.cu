@@ -1,14 +1,20 @@
 // Small kernels of the round: token embedding gather, greedy argmax with top-2 margin, and the
 // accept / rollback step (paper Sec. 3.3, greedy rule).
 #include "hs_internal.h"
+#include "hs_device.cuh"
+
+bool g_hs_pdl = true;
 
 namespace {
+using namespace hsd;
 
 // h[row(b,i)][:] = E[cand[b][col0 + i]]
 __global__ void embed_kernel(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
                              int b0, float *h) {
     const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
-    const int tok = cand[b * Tm + col0 + i];
+    pdl_wait();
+    pdl_trigger();
+    const int tok = __ldcg(cand + b * Tm + col0 + i);
     const uint4 *src = reinterpret_cast<const uint4 *>(E + (size_t)tok * d);
     float *dst = h + (size_t)(lb * T + i) * d;
     for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
@@ -37,9 +43,11 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V
                                                       int32_t *tok_out, int tok_col0, float *margin_out) {
     const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
     const float *row = logits + (size_t)(lb * T + i) * V;
+    pdl_wait();
+    pdl_trigger();
     Top2 t = {-INFINITY, 0x7fffffff, -INFINITY};
     for (int j = threadIdx.x; j < V; j += blockDim.x) {
-        float v = row[j];
+        float v = __ldcg(row + j);
         if (v > t.v1) { t.v2 = t.v1; t.v1 = v; t.i1 = j; }
         else if (v > t.v2) t.v2 = v;
     }
@@ -79,12 +87,14 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V
 __global__ void accept_kernel(AcceptArgs a) {
     const int lb = blockIdx.z, b = a.b0 + lb, rl = blockIdx.y;
     const int k = a.k, Tm = a.Tm;
+    pdl_wait();
+    pdl_trigger();
     const int32_t *cand = a.ctrl.cand + b * Tm, *g = a.ctrl.g + b * Tm;
     int n;
-    if (a.forced_n) n = min(max(a.forced_n[b], 0), k);
-    else { n = 0; while (n < k && cand[n + 1] == g[n]) ++n; }
-    int next = g[n];
-    if (a.forced_next && a.forced_next[b] >= 0) next = a.forced_next[b];
+    if (a.forced_n) n = min(max(__ldcg(a.forced_n + b), 0), k);
+    else { n = 0; while (n < k && __ldcg(cand + n + 1) == __ldcg(g + n)) ++n; }
+    int next = __ldcg(g + n);
+    if (a.forced_next && __ldcg(a.forced_next + b) >= 0) next = __ldcg(a.forced_next + b);
     // conv windows: sequence of raw inputs = [w0 w1 w2 | hist_0 .. hist_k]; new window = entries n+1..n+3
     if (rl < a.n_rl) {
         float *cw = a.cw + ((size_t)rl * a.B + b) * 3 * a.convd;
@@ -94,7 +104,7 @@ __global__ void accept_kernel(AcceptArgs a) {
 #pragma unroll
             for (int j = 0; j < 3; ++j) {
                 int e = n + 1 + j;
-                v[j] = e < 3 ? cw[e * a.convd + c] : hist[(e - 3) * a.convd + c];
+                v[j] = e < 3 ? __ldcg(cw + e * a.convd + c) : __ldcg(hist + (e - 3) * a.convd + c);
             }
 #pragma unroll
             for (int j = 0; j < 3; ++j) cw[j * a.convd + c] = v[j];
@@ -103,11 +113,11 @@ __global__ void accept_kernel(AcceptArgs a) {
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
         int32_t *em = a.ctrl.emitted + b * Tm;
         int d[HS_MAX_T];
-        for (int i = 0; i < k; ++i) d[i] = cand[i + 1];
+        for (int i = 0; i < k; ++i) d[i] = __ldcg(cand + i + 1);
         for (int i = 0; i <= k; ++i) em[i] = i < n ? d[i] : (i == n ? next : -1);
         a.ctrl.n_acc[b] = n;
         a.ctrl.slot[b] = n;
-        a.ctrl.kv_len[b] += n + 1;
+        a.ctrl.kv_len[b] = __ldcg(a.ctrl.kv_len + b) + n + 1;
         a.ctrl.cand[b * Tm] = next;
     }
 }
@@ -116,19 +126,16 @@ __global__ void accept_kernel(AcceptArgs a) {
 
 cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
                          int b0, int nb, float *h, cudaStream_t s) {
-    embed_kernel<<<dim3(T, nb), 128, 0, s>>>(E, d, cand, Tm, col0, T, b0, h);
-    return cudaGetLastError();
+    return launch_pdl(embed_kernel, dim3(T, nb), dim3(128), 0, s, E, d, cand, Tm, col0, T, b0, h);
 }
 
 cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
                           int32_t *tok_out, int tok_col0, float *margin_out, cudaStream_t s) {
-    argmax_kernel<<<dim3(T, nb), 1024, 0, s>>>(logits, V, T, b0, Tm, tok_out, tok_col0, margin_out);
-    return cudaGetLastError();
+    return launch_pdl(argmax_kernel, dim3(T, nb), dim3(1024), 0, s, logits, V, T, b0, Tm, tok_out, tok_col0, margin_out);
 }
 
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s) {
     int chunks = (a.convd + 255) / 256;
     if (chunks < 1) chunks = 1;
-    accept_kernel<<<dim3(chunks, a.n_rl > 0 ? a.n_rl : 1, a.nb), 256, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(accept_kernel, dim3(chunks, a.n_rl > 0 ? a.n_rl : 1, a.nb), dim3(256), 0, s, a);
 }

@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
 
     // ---- issue the state loads first: they do not depend on anything computed here
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
-                        (a.in_slot_stride ? (size_t)a.slot[b] * a.in_slot_stride : 0) +
+                        (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) +
                         ((size_t)h * a.P + p0 + warp * RPW) * N;
     float s[RPW][EPL];
 #pragma unroll
@@ -43,6 +43,10 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
             else { float2 t = *reinterpret_cast<const float2 *>(src); s[r][0] = t.x; s[r][1] = t.y; }
         }
 
+    // the state was written at least two kernels ago; everything below reads the in-projection
+    pdl_wait();
+    pdl_trigger();
+
     // ---- causal conv + SiLU for the channels this block needs: its x strip, all of B and C
     const int nch = SSM_PR + 2 * N;
     const bool owner = (blockIdx.x == 0 && blockIdx.y == 0);   // writes the shared B|C channels' history
@@ -51,10 +55,10 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
         const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
         const float bias = a.conv_b[gc];
         const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
-        float w0 = win[0], w1 = win[a.convd], w2 = win[2 * a.convd];
+        float w0 = __ldcg(win), w1 = __ldcg(win + a.convd), w2 = __ldcg(win + 2 * a.convd);
         const bool wr = c < SSM_PR || owner;
         for (int i = 0; i < T; ++i) {
-            const float raw = a.zx[(size_t)(rowbase + i) * a.in_ld + a.di + gc];
+            const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc);
             const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
             w0 = w1; w1 = w2; w2 = raw;
             if (c < SSM_PR) xs[i][c] = act;
@@ -68,7 +72,7 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
         }
     }
     if (threadIdx.x < T) {
-        const float dt = softplus_f(a.zx[(size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h] + a.dt_bias[h]);
+        const float dt = softplus_f(__ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) + a.dt_bias[h]);
         dt_s[threadIdx.x] = dt;
         a_s[threadIdx.x] = expf(-dt * expf(a.A_log[h]));
     }
@@ -103,7 +107,7 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
         constexpr int LPV = 32 / RPW;
         if ((lane & (LPV - 1)) == 0) {
             const int r = lane / LPV, col = h * a.P + p0 + warp * RPW + r;
-            const float z = a.zx[(size_t)(rowbase + i) * a.in_ld + col];
+            const float z = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + col);
             a.g[(size_t)(rowbase + i) * a.di + col] = (y + Dh * xs[i][warp * RPW + r]) * silu_f(z);
         }
         // state after position i (verify: snapshot i; draft: the scratch state)
@@ -131,7 +135,7 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
     const int nk = a.gh * DK, nv = a.gh * dv;
 
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
-                        (a.in_slot_stride ? (size_t)a.slot[b] * a.in_slot_stride : 0) + (size_t)h * dv * DK;
+                        (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) + (size_t)h * dv * DK;
     float s[RPW][2];
     const bool rows_ok = warp * RPW < dv;
 #pragma unroll
@@ -139,15 +143,17 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
         float2 t = rows_ok ? *reinterpret_cast<const float2 *>(sin_ + (warp * RPW + r) * DK + 2 * lane) : make_float2(0.f, 0.f);
         s[r][0] = t.x; s[r][1] = t.y;
     }
+    pdl_wait();
+    pdl_trigger();
     // conv + SiLU on this head's q, k, v channels
     for (int c = threadIdx.x; c < 2 * DK + dv; c += GDN_THREADS) {
         const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
         const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
         const float bias = a.conv_b[gc];
         const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
-        float w0 = win[0], w1 = win[a.convd], w2 = win[2 * a.convd];
+        float w0 = __ldcg(win), w1 = __ldcg(win + a.convd), w2 = __ldcg(win + 2 * a.convd);
         for (int i = 0; i < T; ++i) {
-            const float raw = a.zx[(size_t)(rowbase + i) * a.in_ld + gc];
+            const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + gc);
             const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
             w0 = w1; w1 = w2; w2 = raw;
             if (c < DK) qs[i][c] = act; else if (c < 2 * DK) ks[i][c - DK] = act; else vs[i][c - 2 * DK] = act;
@@ -160,8 +166,8 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
     }
     if (threadIdx.x < T) {
         const float *row = a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld;
-        al[threadIdx.x] = sigmoid_f(row[2 * nk + 2 * nv + h]);
-        be[threadIdx.x] = sigmoid_f(row[2 * nk + 2 * nv + a.gh + h]);
+        al[threadIdx.x] = sigmoid_f(__ldcg(row + 2 * nk + 2 * nv + h));
+        be[threadIdx.x] = sigmoid_f(__ldcg(row + 2 * nk + 2 * nv + a.gh + h));
     }
     __syncthreads();
     // L2-normalise q and k of every position (one warp per vector)
@@ -209,7 +215,7 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
         const float rstd = rsqrtf(warp_sum(ss) / (float)dv + a.eps);
         const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
         for (int j = lane; j < dv; j += 32) {
-            const float z = row[2 * nk + nv + h * dv + j];
+            const float z = __ldcg(row + 2 * nk + nv + h * dv + j);
             a.g[(size_t)(rowbase + i) * nv + h * dv + j] = os[i][j] * rstd * a.onorm[j] * silu_f(z);
         }
     }
@@ -219,15 +225,13 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
 
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
     dim3 grid(a.P / SSM_PR, a.H, a.nb);
-    if (a.N == 64) ssm_kernel<2><<<grid, SSM_THREADS, 0, s>>>(a);
-    else if (a.N == 128) ssm_kernel<4><<<grid, SSM_THREADS, 0, s>>>(a);
-    else if (a.N == 256) ssm_kernel<8><<<grid, SSM_THREADS, 0, s>>>(a);
-    else return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    if (a.N == 64) return launch_pdl(ssm_kernel<2>, grid, dim3(SSM_THREADS), 0, s, a);
+    if (a.N == 128) return launch_pdl(ssm_kernel<4>, grid, dim3(SSM_THREADS), 0, s, a);
+    if (a.N == 256) return launch_pdl(ssm_kernel<8>, grid, dim3(SSM_THREADS), 0, s, a);
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s) {
     if (a.dk != 64 || a.dv > 64 || (a.dv & 7)) return cudaErrorInvalidValue;
-    gdn_kernel<<<dim3(a.gh, a.nb), GDN_THREADS, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(gdn_kernel, dim3(a.gh, a.nb), dim3(GDN_THREADS), 0, s, a);
 }
