@@ -198,6 +198,11 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->hbuf[cur]; ga.ldx0 = d; ga.xparts = hparts; ga.xpstride = hps;
         ga.norm_w = ly.norm1; ga.eps = c.eps;
         ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
+        // the mixer that follows reads its recurrent state before its own wait: keep it from starting
+        // until this kernel has waited, i.e. until everything older is complete
+        ga.early_trigger = 0;
+        ga.pf_ptr = ly.type == HS_LAYER_ATT ? ly.W_o : ly.W_out;
+        ga.pf_bytes = 2 * (int64_t)d * (ly.type == HS_LAYER_ATT ? c.qh * c.hd : m->gw);
         PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, st_w, s, &m->launches, nullptr), "in_proj");
         // (2) recurrent mixer
         if (ly.type != HS_LAYER_ATT) {
@@ -262,6 +267,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         } else {
             go.W0 = ly.W_o; go.ldw0 = c.qh * c.hd; go.K0 = c.qh * c.hd; go.x0 = m->obuf; go.ldx0 = c.qh * c.hd;
         }
+        go.early_trigger = 1; go.pf_ptr = ly.W_gu; go.pf_bytes = 2 * (int64_t)2 * c.ff * d;
         PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, st_w, s, &m->launches, &hparts), "out_proj");
         cur ^= 1;
         // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
@@ -269,11 +275,19 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         gu.W0 = ly.W_gu; gu.ldw0 = d; gu.K0 = d; gu.x0 = m->hbuf[cur]; gu.ldx0 = d; gu.xparts = hparts; gu.xpstride = hps;
         gu.norm_w = ly.norm2; gu.eps = c.eps;
         gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
+        gu.early_trigger = 1; gu.pf_ptr = ly.W_down; gu.pf_bytes = 2 * (int64_t)d * c.ff;
         PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, st_w, s, &m->launches, nullptr), "gate_up");
         GemvArgs gdn{};
         gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff; gdn.xparts = 1;
         gdn.O = d; gdn.out = m->hbuf[cur ^ 1]; gdn.ldo = d; gdn.opstride = hps; gdn.max_oparts = HS_H_PARTS;
         gdn.resid = m->hbuf[cur]; gdn.rparts = hparts; gdn.rpstride = hps; gdn.nrows = rows; gdn.epi = EPI_RESID;
+        gdn.early_trigger = 1;
+        {   // next projection in the chain: the following layer's in-projection, or the LM head
+            int nl = l + 1;
+            while (nl < c.L && draft && m->layers[nl].type == HS_LAYER_ATT) ++nl;
+            if (nl < c.L) { gdn.pf_ptr = m->layers[nl].W_in; gdn.pf_bytes = 2 * (int64_t)d * (draft ? m->layers[nl].in_rows_draft : m->layers[nl].in_rows_full); }
+            else { gdn.pf_ptr = m->lm_head; gdn.pf_bytes = 2 * (int64_t)c.V * d; }
+        }
         PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, st_w, s, &m->launches, &hparts), "down");
         cur ^= 1;
     }
@@ -282,6 +296,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->hbuf[cur]; lm.ldx0 = d; lm.xparts = hparts; lm.xpstride = hps;
     lm.norm_w = m->final_norm; lm.eps = c.eps;
     lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
+    lm.early_trigger = 1;
     PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
     if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
     else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");

@@ -36,8 +36,8 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(AttnArgs a) {
 
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
     pdl_wait();
-    pdl_trigger();
     const int len = __ldcg(a.kv_len + b);
     const int nch = max(1, (len + a.chunk - 1) / a.chunk);
     if (split >= nch) return;

@@ -38,7 +38,7 @@ struct GemvGeo {
     int kc;              // columns per tile (multiple of 256): a K range is walked in chunks of kc
     int D;               // tiles in flight per warp (depth of each warp's private ring)
     int krmax;           // max(kr0, kr1): row stride of the staged activations
-    int off_x, off_ring; // shared-memory carve-up (bytes)
+    int off_x, off_nw, off_ring; // shared-memory carve-up (bytes)
 };
 
 __device__ __forceinline__ float dot8(const uint4 &w, const float4 &a, const float4 &b, float acc) {
@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     float *rstd_s = reinterpret_cast<float *>(smraw + 256);               // [16]
     float *ss_s = rstd_s + GV_MAXROWS;                                    // [8][16]
     float *x_s = reinterpret_cast<float *>(smraw + g.off_x);              // [nrows][krmax]
+    float *nw_s = reinterpret_cast<float *>(smraw + g.off_nw);            // [krmax] norm weights of this K range
     __nv_bfloat16 *ring = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_ring);   // [8][D][WR][kc]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -122,11 +123,16 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
         for (long long o = lo + (long long)lane * 8192; o < hi; o += 32 * 8192)
             prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
     }
+    // the norm weights are parameters too: fetch them now, they would otherwise miss in L2 after the wait
+    const bool normed = a.norm_w != nullptr && !seg1;
+    if (normed)
+        for (int c = tid * 4; c < kr; c += GV_THREADS * 4)
+            *reinterpret_cast<float4 *>(nw_s + c) = *reinterpret_cast<const float4 *>(a.norm_w + k0 + c);
     pdl_wait();
     if (!a.early_trigger) pdl_trigger();
+    __syncthreads();                       // nw_s complete
 
     // ---- stage the activation rows of this K range (parts summed, norm weight folded in)
-    const bool normed = a.norm_w != nullptr && !seg1;
     const int nrows = a.nrows;
     {
         const float *xsrc = seg1 ? a.x1 : a.x0;
@@ -151,7 +157,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
                 }
                 const bool inside = c >= k0 && c < k0 + kr;
                 float4 nw = make_float4(1.f, 1.f, 1.f, 1.f);
-                if (normed && inside) nw = *reinterpret_cast<const float4 *>(a.norm_w + c);
+                if (normed && inside) nw = *reinterpret_cast<const float4 *>(nw_s + (c - k0));
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if (rbase + j >= nrows) continue;
@@ -321,7 +327,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     const size_t tile = (size_t)WR * g.kc * 2;
     const size_t xs = (size_t)a.nrows * g.krmax * 4;
     g.off_x = 1024;
-    g.off_ring = (int)((g.off_x + xs + 127) / 128 * 128);
+    g.off_nw = (int)((g.off_x + xs + 127) / 128 * 128);
+    g.off_ring = g.off_nw + (a.norm_w ? g.krmax * 4 : 0);
     int D = 1;
     while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= GV_SMEM_PAIR) ++D;
     g.D = D;

@@ -12,8 +12,8 @@ using namespace hsd;
 __global__ void embed_kernel(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
                              int b0, float *h) {
     const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
-    pdl_wait();
     pdl_trigger();
+    pdl_wait();
     const int tok = __ldcg(cand + b * Tm + col0 + i);
     const uint4 *src = reinterpret_cast<const uint4 *>(E + (size_t)tok * d);
     float *dst = h + (size_t)(lb * T + i) * d;
@@ -43,8 +43,8 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V
                                                       int32_t *tok_out, int tok_col0, float *margin_out) {
     const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
     const float *row = logits + (size_t)(lb * T + i) * V;
-    pdl_wait();
     pdl_trigger();
+    pdl_wait();
     Top2 t = {-INFINITY, 0x7fffffff, -INFINITY};
     for (int j = threadIdx.x; j < V; j += blockDim.x) {
         float v = __ldcg(row + j);
@@ -87,8 +87,8 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V
 __global__ void accept_kernel(AcceptArgs a) {
     const int lb = blockIdx.z, b = a.b0 + lb, rl = blockIdx.y;
     const int k = a.k, Tm = a.Tm;
-    pdl_wait();
     pdl_trigger();
+    pdl_wait();
     const int32_t *cand = a.ctrl.cand + b * Tm, *g = a.ctrl.g + b * Tm;
     int n;
     if (a.forced_n) n = min(max(__ldcg(a.forced_n + b), 0), k);

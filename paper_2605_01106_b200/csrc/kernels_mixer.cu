@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
     const int p0 = blockIdx.x * SSM_PR, h = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, T = a.T;
     const int rowbase = lb * T;
+    pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
     // ---- issue the state loads first: they do not depend on anything computed here
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
@@ -43,9 +44,10 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
             else { float2 t = *reinterpret_cast<const float2 *>(src); s[r][0] = t.x; s[r][1] = t.y; }
         }
 
-    // the state was written at least two kernels ago; everything below reads the in-projection
+    // The state was written at least two kernels ago and the in-projection before this kernel only
+    // lets it start after its own wait, so everything older than that projection is complete: the
+    // state loads above are safe.  Everything below reads the in-projection.
     pdl_wait();
-    pdl_trigger();
 
     // ---- causal conv + SiLU for the channels this block needs: its x strip, all of B and C
     const int nch = SSM_PR + 2 * N;
@@ -132,6 +134,7 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
     __shared__ float vs[HS_MAX_T][64], os[HS_MAX_T][64], al[HS_MAX_T], be[HS_MAX_T];
     const int h = blockIdx.x, lb = blockIdx.y, b = a.b0 + lb, T = a.T, dv = a.dv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, rowbase = lb * T;
+    pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
     const int nk = a.gh * DK, nv = a.gh * dv;
 
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
@@ -144,7 +147,6 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
         s[r][0] = t.x; s[r][1] = t.y;
     }
     pdl_wait();
-    pdl_trigger();
     // conv + SiLU on this head's q, k, v channels
     for (int c = threadIdx.x; c < 2 * DK + dv; c += GDN_THREADS) {
         const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
