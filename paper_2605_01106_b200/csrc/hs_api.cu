@@ -109,8 +109,9 @@ Derived derive(const hs_config &c) {
     v.convd = conv_channels(c);
     v.gw = c.arch == HS_ARCH_PARALLEL ? d_inner(c) : c.gh * c.gdv;
     v.state_elems = c.arch == HS_ARCH_PARALLEL ? (int64_t)c.H * c.P * c.N : (int64_t)c.gh * c.gdv * c.gdk;
-    int chunk = 256;
-    while (chunk > 64 && (int64_t)c.max_batch * c.kvh * ((c.kv_capacity + chunk - 1) / chunk) < 296) chunk >>= 1;
+    // keys per attention CTA: the largest of 128 / 64 / 32 that still gives about two CTAs per SM
+    int chunk = 128;
+    while (chunk > 32 && (int64_t)c.max_batch * c.kvh * ((c.kv_capacity + chunk - 1) / chunk) < 296) chunk >>= 1;
     v.att_chunk = chunk;
     v.att_nch = (c.kv_capacity + chunk - 1) / chunk;
     return v;

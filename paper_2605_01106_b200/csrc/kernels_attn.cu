@@ -1,14 +1,20 @@
 // Verify-mode attention: the T = k+1 new positions of a sequence attend over its KV cache plus the
 // new rows themselves (causal among the new ones), grouped-query heads, split over the cache length.
 //
-// grid = (max splits, kv heads, sequences).  A block handles one split of `chunk` cached keys for
-// the G*T query rows that share its KV head (G = q heads per KV head): K/V tiles of 32 keys are
-// staged in shared memory as bf16, scores and the online softmax run in fp32, and the block writes
-// either the final rows (single split) or an un-normalised partial (m, l, acc).  The block that
-// covers the end of the cache also applies RoPE to the new K rows, appends the T new K/V rows
-// (bf16) to the cache and attends to them from shared memory, so nothing written by this launch is
-// read back from global memory by another block.  Partials are merged by whichever block arrives
-// last (ticket counter, no spinning), always in split order, so the result is reproducible.
+// grid = (max splits, kv heads, sequences); one CTA = one chunk of CK cached keys for the G*T query
+// rows that share its KV head (G = q heads per KV head).
+//  * Before the programmatic-dependent-launch wait the CTA reads kv_len (written at least two
+//    kernels earlier), starts two bulk asynchronous copies - its K chunk and its V chunk, each one
+//    contiguous piece of the cache - and fetches the RoPE rows of the new positions.
+//  * After the wait it rotates and scales the queries into shared memory; the CTA of the last chunk
+//    also rotates the T new K rows, rounds K and V to bf16 exactly as they are cached, appends them to
+//    the cache and keeps them in shared memory behind the cached keys, so nothing written by this
+//    launch is read back from global memory by another block.
+//  * Scores: lane = key, each warp takes a subset of the query rows; the dense key rows are read in a
+//    per-lane rotated chunk order so that the 128-bit reads do not collide on a bank.  One softmax per
+//    chunk (the whole chunk is resident), then P V with thread = output dimension.
+//  * Several chunks: every CTA publishes an un-normalised partial (m, l, acc); the CTA that arrives
+//    last (ticket counter, no spinning) merges them in chunk order, so the result is reproducible.
 #include "hs_internal.h"
 #include "hs_device.cuh"
 
@@ -16,202 +22,274 @@ namespace {
 using namespace hsd;
 
 constexpr int AT_THREADS = 128;
-constexpr int KT = 32;                 // keys per tile
+constexpr int AT_WARPS = 4;
 
 template <int HD>
-__global__ void __launch_bounds__(AT_THREADS) attn_kernel(AttnArgs a) {
-    constexpr int KSTR = HD + 8;       // padded bf16 row stride: 16-byte aligned, conflict-free 128-bit reads
-    extern __shared__ __align__(16) unsigned char smraw[];
-    const int G = a.qh / a.kvh, T = a.T, GT = G * T;
-    float *q_s = reinterpret_cast<float *>(smraw);                         // [GT][HD] (RoPE'd, pre-scaled)
-    float *p_s = q_s + HS_MAX_GT * HD;                                     // [GT][KT] scores -> probabilities
-    float *m_s = p_s + HS_MAX_GT * KT;                                     // [GT] running max
-    float *l_s = m_s + HS_MAX_GT;                                          // [GT] running sum
-    float *c_s = l_s + HS_MAX_GT;                                          // [GT] rescale of this tile
-    __nv_bfloat16 *K_s = reinterpret_cast<__nv_bfloat16 *>(c_s + HS_MAX_GT);   // [KT][KSTR]
-    __nv_bfloat16 *V_s = K_s + KT * KSTR;                                  // [KT][KSTR]
-    __nv_bfloat16 *Kn_s = V_s + KT * KSTR;                                 // [HS_MAX_T][KSTR] new rows
-    __nv_bfloat16 *Vn_s = Kn_s + HS_MAX_T * KSTR;
+struct AttnSmem {
+    // offsets in bytes for a chunk capacity of ck cached keys (+ up to 16 new ones)
+    static __host__ __device__ int keys(int ck) { return ck + 16; }
+    static __host__ __device__ size_t k_off() { return 128; }
+    static __host__ __device__ size_t v_off(int ck) { return k_off() + (size_t)keys(ck) * HD * 2; }
+    static __host__ __device__ size_t q_off(int ck) { return v_off(ck) + (size_t)keys(ck) * HD * 2; }
+    static __host__ __device__ size_t p_off(int ck) { return q_off(ck) + (size_t)HS_MAX_GT * HD * 4; }
+    static __host__ __device__ size_t ml_off(int ck) { return p_off(ck) + (size_t)HS_MAX_GT * keys(ck) * 4; }
+    static __host__ __device__ size_t rope_off(int ck) { return ml_off(ck) + (size_t)HS_MAX_GT * 2 * 4; }
+    static __host__ __device__ size_t total(int ck) { return rope_off(ck) + (size_t)HS_MAX_T * (HD / 2) * 8; }
+};
+
+template <int HD, int GTB>      // GTB: compile-time bound of G*T (16, 32 or 48)
+__global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
+    using L = AttnSmem<HD>;
+    constexpr int NC = HD / 8;             // 16-byte chunks per key row
+    extern __shared__ __align__(128) unsigned char smraw[];
+    const int CK = a.chunk;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(smraw);
+    __nv_bfloat16 *K_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L::k_off());      // [CK + 16][HD]
+    __nv_bfloat16 *V_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L::v_off(CK));
+    float *q_s = reinterpret_cast<float *>(smraw + L::q_off(CK));                    // [GT][HD] rotated, pre-scaled
+    float *p_s = reinterpret_cast<float *>(smraw + L::p_off(CK));                    // [GT][CK + 16]
+    float *ml_s = reinterpret_cast<float *>(smraw + L::ml_off(CK));                  // [GT][2]
+    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L::rope_off(CK));            // [T][HD/2]
     __shared__ int ticket_s;
 
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = a.qh / a.kvh, T = a.T, GT = G * T, PST = L::keys(CK);
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
-    pdl_wait();
+
+    // ---- before the wait: kv_len, the cached chunk, the RoPE rows
     const int len = __ldcg(a.kv_len + b);
-    const int nch = max(1, (len + a.chunk - 1) / a.chunk);
-    if (split >= nch) return;
-    if (len + T > a.cap) {             // never write past the cache; the host reports the status word
+    const int nsplit = max(1, (len + CK - 1) / CK);
+    if (split >= nsplit) return;
+    const bool last = split == nsplit - 1;
+    const int c0 = split * CK, ncache = max(0, min(len, c0 + CK) - c0);
+    const bool overflow = len + T > a.cap;       // never write past the cache; the host reports the status word
+    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    if (tid == 0) { mbar_init(bar, 1); mbar_fence_init(); }
+    __syncthreads();
+    if (tid == 0 && ncache > 0 && !overflow) {
+        const uint32_t bytes = (uint32_t)ncache * HD * 2;
+        mbar_expect_tx(bar, 2 * bytes);
+        bulk_g2s(K_s, Kb + (size_t)c0 * HD, bytes, bar);
+        bulk_g2s(V_s, Vb + (size_t)c0 * HD, bytes, bar);
+    }
+    if (!overflow)
+        for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
+            const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+            rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
+        }
+    pdl_wait();
+    if (overflow) {
         if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
         return;
     }
-    const bool last = (split == nch - 1);
-    const int rowbase = lb * T;
-    const float scale = rsqrtf((float)HD);
+    __syncthreads();                        // rope_s complete
 
     // ---- queries: RoPE at position len + i, pre-multiplied by 1/sqrt(hd)
+    const int rowbase = lb * T;
+    const float scale = rsqrtf((float)HD);
     for (int idx = tid; idx < GT * (HD / 2); idx += AT_THREADS) {
         const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
         const int gq = qi / T, i = qi - gq * T;
         const float *src = a.zx + (size_t)(rowbase + i) * a.in_ld + a.q_off + (kh * G + gq) * HD;
-        const float2 cs = a.rope[(size_t)(len + i) * (HD / 2) + e];
+        const float2 cs = rope_s[i * (HD / 2) + e];
         const float x0 = __ldcg(src + e), x1 = __ldcg(src + e + HD / 2);
         q_s[qi * HD + e] = (x0 * cs.x - x1 * cs.y) * scale;
         q_s[qi * HD + e + HD / 2] = (x1 * cs.x + x0 * cs.y) * scale;
     }
-    if (tid < GT) { m_s[tid] = -INFINITY; l_s[tid] = 0.f; }
-    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    int nkeys = ncache;
     if (last) {
-        // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached
+        // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached, behind the cached keys
         for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
             const int i = idx / (HD / 2), e = idx - i * (HD / 2);
             const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
-            const float2 cs = a.rope[(size_t)(len + i) * (HD / 2) + e];
+            const float2 cs = rope_s[idx];
             const float x0 = __ldcg(row + a.k_off + kh * HD + e), x1 = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
             const __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * cs.x - x1 * cs.y);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
             const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
             const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
-            Kn_s[i * KSTR + e] = k0; Kn_s[i * KSTR + e + HD / 2] = k1;
-            Vn_s[i * KSTR + e] = v0; Vn_s[i * KSTR + e + HD / 2] = v1;
+            const int j = ncache + i;
+            K_s[j * HD + e] = k0; K_s[j * HD + e + HD / 2] = k1;
+            V_s[j * HD + e] = v0; V_s[j * HD + e + HD / 2] = v1;
             Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
             Vb[(size_t)(len + i) * HD + e] = v0; Vb[(size_t)(len + i) * HD + e + HD / 2] = v1;
         }
+        nkeys += T;
     }
-    float acc[HS_MAX_GT];              // thread tid < HD owns output dim tid of every query row
+    bool landed = true;
+    if (ncache > 0) landed = mbar_wait(bar, 0);
+    if (!__syncthreads_and(landed)) {
+        if (tid == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
+        return;
+    }
+
+    // ---- scores: lane = key (tiles of 32), warp w takes query rows w, w + 4, ...
+    for (int j0 = 0; j0 < nkeys; j0 += 32) {
+        const int j = j0 + lane;
+        const bool kvalid = j < nkeys;
+        const uint4 *krow = reinterpret_cast<const uint4 *>(K_s + (size_t)min(j, nkeys - 1) * HD);
+        for (int qb = warp; qb < GT; qb += AT_WARPS * 4) {
+            // up to four query rows per pass: qb, qb + 4, qb + 8, qb + 12
+            float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+            for (int c = 0; c < NC; ++c) {
+                const int cc = (c + lane) & (NC - 1);          // rotated chunk order: conflict-free key reads
+                const uint4 w = krow[cc];
+                const float k0 = bf_lo(w.x), k1 = bf_hi(w.x), k2 = bf_lo(w.y), k3 = bf_hi(w.y);
+                const float k4 = bf_lo(w.z), k5 = bf_hi(w.z), k6 = bf_lo(w.w), k7 = bf_hi(w.w);
 #pragma unroll
-    for (int qi = 0; qi < HS_MAX_GT; ++qi) acc[qi] = 0.f;
+                for (int u = 0; u < 4; ++u) {
+                    const int qi = qb + u * AT_WARPS;
+                    if (qi < GT) {
+                        const float4 qa = *reinterpret_cast<const float4 *>(q_s + qi * HD + cc * 8);
+                        const float4 qc = *reinterpret_cast<const float4 *>(q_s + qi * HD + cc * 8 + 4);
+                        d[u] = fmaf(k0, qa.x, fmaf(k1, qa.y, fmaf(k2, qa.z, fmaf(k3, qa.w, d[u]))));
+                        d[u] = fmaf(k4, qc.x, fmaf(k5, qc.y, fmaf(k6, qc.z, fmaf(k7, qc.w, d[u]))));
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int qi = qb + u * AT_WARPS;
+                if (qi < GT && kvalid) {
+                    const int i = qi % T;
+                    const bool masked = last && j >= ncache && (j - ncache) > i;     // causal among the new rows
+                    p_s[qi * PST + j] = masked ? -INFINITY : d[u];
+                }
+            }
+        }
+    }
     __syncthreads();
-
-    const int c0 = split * a.chunk, c1 = min(len, c0 + a.chunk);
-    const int ncache = max(0, c1 - c0);
-    const int ntile_cache = (ncache + KT - 1) / KT;
-    const int ntile = ntile_cache + (last ? 1 : 0);
-    for (int t = 0; t < ntile; ++t) {
-        const bool fresh = (t == ntile_cache);             // the tile of new rows (only when last)
-        const int k0 = fresh ? len : c0 + t * KT;          // absolute index of the tile's first key
-        const int nkeys = fresh ? T : min(KT, c1 - k0);
-        // ---- stage the tile
-        if (!fresh) {
-            for (int idx = tid; idx < KT * (HD / 8); idx += AT_THREADS) {
-                const int j = idx / (HD / 8), c = idx - j * (HD / 8);
-                uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-                if (j < nkeys) {
-                    kv = ldg_stream(Kb + (size_t)(k0 + j) * HD + 8 * c);
-                    vv = ldg_stream(Vb + (size_t)(k0 + j) * HD + 8 * c);
-                }
-                *reinterpret_cast<uint4 *>(K_s + j * KSTR + 8 * c) = kv;
-                *reinterpret_cast<uint4 *>(V_s + j * KSTR + 8 * c) = vv;
-            }
-            __syncthreads();
+    // ---- softmax statistics of the chunk: one warp per query row
+    for (int qi = warp; qi < GT; qi += AT_WARPS) {
+        float mx = -INFINITY;
+        for (int j = lane; j < nkeys; j += 32) mx = fmaxf(mx, p_s[qi * PST + j]);
+        mx = warp_max(mx);
+        float sum = 0.f;
+        for (int j = lane; j < nkeys; j += 32) {
+            const float p = expf(p_s[qi * PST + j] - mx);        // expf(-inf) = 0 for masked keys
+            p_s[qi * PST + j] = p;
+            sum += p;
         }
-        const __nv_bfloat16 *Kt_ = fresh ? Kn_s : K_s, *Vt_ = fresh ? Vn_s : V_s;
-        // ---- scores: lane = key, warp w takes query rows w, w+4, ...
-        for (int qi = warp; qi < GT; qi += AT_THREADS / 32) {
-            float sc = -INFINITY;
-            const int i = qi % T;
-            if (lane < nkeys && (!fresh || lane <= i)) {     // causal among the new rows
-                const uint4 *kr = reinterpret_cast<const uint4 *>(Kt_ + lane * KSTR);
-                const float4 *qr = reinterpret_cast<const float4 *>(q_s + qi * HD);
-                float d = 0.f;
-#pragma unroll
-                for (int c = 0; c < HD / 8; ++c) {
-                    const uint4 w = kr[c];
-                    const float4 qa = qr[2 * c], qb = qr[2 * c + 1];
-                    d = fmaf(bf_lo(w.x), qa.x, d); d = fmaf(bf_hi(w.x), qa.y, d);
-                    d = fmaf(bf_lo(w.y), qa.z, d); d = fmaf(bf_hi(w.y), qa.w, d);
-                    d = fmaf(bf_lo(w.z), qb.x, d); d = fmaf(bf_hi(w.z), qb.y, d);
-                    d = fmaf(bf_lo(w.w), qb.z, d); d = fmaf(bf_hi(w.w), qb.w, d);
-                }
-                sc = d;
-            }
-            const float m_old = m_s[qi];
-            const float m_new = fmaxf(m_old, warp_max(sc));
-            const float p = (sc == -INFINITY) ? 0.f : expf(sc - m_new);
-            const float psum = warp_sum(p);
-            p_s[qi * KT + lane] = p;
-            if (lane == 0) {
-                const float corr = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
-                c_s[qi] = corr; m_s[qi] = m_new; l_s[qi] = l_s[qi] * corr + psum;
-            }
-        }
-        __syncthreads();
-        // ---- acc <- acc * corr + P V : thread = output dim
-        if (tid < HD) {
-#pragma unroll
-            for (int qi = 0; qi < HS_MAX_GT; ++qi) if (qi < GT) acc[qi] *= c_s[qi];
-            for (int j = 0; j < nkeys; ++j) {
-                const float v = __bfloat162float(Vt_[j * KSTR + tid]);
-#pragma unroll
-                for (int qi = 0; qi < HS_MAX_GT; ++qi) if (qi < GT) acc[qi] = fmaf(p_s[qi * KT + j], v, acc[qi]);
-            }
-        }
-        __syncthreads();
+        sum = warp_sum(sum);
+        if (lane == 0) { ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = sum; }
     }
-
+    __syncthreads();
+    // ---- acc = P V : thread = output dimension
+    float acc[GTB];
+#pragma unroll
+    for (int qi = 0; qi < GTB; ++qi) acc[qi] = 0.f;
+    if (tid < HD) {
+        for (int j = 0; j < nkeys; ++j) {
+            const float v = __bfloat162float(V_s[(size_t)j * HD + tid]);
+#pragma unroll
+            for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc[qi] = fmaf(p_s[qi * PST + j], v, acc[qi]);
+        }
+    }
     float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
-    if (nch == 1) {
+    if (nsplit == 1) {
         if (tid < HD) {
 #pragma unroll
-            for (int qi = 0; qi < HS_MAX_GT; ++qi)
+            for (int qi = 0; qi < GTB; ++qi)
                 if (qi < GT) {
                     const int gq = qi / T, i = qi - gq * T;
-                    o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + tid] = acc[qi] / l_s[qi];
+                    o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + tid] = acc[qi] / ml_s[2 * qi + 1];
                 }
         }
         return;
     }
-    // ---- several splits: publish the partial, the last block to arrive merges in split order
+    // ---- several chunks: publish the partial, the last block to arrive merges in chunk order
     const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
     float *pa = a.part_acc + (pbase + split) * HS_MAX_GT * HD;
     float *pm = a.part_ml + (pbase + split) * HS_MAX_GT * 2;
     if (tid < HD) {
 #pragma unroll
-        for (int qi = 0; qi < HS_MAX_GT; ++qi) if (qi < GT) pa[qi * HD + tid] = acc[qi];
+        for (int qi = 0; qi < GTB; ++qi) if (qi < GT) pa[qi * HD + tid] = acc[qi];
     }
-    if (tid < GT) { pm[2 * tid] = m_s[tid]; pm[2 * tid + 1] = l_s[tid]; }
+    if (tid < 2 * GT) pm[tid] = ml_s[tid];
     __threadfence();
     __syncthreads();
     if (tid == 0) ticket_s = atomicAdd(a.counters + b * a.kvh + kh, 1);
     __syncthreads();
-    if (ticket_s != nch - 1) return;
+    if (ticket_s != nsplit - 1) return;
     __threadfence();
     if (tid == 0) a.counters[b * a.kvh + kh] = 0;          // ready for the next launch
     const float *pa0 = a.part_acc + pbase * HS_MAX_GT * HD;
     const float *pm0 = a.part_ml + pbase * HS_MAX_GT * 2;
-    if (tid < HD)
-        for (int qi = 0; qi < GT; ++qi) {
-            float M = -INFINITY;
-            for (int c = 0; c < nch; ++c) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
-            float num = 0.f, den = 0.f;
-            for (int c = 0; c < nch; ++c) {
-                const float w = expf(__ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2) - M);
-                den = fmaf(w, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2 + 1), den);
-                num = fmaf(w, __ldcg(pa0 + ((size_t)c * HS_MAX_GT + qi) * HD + tid), num);
-            }
-            const int gq = qi / T, i = qi - gq * T;
-            o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + tid] = num / den;
+    float *w_s = p_s;                                        // [GT][PST]: merge weights of PST chunks per pass
+    for (int qi = warp; qi < GT; qi += AT_WARPS) {
+        float M = -INFINITY;
+        for (int c = lane; c < nsplit; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+        M = warp_max(M);
+        float den = 0.f;
+        for (int c = lane; c < nsplit; c += 32) {
+            const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+            den = fmaf(expf(mlv.x - M), mlv.y, den);
         }
+        den = warp_sum(den);
+        if (lane == 0) { ml_s[2 * qi] = M; ml_s[2 * qi + 1] = den; }
+    }
+#pragma unroll
+    for (int qi = 0; qi < GTB; ++qi) acc[qi] = 0.f;
+    for (int cb = 0; cb < nsplit; cb += PST) {               // chunks in passes of PST
+        const int nc = min(PST, nsplit - cb);
+        __syncthreads();                                     // ml_s ready / previous pass done with w_s
+        for (int idx = tid; idx < GT * nc; idx += AT_THREADS) {
+            const int qi = idx / nc, c = idx - qi * nc;
+            w_s[qi * PST + c] = expf(__ldcg(pm0 + ((size_t)(cb + c) * HS_MAX_GT + qi) * 2) - ml_s[2 * qi]);
+        }
+        __syncthreads();
+        if (tid < HD) {
+            for (int c = 0; c < nc; ++c) {
+                const float *src = pa0 + (size_t)(cb + c) * HS_MAX_GT * HD + tid;
+#pragma unroll
+                for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc[qi] = fmaf(w_s[qi * PST + c], __ldcg(src + qi * HD), acc[qi]);
+            }
+        }
+    }
+    if (tid < HD) {
+#pragma unroll
+        for (int qi = 0; qi < GTB; ++qi)
+            if (qi < GT) {
+                const int gq = qi / T, i = qi - gq * T;
+                o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + tid] = acc[qi] / ml_s[2 * qi + 1];
+            }
+    }
 }
 
-template <int HD>
-size_t attn_smem() {
-    return (size_t)(HS_MAX_GT * HD + HS_MAX_GT * KT + 3 * HS_MAX_GT) * 4 +
-           (size_t)(2 * KT + 2 * HS_MAX_T) * (HD + 8) * 2;
+template <int HD, int GTB>
+cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
+    dim3 grid(a.nch, a.kvh, a.nb);
+    return launch_pdl(attn_kernel<HD, GTB>, grid, dim3(AT_THREADS), AttnSmem<HD>::total(a.chunk), s, a);
+}
+
+template <int HD, int GTB>
+cudaError_t configure_t() {
+    cudaError_t e = cudaFuncSetAttribute(attn_kernel<HD, GTB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnSmem<HD>::total(128));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<HD, GTB>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+    return e;
 }
 
 }  // namespace
 
 cudaError_t configure_attn() {
-    cudaError_t e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<128>());
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<64>());
+    cudaError_t e = configure_t<128, 16>();
+    if (e == cudaSuccess) e = configure_t<128, 32>();
+    if (e == cudaSuccess) e = configure_t<128, 48>();
+    if (e == cudaSuccess) e = configure_t<64, 16>();
+    if (e == cudaSuccess) e = configure_t<64, 32>();
+    if (e == cudaSuccess) e = configure_t<64, 48>();
     return e;
 }
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
-    dim3 grid(a.nch, a.kvh, a.nb);
-    if (a.hd == 128) return launch_pdl(attn_kernel<128>, grid, dim3(AT_THREADS), attn_smem<128>(), s, a);
-    if (a.hd == 64) return launch_pdl(attn_kernel<64>, grid, dim3(AT_THREADS), attn_smem<64>(), s, a);
+    const int GT = (a.qh / a.kvh) * a.T;
+    if (GT > HS_MAX_GT || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128)) return cudaErrorInvalidValue;
+    const int gtb = GT <= 16 ? 16 : GT <= 32 ? 32 : 48;
+#define CASE(hd_, g_) if (a.hd == hd_ && gtb == g_) return launch_t<hd_, g_>(a, s)
+    CASE(128, 16); CASE(128, 32); CASE(128, 48); CASE(64, 16); CASE(64, 32); CASE(64, 48);
+#undef CASE
     return cudaErrorInvalidValue;
 }
