@@ -119,8 +119,8 @@ Derived derive(const hs_config &c) {
 
 // layout of the work buffer; base may be null to only measure
 struct WorkLayout {
-    int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters;
-    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, total;
+    int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters;
+    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, am_part, total;
 };
 
 WorkLayout work_layout(const hs_config &c, const Derived &v) {
@@ -130,7 +130,7 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.cand = take(4 * v.R); w.g = take(4 * v.R); w.margin = take(4 * v.R);
     w.n_acc = take(4 * v.B); w.emitted = take(4 * v.R);
     w.stage_n = take(4 * v.B); w.stage_next = take(4 * v.B);
-    w.status = take(4); w.counters = take((int64_t)4 * v.B * c.kvh);
+    w.status = take(4); w.counters = take((int64_t)4 * v.B * c.kvh); w.am_counters = take((int64_t)4 * v.R);
     w.rope = take((int64_t)c.kv_capacity * (c.hd / 2) * 8);
     w.h = take((int64_t)4 * 2 * HS_H_PARTS * v.R * c.d);
     w.zx = take((int64_t)4 * v.R * v.in_rows_max);
@@ -140,6 +140,7 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.logits = take((int64_t)4 * v.R * c.V);
     w.att_acc = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * c.hd);
     w.att_ml = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * 2);
+    w.am_part = take((int64_t)16 * v.R * HS_ARGMAX_CHUNKS);
     w.total = off;
     return w;
 }
@@ -299,8 +300,8 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
     lm.early_trigger = 1;
     PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
-    if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, s), "argmax");
-    else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, s), "argmax");
+    if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, m->am_part, m->ctrl.am_counters, s), "argmax");
+    else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, m->am_part, m->ctrl.am_counters, s), "argmax");
     ++m->launches;
     m->last_rows = rows;
     return HS_OK;
@@ -414,11 +415,11 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     m->ctrl.cand = (int32_t *)(w + wl.cand); m->ctrl.g = (int32_t *)(w + wl.g); m->ctrl.margin = (float *)(w + wl.margin);
     m->ctrl.n_acc = (int32_t *)(w + wl.n_acc); m->ctrl.emitted = (int32_t *)(w + wl.emitted);
     m->ctrl.stage_n = (int32_t *)(w + wl.stage_n); m->ctrl.stage_next = (int32_t *)(w + wl.stage_next);
-    m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters);
+    m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters); m->ctrl.am_counters = (int32_t *)(w + wl.am_counters);
     m->rope = (float2 *)(w + wl.rope);
     m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
     m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits);
-    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml);
+    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part;
     // conv buffer: committed windows | verify history | draft ping-pong
     float *cv = (float *)bufs->conv;
     const size_t win = (size_t)v.n_rl * v.B * 3 * v.convd;

@@ -11,6 +11,7 @@
 #define HS_MAX_K 8
 #define HS_MAX_T (HS_MAX_K + 1)
 #define HS_H_PARTS 4          // a projection may leave the residual stream as up to 4 partial sums
+#define HS_ARGMAX_CHUNKS 32    // CTAs that share one logits row in the argmax
 #define HS_MAX_GT 48          // (q heads per kv head) * (k+1) upper bound of the attention kernel
 
 // ---------------------------------------------------------------------------------------------
@@ -29,6 +30,7 @@ struct HsCtrl {
     int32_t *stage_next;  // [B]
     int32_t *status;      // [1]   first error a kernel recorded
     int32_t *counters;    // [B][kvh] split-KV arrival tickets (zero between launches)
+    int32_t *am_counters; // [B][Tm] argmax arrival tickets (zero between launches)
 };
 
 struct HsLayer {
@@ -61,6 +63,7 @@ struct hs_model {
     float *hbuf[2];            // residual stream, ping-pong; each [HS_H_PARTS][B*Tm][d] partial sums
     float *zx, *gbuf, *obuf, *abuf, *logits;
     float *att_acc, *att_ml;
+    void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
     // conv buffers
     float *cw, *hist, *dcw;
     __nv_bfloat16 *Kc, *Vc;
@@ -165,8 +168,10 @@ struct AttnArgs {
 };
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);
 
+// part: scratch of HS_ARGMAX_CHUNKS * 16 bytes per logits row (row slot b * Tm + i); counters: one int32 per
+// row slot, zero between launches
 cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
-                          int32_t *tok_out, int tok_col0, float *margin_out, cudaStream_t s);
+                          int32_t *tok_out, int tok_col0, float *margin_out, void *part, int32_t *counters, cudaStream_t s);
 
 struct AcceptArgs {
     int k, Tm, b0, nb, n_rl, B, convd;

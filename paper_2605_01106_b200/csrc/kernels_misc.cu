@@ -38,19 +38,19 @@ __device__ __forceinline__ Top2 top2_merge(const Top2 &a, const Top2 &b) {
     return r;
 }
 
-// one block per logits row: token = argmax (lowest id on ties), margin = top1 - top2
-__global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V, int T, int b0, int Tm,
-                                                      int32_t *tok_out, int tok_col0, float *margin_out) {
-    const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
-    const float *row = logits + (size_t)(lb * T + i) * V;
-    pdl_trigger();
-    pdl_wait();
-    Top2 t = {-INFINITY, 0x7fffffff, -INFINITY};
-    for (int j = threadIdx.x; j < V; j += blockDim.x) {
-        float v = __ldcg(row + j);
-        if (v > t.v1) { t.v2 = t.v1; t.v1 = v; t.i1 = j; }
-        else if (v > t.v2) t.v2 = v;
-    }
+// Greedy argmax with top-2 margin over V logits per row, split over HS_ARGMAX_CHUNKS CTAs per row.
+// grid = (chunks, T, nb).  A CTA scans its slice (lowest id wins a tie), writes a partial
+// (top value, its id, runner-up) to scratch and takes a ticket; the CTA that arrives last merges the
+// row's partials - the merge is order-independent, so the result is reproducible - writes the token
+// and the margin and puts the ticket counter back to zero for the next launch.
+struct ArgmaxArgs {
+    const float *logits; int V, T, b0, Tm;
+    int32_t *tok_out; int tok_col0; float *margin_out;
+    float4 *part;            // scratch [rows][HS_ARGMAX_CHUNKS]
+    int32_t *counters;       // scratch [rows], zero between launches
+};
+
+__device__ __forceinline__ Top2 top2_warp(Top2 t) {
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) {
         Top2 u;
@@ -59,24 +59,58 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *logits, int V
         u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
         t = top2_merge(t, u);
     }
-    __shared__ Top2 s[32];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    return t;
+}
+
+__global__ void __launch_bounds__(256) argmax_kernel(const ArgmaxArgs a) {
+    const int chunk = blockIdx.x, i = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
+    const int nchunk = gridDim.x;
+    const float *row = a.logits + (size_t)(lb * a.T + i) * a.V;
+    const int srow = b * a.Tm + i;                                // scratch slot of this logits row
+    const int per = ((a.V + nchunk - 1) / nchunk + 3) & ~3;
+    const int lo = chunk * per, hi = min(a.V, lo + per);
+    pdl_trigger();
+    pdl_wait();
+    Top2 t = {-INFINITY, 0x7fffffff, -INFINITY};
+    auto feed = [&](float v, int j) {
+        if (v > t.v1) { t.v2 = t.v1; t.v1 = v; t.i1 = j; }
+        else if (v > t.v2) t.v2 = v;
+    };
+    if ((a.V & 3) == 0) {
+        for (int j = lo + threadIdx.x * 4; j < hi; j += blockDim.x * 4) {
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(row + j));
+            feed(v.x, j); feed(v.y, j + 1); feed(v.z, j + 2); feed(v.w, j + 3);
+        }
+    } else {
+        for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) feed(__ldcg(row + j), j);
+    }
+    t = top2_warp(t);
+    __shared__ Top2 s[8];
+    __shared__ int ticket_s;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (lane == 0) s[warp] = t;
     __syncthreads();
-    if (warp == 0) {
-        t = lane < nw ? s[lane] : Top2{-INFINITY, 0x7fffffff, -INFINITY};
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            Top2 u;
-            u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
-            u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
-            u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
-            t = top2_merge(t, u);
-        }
-        if (lane == 0) {
-            tok_out[b * Tm + tok_col0 + i] = t.i1;
-            if (margin_out) margin_out[b * Tm + i] = t.v1 - t.v2;
-        }
+    if (warp != 0) return;
+    t = lane < (int)(blockDim.x >> 5) ? s[lane] : Top2{-INFINITY, 0x7fffffff, -INFINITY};
+    t = top2_warp(t);
+    if (lane == 0) {
+        a.part[(size_t)srow * nchunk + chunk] = make_float4(t.v1, __int_as_float(t.i1), t.v2, 0.f);
+        __threadfence();
+        ticket_s = atomicAdd(a.counters + srow, 1);
+    }
+    __syncwarp();
+    if (ticket_s != nchunk - 1) return;
+    __threadfence();
+    t = Top2{-INFINITY, 0x7fffffff, -INFINITY};
+    for (int c = lane; c < nchunk; c += 32) {
+        const float4 p = __ldcg(a.part + (size_t)srow * nchunk + c);
+        t = top2_merge(t, Top2{p.x, __float_as_int(p.y), p.z});
+    }
+    t = top2_warp(t);
+    if (lane == 0) {
+        a.counters[srow] = 0;
+        a.tok_out[b * a.Tm + a.tok_col0 + i] = t.i1;
+        if (a.margin_out) a.margin_out[b * a.Tm + i] = t.v1 - t.v2;
     }
 }
 
@@ -130,8 +164,9 @@ cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int
 }
 
 cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
-                          int32_t *tok_out, int tok_col0, float *margin_out, cudaStream_t s) {
-    return launch_pdl(argmax_kernel, dim3(T, nb), dim3(1024), 0, s, logits, V, T, b0, Tm, tok_out, tok_col0, margin_out);
+                          int32_t *tok_out, int tok_col0, float *margin_out, void *part, int32_t *counters, cudaStream_t s) {
+    ArgmaxArgs a{logits, V, T, b0, Tm, tok_out, tok_col0, margin_out, reinterpret_cast<float4 *>(part), counters};
+    return launch_pdl(argmax_kernel, dim3(HS_ARGMAX_CHUNKS, T, nb), dim3(256), 0, s, a);
 }
 
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s) {
