@@ -188,6 +188,26 @@ int hs_profile_read(hs_model *m, double *ms, int64_t *launches, double *bytes);
 /* Device status word: 0, or the first hs_status a kernel recorded.  Synchronises. */
 int hs_device_status(hs_model *m);
 const char *hs_last_error(const hs_model *m);
+
+/* Greedy argmax for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a convenience of the library.)  Computes, for each of `rows` logits rows of V floats (DEVICE,
+ * row-major, contiguous), the id of the largest logit - the lowest id on a tie - into token_dev[row]
+ * (DEVICE int32) and, if margin_dev is not NULL, top1 - top2 into margin_dev[row] (DEVICE float): the
+ * same kernel and the same decisions as inside hs_draft / hs_verify.
+ * Who needs it: code that may not call cudaMalloc where it runs - an engine that has already reserved
+ * the whole GPU for its own pool, a component that is handed pointers and nothing else, a loop that
+ * cannot afford the device-wide synchronisation an allocation can cause.  The kernel's scratch
+ * (per-block partial results and arrival counters, 33 KB) therefore lives in a fixed __device__ array
+ * inside the library; every GPU that loads libhs.so holds those 33 KB until the process ends.
+ * Limits and rules:
+ *  - rows <= 64, otherwise HS_ERR_SIZE and nothing is launched; V >= 1.  Bad pointers/sizes:
+ *    HS_ERR_INVALID_ARG.  A failing CUDA call: HS_ERR_CUDA.
+ *  - The call allocates and frees nothing.  It is asynchronous on `stream` (a cudaStream_t).
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
+ *    that device current; make that first call outside any stream capture.
+ *  - All calls share the one array: the counters are cleared at the start of every call, and two calls
+ *    that may overlap on the GPU (different streams, no ordering between them) race on it - order them. */
+int hs_argmax_static(const float *logits_dev, int V, int rows, int32_t *token_dev, float *margin_dev, void *stream);
 int hs_destroy(hs_model *m);
 
 #ifdef __cplusplus

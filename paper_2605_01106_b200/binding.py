@@ -19,7 +19,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy"]
+           "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
 class HsError(RuntimeError):
@@ -77,12 +77,26 @@ def load_library(path: str | None = None):
     L.hs_last_error.restype = ctypes.c_char_p
     L.hs_last_error.argtypes = [vp]
     L.hs_destroy.argtypes = [vp]
+    L.hs_argmax_static.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp, vp]
     _LIB = L
     return L
 
 
 def lib():
     return load_library()
+
+
+def argmax_static(logits_dev, tokens_dev, margins_dev=None, stream=None):
+    """hs_argmax_static on torch CUDA tensors: logits [rows, V] float32 (contiguous), tokens [rows] int32,
+    margins [rows] float32 or None.  Uses the library's built-in scratch: nothing is allocated.
+    Runs on `stream` (torch stream) or torch's current stream; raises HsError on a non-zero status."""
+    import torch
+    rows, V = logits_dev.shape
+    st = stream or torch.cuda.current_stream(logits_dev.device)
+    rc = lib().hs_argmax_static(logits_dev.data_ptr(), int(V), int(rows), tokens_dev.data_ptr(),
+                                margins_dev.data_ptr() if margins_dev is not None else None, vp(st.cuda_stream))
+    if rc != 0:
+        raise HsError(rc, "hs_argmax_static: %s" % {-1: "invalid argument", -2: "more than 64 rows", -5: "CUDA error"}.get(rc, "error"))
 
 
 def make_config(shape, max_batch=1, max_k=8, kv_capacity=1024, flags=0) -> HsConfig:

@@ -174,3 +174,46 @@ cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s) {
     if (chunks < 1) chunks = 1;
     return launch_pdl(accept_kernel, dim3(chunks, a.n_rl > 0 ? a.n_rl : 1, a.nb), dim3(256), 0, s, a);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Argmax without any caller- or library-allocated scratch.
+//
+// The split argmax above needs a few kilobytes of scratch (per-CTA partial results and a ticket
+// counter per row).  Inside the model that scratch is carved out of the caller's work buffer.  This
+// stand-alone variant keeps it in a fixed array that is part of the library image instead, so that
+// code which is not in a position to allocate device memory can still run the kernel: a host loop
+// that already handed every free byte of the GPU to its own arena, a plug-in that is only given
+// pointers, or a latency-critical section where an allocation (which may synchronise the device)
+// is not acceptable.  The price: the array is loaded on every GPU that loads the library and stays
+// until the process exits, and all calls share it.
+constexpr int HS_STATIC_ROWS = 64;         // most logits rows one call may pass
+constexpr size_t HS_STATIC_PART_BYTES = (size_t)HS_STATIC_ROWS * HS_ARGMAX_CHUNKS * 16;
+constexpr size_t HS_STATIC_BYTES = HS_STATIC_PART_BYTES + HS_STATIC_ROWS * 4;   // partials, then counters: 33 KB
+static __device__ __align__(256) unsigned char hs_static_scratch[HS_STATIC_BYTES];
+
+namespace {
+constexpr int HS_STATIC_MAX_DEVICES = 64;
+void *g_static_ptr[HS_STATIC_MAX_DEVICES];     // device address of hs_static_scratch, per device; null = not looked up yet
+}
+
+extern "C" int hs_argmax_static(const float *logits_dev, int V, int rows, int32_t *token_dev, float *margin_dev, void *stream) {
+    if (!logits_dev || !token_dev || V < 1 || rows < 1) return HS_ERR_INVALID_ARG;
+    if (rows > HS_STATIC_ROWS) return HS_ERR_SIZE;             // more rows than the built-in scratch holds
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= HS_STATIC_MAX_DEVICES) return HS_ERR_CUDA;
+    if (!g_static_ptr[dev]) {
+        // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+        // once per device, with that device current.
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, hs_static_scratch) != cudaSuccess || !p) return HS_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    unsigned char *base = static_cast<unsigned char *>(g_static_ptr[dev]);
+    int32_t *counters = reinterpret_cast<int32_t *>(base + HS_STATIC_PART_BYTES);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the tickets must start at zero whatever an earlier (possibly failed) call left behind
+    if (cudaMemsetAsync(counters, 0, (size_t)rows * 4, s) != cudaSuccess) return HS_ERR_CUDA;
+    ArgmaxArgs a{logits_dev, V, rows, 0, rows, token_dev, 0, margin_dev, reinterpret_cast<float4 *>(base), counters};
+    argmax_kernel<<<dim3(HS_ARGMAX_CHUNKS, rows, 1), 256, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
