@@ -242,6 +242,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
         }
         __syncthreads();
         if (tid < HD) {
+#pragma unroll 4
             for (int c = 0; c < nc; ++c) {
                 const float *src = pa0 + (size_t)(cb + c) * HS_MAX_GT * HD + tid;
 #pragma unroll

@@ -44,44 +44,75 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
             else { float2 t = *reinterpret_cast<const float2 *>(src); s[r][0] = t.x; s[r][1] = t.y; }
         }
 
-    // The state was written at least two kernels ago and the in-projection before this kernel only
-    // lets it start after its own wait, so everything older than that projection is complete: the
-    // state loads above are safe.  Everything below reads the in-projection.
-    pdl_wait();
-
-    // ---- causal conv + SiLU for the channels this block needs: its x strip, all of B and C
-    const int nch = SSM_PR + 2 * N;
+    // ---- still before the wait: everything of the conv that is a parameter or older state.
+    // A thread owns the channels tid, tid + 128, ... of this block's set: its x strip, all of B and C.
+    constexpr int NCH = SSM_PR + 2 * N;
+    constexpr int CPT = (NCH + SSM_THREADS - 1) / SSM_THREADS;
+    __shared__ float zs[HS_MAX_T][SSM_PR];
     const bool owner = (blockIdx.x == 0 && blockIdx.y == 0);   // writes the shared B|C channels' history
-    for (int c = threadIdx.x; c < nch; c += SSM_THREADS) {
-        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
-        const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
-        const float bias = a.conv_b[gc];
-        const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
-        float w0 = __ldcg(win), w1 = __ldcg(win + a.convd), w2 = __ldcg(win + 2 * a.convd);
-        const bool wr = c < SSM_PR || owner;
-        for (int i = 0; i < T; ++i) {
-            const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc);
-            const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
-            w0 = w1; w1 = w2; w2 = raw;
-            if (c < SSM_PR) xs[i][c] = act;
-            else if (c < SSM_PR + N) Bs[i][c - SSM_PR] = act;
-            else Cs[i][c - SSM_PR - N] = act;
-            if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
-        }
-        if (wr && a.win_out) {
-            float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
-            wo[0] = w0; wo[a.convd] = w1; wo[2 * a.convd] = w2;
+    float4 tap[CPT];
+    float bias[CPT], w0[CPT], w1[CPT], w2[CPT];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+            tap[q] = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
+            bias[q] = a.conv_b[gc];
+            const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
+            w0[q] = __ldcg(win); w1[q] = __ldcg(win + a.convd); w2[q] = __ldcg(win + 2 * a.convd);
         }
     }
+    const float Aexp = expf(a.A_log[h]), dtb = a.dt_bias[h], Dh = a.D[h];
+    // The state and the conv window were written at least two kernels ago and the in-projection before
+    // this kernel only lets it start after its own wait, so everything older than that projection is
+    // complete: the loads above are safe.  Everything below reads the in-projection.
+    pdl_wait();
+
+    // ---- raw conv inputs, gate inputs and dt of all T positions: one sweep of independent loads
+    for (int idx = threadIdx.x; idx < T * NCH; idx += SSM_THREADS) {
+        const int i = idx / NCH, c = idx - i * NCH;
+        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+        const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc);
+        if (c < SSM_PR) xs[i][c] = raw;
+        else if (c < SSM_PR + N) Bs[i][c - SSM_PR] = raw;
+        else Cs[i][c - SSM_PR - N] = raw;
+    }
+    for (int idx = threadIdx.x; idx < T * SSM_PR; idx += SSM_THREADS) {
+        const int i = idx / SSM_PR, c = idx - i * SSM_PR;
+        zs[i][c] = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c);
+    }
     if (threadIdx.x < T) {
-        const float dt = softplus_f(__ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) + a.dt_bias[h]);
+        const float dt = softplus_f(__ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) + dtb);
         dt_s[threadIdx.x] = dt;
-        a_s[threadIdx.x] = expf(-dt * expf(a.A_log[h]));
+        a_s[threadIdx.x] = expf(-dt * Aexp);
+    }
+    __syncthreads();
+    // ---- causal conv + SiLU in place (one thread walks the positions of its channel)
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+            float *col = c < SSM_PR ? &xs[0][c] : c < SSM_PR + N ? &Bs[0][c - SSM_PR] : &Cs[0][c - SSM_PR - N];
+            const int stride = c < SSM_PR ? SSM_PR : N;
+            const bool wr = c < SSM_PR || owner;
+            float v0 = w0[q], v1 = w1[q], v2 = w2[q];
+            for (int i = 0; i < T; ++i) {
+                const float raw = col[i * stride];
+                col[i * stride] = silu_f(bias[q] + tap[q].x * v0 + tap[q].y * v1 + tap[q].z * v2 + tap[q].w * raw);
+                v0 = v1; v1 = v2; v2 = raw;
+                if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+            }
+            if (wr && a.win_out) {
+                float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
+                wo[0] = v0; wo[a.convd] = v1; wo[2 * a.convd] = v2;
+            }
+        }
     }
     __syncthreads();
 
     // ---- recurrence over the T positions
-    const float Dh = a.D[h];
     float *sout = a.state_out + (size_t)b * a.out_seq_stride + ((size_t)h * a.P + p0 + warp * RPW) * N;
     for (int i = 0; i < T; ++i) {
         const float dec = a_s[i], dt = dt_s[i];
@@ -109,7 +140,7 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
         constexpr int LPV = 32 / RPW;
         if ((lane & (LPV - 1)) == 0) {
             const int r = lane / LPV, col = h * a.P + p0 + warp * RPW + r;
-            const float z = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + col);
+            const float z = zs[i][warp * RPW + r];
             a.g[(size_t)(rowbase + i) * a.di + col] = (y + Dh * xs[i][warp * RPW + r]) * silu_f(z);
         }
         // state after position i (verify: snapshot i; draft: the scratch state)
