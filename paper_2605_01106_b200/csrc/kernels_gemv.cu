@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
 }
 
 int g_sms = 148;
-constexpr size_t GV_SMEM_MAX = 200 * 1024;
+constexpr size_t GV_SMEM_MAX = 224 * 1024;
 constexpr size_t GV_SMEM_PAIR = 127 * 1024;   // below this the CTA of the next kernel fits beside it
 
 template <int R, int WR>
@@ -272,25 +272,27 @@ cudaError_t configure_gemv() {
 // Launches the projection.  a.max_oparts > 1 allows a K split for the residual epilogue; the number
 // of parts written is returned in *oparts (1 for the other epilogues).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts) {
-    // More than four activation rows are walked in passes over tiles that stay resident; when a K range
-    // is too wide for that (more than one chunk), the rows go in launches of four.
-    if (a.nrows > 4 && a.nrows <= GV_MAXROWS) {
+    // Activation rows beyond what one launch holds go in several launches (the weights are streamed again
+    // for each).  One launch takes up to 16 rows, walked in passes of at most four over tiles that stay
+    // resident; when a K range is too wide for that (more than one chunk) a launch takes four rows.
+    auto rows_launch = [&](int step) -> cudaError_t {
+        for (int r = 0; r < a.nrows; r += step) {
+            GemvArgs b = a;
+            b.nrows = a.nrows - r < step ? a.nrows - r : step;
+            b.x0 = a.x0 + (size_t)r * a.ldx0;
+            if (a.x1) b.x1 = a.x1 + (size_t)r * a.ldx1;
+            b.out = a.out + (size_t)r * a.ldo;
+            if (a.resid) b.resid = a.resid + (size_t)r * a.ldo;
+            cudaError_t e = launch_gemv(b, status, s, launches, oparts);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    };
+    if (a.nrows > 4) {
         const int K = a.K0 > a.K1 ? a.K0 : a.K1;
         const bool splittable = a.epi == EPI_RESID && a.max_oparts > 1;
-        const int kr = splittable ? 1280 : K;
-        if ((splittable ? (a.K0 + a.K1 + 3) / 4 : K) > 1280 && kr > 0) {
-            for (int r = 0; r < a.nrows; r += 4) {
-                GemvArgs b = a;
-                b.nrows = a.nrows - r < 4 ? a.nrows - r : 4;
-                b.x0 = a.x0 + (size_t)r * a.ldx0;
-                if (a.x1) b.x1 = a.x1 + (size_t)r * a.ldx1;
-                b.out = a.out + (size_t)r * a.ldo;
-                if (a.resid) b.resid = a.resid + (size_t)r * a.ldo;
-                cudaError_t e = launch_gemv(b, status, s, launches, oparts);
-                if (e != cudaSuccess) return e;
-            }
-            return cudaSuccess;
-        }
+        if ((splittable ? (a.K0 + a.K1 + 3) / 4 : K) > 1280) return rows_launch(4);
+        if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     }
     if ((a.K0 & 255) || (a.K1 & 255) || a.K0 < 256 || a.O < 2 || a.nrows < 1 || a.nrows > GV_MAXROWS) return cudaErrorInvalidValue;
     GemvGeo g{};
@@ -320,21 +322,26 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     const int nrow_max = ceil_div(units, g.NR) * g.unit;
     // tile: 4 weight rows per warp when that already gives every warp a tile, else 8
     const int WR = nrow_max <= 4 * GV_WARPS ? 4 : 8;
-    // chunk of at most 1280 columns, as even as possible
-    const int nch = ceil_div(g.krmax, 1280);
-    g.kc = ceil_div(ceil_div(g.krmax, nch), 256) * 256;
-    const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * ceil_div(g.krmax, g.kc);
-    const size_t tile = (size_t)WR * g.kc * 2;
+    // chunk of at most 1280 columns, as even as possible; narrower if the ring would not fit
     const size_t xs = (size_t)a.nrows * g.krmax * 4;
     g.off_x = 1024;
     g.off_nw = (int)((g.off_x + xs + 127) / 128 * 128);
     g.off_ring = g.off_nw + (a.norm_w ? g.krmax * 4 : 0);
+    const int ring_warps = ceil_div(nrow_max, WR) < GV_WARPS ? ceil_div(nrow_max, WR) : GV_WARPS;
+    size_t tile = 0;
+    for (int nch = ceil_div(g.krmax, 1280);; ++nch) {
+        g.kc = ceil_div(ceil_div(g.krmax, nch), 256) * 256;
+        tile = (size_t)WR * g.kc * 2;
+        if (g.off_ring + tile * ring_warps <= GV_SMEM_MAX || g.kc == 256) break;
+    }
+    const int nchunks = ceil_div(g.krmax, g.kc);
+    if (a.nrows > 4 && nchunks > 1) return rows_launch(4);      // passes need every chunk of a row group resident
+    const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * nchunks;
     int D = 1;
     while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= GV_SMEM_PAIR) ++D;
     g.D = D;
-    const int ring_warps = ceil_div(nrow_max, WR) < GV_WARPS ? ceil_div(nrow_max, WR) : GV_WARPS;
     const size_t smem = g.off_ring + tile * ring_warps * D;
-    if (smem > GV_SMEM_MAX) return cudaErrorInvalidValue;
+    if (smem > GV_SMEM_MAX) return a.nrows > 1 ? rows_launch((a.nrows + 1) / 2) : cudaErrorInvalidValue;
     if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
     if (launches) ++*launches;
     // rows held in registers per pass: as even as possible over ceil(nrows / 4) passes

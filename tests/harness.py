@@ -36,6 +36,8 @@ def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
     """Committed recurrent state, conv window and KV rows of every sequence against the oracle."""
     worst = 0.0
     for b, o in enumerate(seqs):
+        if o is None:
+            continue
         kv_len, pending = eng.get_context(b)
         assert kv_len == o.len, ("kv_len", b, kv_len, o.len)
         assert pending == o.pending, ("pending", b, pending, o.pending)
@@ -68,7 +70,8 @@ def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
 
 def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_every=1, check_logits=True,
                torch=None):
-    """seqs: oracle sequences, one per active GPU sequence, already holding the same context.
+    """seqs: oracle sequences, one per active GPU sequence, already holding the same context; an entry may be
+    None for a sequence that runs on the GPU without being compared (then `forced` is required).
     forced: None (real acceptance) or int array [batch][rounds] of forced accept lengths."""
     import torch as _torch
     torch = torch or _torch
@@ -79,6 +82,10 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
         # ---- oracle: draft (with logits, for the margins), then the whole round on those candidates
         ora = []
         for b, o in enumerate(seqs):
+            if o is None:
+                assert forced is not None
+                ora.append(None)
+                continue
             if k > 0:
                 d, dlg = o.draft_only(k, want_logits=True)
                 dm = np.array([oracle.argmax_margin(dlg[i])[1] for i in range(k)])
@@ -96,6 +103,8 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
         gc, _, _ = eng.get_round(k)
         resync = False
         for b in range(B):
+            if ora[b] is None:
+                continue
             for i in range(T):
                 if gc[b, i] != ora[b]["cand"][i]:
                     m = ora[b]["draft_margin"][i - 1] if i > 0 else np.inf
@@ -103,12 +112,14 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
                     rep.listed.append((r, b, "draft", i, float(m)))
                     resync = True
                     break
-        cand_all = np.stack([o["cand"] for o in ora]).astype(np.int32)
+        cand_all = np.stack([o["cand"] if o is not None else gc[b] for b, o in enumerate(ora)]).astype(np.int32)
         eng.verify(k, torch.from_numpy(cand_all).to(dev) if resync else None)
         gc, gg, gm = eng.get_round(k)
         assert np.array_equal(gc, cand_all)
         force_accept = resync
         for b in range(B):
+            if ora[b] is None:
+                continue
             for i in range(T):
                 if gg[b, i] != ora[b]["g"][i]:
                     m = ora[b]["margin"][i]
@@ -118,6 +129,8 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
         if check_logits:
             lg = eng.get_logits(B * T).reshape(B, T, V)
             for b in range(B):
+                if ora[b] is None:
+                    continue
                 err = np.abs(lg[b] - ora[b]["logits"]).max()
                 assert err <= LOGIT_TOL, ("logits", r, b, err)
                 rep.max_logit_err = max(rep.max_logit_err, float(err))
@@ -125,11 +138,15 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
         #      narrow-margin position made the GPU's own decision differ)
         fn_dev = fx_dev = None
         if forced is not None or force_accept:
-            fn_dev = torch.tensor([o["n"] for o in ora], dtype=torch.int32, device=dev)
+            fn_dev = torch.tensor([o["n"] if o is not None else int(forced[b][r]) for b, o in enumerate(ora)],
+                                  dtype=torch.int32, device=dev)
         if force_accept:
-            fx_dev = torch.tensor([int(o["emitted"][-1]) for o in ora], dtype=torch.int32, device=dev)
+            fx_dev = torch.tensor([int(o["emitted"][-1]) if o is not None else -1 for o in ora], dtype=torch.int32, device=dev)
         n, em = eng.accept_rollback(fn_dev, fx_dev, readback=True)
         for b in range(B):
+            if ora[b] is None:
+                assert n[b] == forced[b][r]
+                continue
             assert n[b] == ora[b]["n"], ("accept length", r, b, n[b], ora[b]["n"])
             want = ora[b]["emitted"]
             assert np.array_equal(em[b, : n[b] + 1], want), ("emitted", r, b, em[b], want)
@@ -140,3 +157,30 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
         if check_states_every and (r % check_states_every == 0 or r == rounds - 1):
             compare_states(eng, seqs, shape, rep, kv_rows=2 * T + 2)
     return rep
+
+
+def inject_context(eng, oseq, shape, b, kv_len, pending, seed=3):
+    """Give GPU sequence b and the oracle sequence `oseq` (or None: GPU only, recurrent state only) the same
+    synthetic context: seeded recurrent state, conv window and kv_len KV rows per layer, plus the pending token."""
+    s = shape
+    for l in range(s.L):
+        t = s.layer_type(l)
+        if t != hi.LAYER_ATT:
+            kind, ctx = (hs.STATE_SSM, hi.CTX_SSM) if t == hi.LAYER_PAR else (hs.STATE_GDN, hi.CTX_GDN)
+            st = hi.injected_state(s, l, b, ctx, seed)
+            cv = hi.injected_state(s, l, b, hi.CTX_CONV, seed)
+            eng.import_state(l, b, kind, st)
+            eng.import_state(l, b, hs.STATE_CONV, cv)
+            if oseq is not None:
+                (oseq.ssm() if t == hi.LAYER_PAR else oseq.gdn())[l] = st
+                oseq.conv()[l] = cv
+        if t != hi.LAYER_GDN and oseq is not None and kv_len > 0:
+            K = hi.injected_kv(s, l, b, kv_len, hi.CTX_K, seed)
+            V = hi.injected_kv(s, l, b, kv_len, hi.CTX_V, seed)
+            eng.import_state(l, b, hs.STATE_K, K)
+            eng.import_state(l, b, hs.STATE_V, V)
+            oseq.k()[l, :kv_len] = K
+            oseq.v()[l, :kv_len] = V
+    eng.set_context(b, kv_len, pending)
+    if oseq is not None:
+        oseq.set(kv_len, pending)

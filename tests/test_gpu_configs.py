@@ -1,0 +1,99 @@
+"""Parity of the CUDA library with the CPU oracle at the full sizes of the five workloads, in the launch
+configuration the benchmark times (CUDA graphs on).  Contexts too long to prefill on the CPU are injected:
+the same seeded recurrent state, conv window and KV rows are given to both sides (prefill itself is compared
+on the small configurations).  Every comparison is round by round: candidates, argmax, accept length,
+emitted tokens bit-exact where the oracle's margin exceeds 1e-2, logits within 2e-2, states within 1e-3."""
+import numpy as np
+import pytest
+
+import hs_inputs as hi
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    import oracle
+    from paper_2605_01106_b200 import build, binding
+    build.build()
+    import harness
+    return dict(torch=torch, oracle=oracle, hs=binding, harness=harness)
+
+
+_W = {}
+
+
+def make(env, name, batch, max_k, cap, checked, ctx_lens, small_init="jitter"):
+    s = hi.CONFIGS[name]
+    if (name, small_init) not in _W:
+        _W.clear()                                     # one large blob at a time
+        _W[(name, small_init)] = hi.make_weights(s, 0, small_init)
+    blob, table = _W[(name, small_init)]
+    eng = env["hs"].Engine(s, blob, max_batch=batch, max_k=max_k, kv_capacity=cap, flags=env["hs"].HS_FLAG_GRAPHS)
+    model = env["oracle"].Model(s, blob, table, cap)
+    seqs = []
+    for b in range(batch):
+        q = model.new_seq() if b in checked else None
+        pending = int(hi.make_prompt(s.V, 1, seq=1000 + b)[0])
+        env["harness"].inject_context(eng, q, s, b, int(ctx_lens[b]), pending)
+        seqs.append(q)
+    eng.set_batch(batch)
+    return s, eng, model, seqs
+
+
+def test_cfg2_full_size_all_k(env):
+    s, eng, model, seqs = make(env, "cfg2_0p5b", 1, 8, 640, {0}, [512])
+    rep = None
+    for k, rounds in ((1, 2), (2, 3), (4, 2), (8, 1)):
+        forced = [hi.forced_accept(k, rounds, seq=k)]
+        rep = env["harness"].run_rounds(eng, seqs, s, k, rounds, forced=forced, rep=rep)
+    print(rep)
+    assert eng.device_status() == 0 and rep.rounds == 8
+
+
+def test_cfg2_full_size_real_acceptance(env):
+    s, eng, model, seqs = make(env, "cfg2_0p5b", 1, 2, 600, {0}, [512])
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 3)
+    print(rep)
+    assert eng.device_status() == 0
+
+
+def test_cfg4_sequential_full_size(env):
+    s, eng, model, seqs = make(env, "cfg4_seq", 1, 4, 1100, {0}, [1024])
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 2, forced=[hi.forced_accept(2, 2, seq=1)])
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=[hi.forced_accept(4, 1, seq=2)], rep=rep)
+    print(rep)
+    assert eng.device_status() == 0
+
+
+def test_cfg3_3b_batch1(env):
+    s, eng, model, seqs = make(env, "cfg3_3b", 1, 4, 2100, {0}, [2048], small_init="unit")
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 1, forced=[[1]])
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=[[2]], rep=rep)
+    print(rep)
+    assert eng.device_status() == 0
+
+
+def test_cfg3_3b_batch8_two_checked(env):
+    s, eng, model, seqs = make(env, "cfg3_3b", 8, 4, 2100, {0, 5}, [2048] * 8, small_init="unit")
+    forced = [hi.forced_accept(4, 1, seq=b) for b in range(8)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=forced)
+    print(rep)
+    assert eng.device_status() == 0
+
+
+def test_cfg5_batch64_ragged_sampled(env):
+    # 64 sequences with contexts uniform in [4096, 16384]; four of them carry a full seeded context on both
+    # sides and are compared, the others run beside them with their own accept pattern (ragged rollback)
+    s = hi.CONFIGS["cfg5_b64"]
+    lens = hi.context_lengths(64, 4096, 16384)
+    checked = {0, 17, 38, 63}
+    s, eng, model, seqs = make(env, "cfg5_b64", 64, 4, 16384 + 32, checked, lens)
+    forced = [hi.forced_accept(4, 2, seq=b) for b in range(64)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 2, forced=forced)
+    print(rep, sorted(set(int(x) for x in lens))[:3])
+    for b in range(64):
+        kv, _ = eng.get_context(b)
+        assert kv == lens[b] + int((np.array(forced[b]) + 1).sum())
+    assert len(rep.n_hist) >= 2 and eng.device_status() == 0
