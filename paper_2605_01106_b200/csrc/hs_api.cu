@@ -178,8 +178,19 @@ double gemv_bytes(const GemvArgs &a) {
 //   draft = false: full model M_H (verify);  draft = true: draft model M_S, one position,
 //   reading candidate column `col` and, for step > 0, the scratch state of the previous step.
 // ------------------------------------------------------------------------------------------------
+// keys per attention CTA for this launch: small enough to spread a short context over the eight CTAs of one
+// cluster (which combine their partials in shared memory), never below the size the partial buffers were
+// laid out for
+int attn_chunk(const hs_model *m, int T, int b0, int nb) {
+    int maxlen = 0;
+    for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
+    const int want = maxlen + T <= 256 ? 32 : maxlen + T <= 512 ? 64 : 128;
+    return want > m->att_chunk ? want : m->att_chunk;
+}
+
 int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     const hs_config &c = m->c;
+    const int at_chunk = draft ? m->att_chunk : attn_chunk(m, T, b0, nb);
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
@@ -253,7 +264,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             aa.Kc = m->Kc + ly.al * per_layer; aa.Vc = m->Vc + ly.al * per_layer; aa.cap = c.kv_capacity;
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
-            aa.chunk = m->att_chunk; aa.nch = m->att_nch; aa.T = T; aa.b0 = b0; aa.nb = nb;
+            aa.chunk = at_chunk; aa.nch = (c.kv_capacity + at_chunk - 1) / at_chunk; aa.T = T; aa.b0 = b0; aa.nb = nb;
             PROF(HS_PROF_ATTN, 0, launch_attn(aa, s), "attention");
             ++m->launches;
         }
@@ -514,7 +525,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
-    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
+    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_chunk(m, T, 0, nb) << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
     return HS_OK;

@@ -17,12 +17,15 @@
 //    last (ticket counter, no spinning) merges them in chunk order, so the result is reproducible.
 #include "hs_internal.h"
 #include "hs_device.cuh"
+#include <cooperative_groups.h>
 
 namespace {
 using namespace hsd;
+namespace cg = cooperative_groups;
 
 constexpr int AT_THREADS = 128;
 constexpr int AT_WARPS = 4;
+constexpr int AT_CL = 8;               // CTAs (chunks) per thread-block cluster
 
 template <int HD>
 struct AttnSmem {
@@ -60,7 +63,11 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     // ---- before the wait: kv_len, the cached chunk, the RoPE rows
     const int len = __ldcg(a.kv_len + b);
     const int nsplit = max(1, (len + CK - 1) / CK);
-    if (split >= nsplit) return;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank(), cl = split / AT_CL;
+    if (cl * AT_CL >= nsplit) return;             // the whole cluster is beyond the cache: nobody reaches a barrier
+    // a CTA beyond the last chunk of a live cluster has no keys: it contributes (m, l) = (-inf, 0) and still
+    // takes its share of the cluster's reduction
     const bool last = split == nsplit - 1;
     const int c0 = split * CK, ncache = max(0, min(len, c0 + CK) - c0);
     const bool overflow = len + T > a.cap;       // never write past the cache; the host reports the status word
@@ -89,14 +96,31 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     // ---- queries: RoPE at position len + i, pre-multiplied by 1/sqrt(hd)
     const int rowbase = lb * T;
     const float scale = rsqrtf((float)HD);
-    for (int idx = tid; idx < GT * (HD / 2); idx += AT_THREADS) {
-        const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
-        const int gq = qi / T, i = qi - gq * T;
-        const float *src = a.zx + (size_t)(rowbase + i) * a.in_ld + a.q_off + (kh * G + gq) * HD;
-        const float2 cs = rope_s[i * (HD / 2) + e];
-        const float x0 = __ldcg(src + e), x1 = __ldcg(src + e + HD / 2);
-        q_s[qi * HD + e] = (x0 * cs.x - x1 * cs.y) * scale;
-        q_s[qi * HD + e + HD / 2] = (x1 * cs.x + x0 * cs.y) * scale;
+    for (int base = 0; base < GT * (HD / 2); base += AT_THREADS * 6) {
+        // six elements per thread and sweep: all twelve loads are issued before the first is used
+        float x0[6], x1[6];
+#pragma unroll
+        for (int u = 0; u < 6; ++u) {
+            const int idx = base + u * AT_THREADS + tid;
+            x0[u] = x1[u] = 0.f;
+            if (idx < GT * (HD / 2)) {
+                const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
+                const int gq = qi / T, i = qi - gq * T;
+                const float *src = a.zx + (size_t)(rowbase + i) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HD / 2);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 6; ++u) {
+            const int idx = base + u * AT_THREADS + tid;
+            if (idx < GT * (HD / 2)) {
+                const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
+                const int i = qi % T;
+                const float2 cs = rope_s[i * (HD / 2) + e];
+                q_s[qi * HD + e] = (x0[u] * cs.x - x1[u] * cs.y) * scale;
+                q_s[qi * HD + e + HD / 2] = (x1[u] * cs.x + x0[u] * cs.y) * scale;
+            }
+        }
     }
     int nkeys = ncache;
     if (last) {
@@ -120,9 +144,9 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     }
     bool landed = true;
     if (ncache > 0) landed = mbar_wait(bar, 0);
-    if (!__syncthreads_and(landed)) {
+    if (!__syncthreads_and(landed)) {             // a copy never landed: report it, contribute nothing, keep the barriers
         if (tid == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
-        return;
+        nkeys = 0;
     }
 
     // ---- scores: lane = key (tiles of 32), warp w takes query rows w, w + 4, ...
@@ -189,42 +213,76 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
         }
     }
     float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
-    if (nsplit == 1) {
-        if (tid < HD) {
-#pragma unroll
-            for (int qi = 0; qi < GTB; ++qi)
-                if (qi < GT) {
-                    const int gq = qi / T, i = qi - gq * T;
-                    o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + tid] = acc[qi] / ml_s[2 * qi + 1];
-                }
-        }
-        return;
-    }
-    // ---- several chunks: publish the partial, the last block to arrive merges in chunk order
-    const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
-    float *pa = a.part_acc + (pbase + split) * HS_MAX_GT * HD;
-    float *pm = a.part_ml + (pbase + split) * HS_MAX_GT * 2;
+    // ---- combine the chunks of this cluster through distributed shared memory: every CTA leaves its partial
+    //      (m, l, acc) in its own shared memory, rank r then sums output dims [r * DS, (r + 1) * DS) over all ranks
+    constexpr int DS = HD / AT_CL;
+    float *acc_s = q_s;                                      // [GT][HD]; the queries are no longer needed
     if (tid < HD) {
 #pragma unroll
-        for (int qi = 0; qi < GTB; ++qi) if (qi < GT) pa[qi * HD + tid] = acc[qi];
+        for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc_s[qi * HD + tid] = acc[qi];
     }
-    if (tid < 2 * GT) pm[tid] = ml_s[tid];
+    cluster.sync();
+    float *mlr_s = p_s;                                      // [AT_CL][GT][2] copies of every rank's (m, l)
+    float *wr_s = mlr_s + AT_CL * HS_MAX_GT * 2;             // [AT_CL][GT] merge weights
+    float *Md_s = wr_s + AT_CL * HS_MAX_GT;                  // [GT][2] merged (M, den)
+    for (int idx = tid; idx < AT_CL * GT * 2; idx += AT_THREADS) {
+        const int r = idx / (GT * 2), rem = idx - r * (GT * 2);
+        mlr_s[idx] = cluster.map_shared_rank(ml_s, r)[rem];
+    }
+    __syncthreads();
+    if (tid < GT) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < AT_CL; ++r) M = fmaxf(M, mlr_s[(r * GT + tid) * 2]);
+        float den = 0.f;
+#pragma unroll
+        for (int r = 0; r < AT_CL; ++r) {
+            const float mr = mlr_s[(r * GT + tid) * 2];
+            const float w = mr == -INFINITY ? 0.f : expf(mr - M);
+            wr_s[r * GT + tid] = w;
+            den = fmaf(w, mlr_s[(r * GT + tid) * 2 + 1], den);
+        }
+        Md_s[2 * tid] = M; Md_s[2 * tid + 1] = den;
+    }
+    __syncthreads();
+    const int nclus = (nsplit + AT_CL - 1) / AT_CL;
+    const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
+    for (int idx = tid; idx < GT * DS; idx += AT_THREADS) {
+        const int qi = idx / DS, d = crank * DS + (idx - qi * DS);
+        float v[AT_CL];
+#pragma unroll
+        for (int r = 0; r < AT_CL; ++r) v[r] = cluster.map_shared_rank(acc_s, r)[qi * HD + d];
+        float sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < AT_CL; ++r) sum = fmaf(wr_s[r * GT + qi], v[r], sum);
+        if (nclus == 1) {
+            const int gq = qi / T, i = qi - gq * T;
+            o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d] = sum / Md_s[2 * qi + 1];
+        } else {
+            a.part_acc[(pbase + cl) * HS_MAX_GT * HD + qi * HD + d] = sum;
+        }
+    }
+    if (nclus > 1 && crank == 0 && tid < 2 * GT) a.part_ml[(pbase + cl) * HS_MAX_GT * 2 + tid] = Md_s[tid];
+    cluster.sync();                                          // peers may still be reading this CTA's shared memory
+    if (nclus == 1) return;
+    // ---- several clusters: the CTA that arrives last merges the cluster partials in order
     __threadfence();
     __syncthreads();
     if (tid == 0) ticket_s = atomicAdd(a.counters + b * a.kvh + kh, 1);
     __syncthreads();
-    if (ticket_s != nsplit - 1) return;
+    if (ticket_s != nclus * AT_CL - 1) return;
     __threadfence();
     if (tid == 0) a.counters[b * a.kvh + kh] = 0;          // ready for the next launch
+    const int nmerge = nclus;
     const float *pa0 = a.part_acc + pbase * HS_MAX_GT * HD;
     const float *pm0 = a.part_ml + pbase * HS_MAX_GT * 2;
     float *w_s = p_s;                                        // [GT][PST]: merge weights of PST chunks per pass
     for (int qi = warp; qi < GT; qi += AT_WARPS) {
         float M = -INFINITY;
-        for (int c = lane; c < nsplit; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+        for (int c = lane; c < nmerge; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
         M = warp_max(M);
         float den = 0.f;
-        for (int c = lane; c < nsplit; c += 32) {
+        for (int c = lane; c < nmerge; c += 32) {
             const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
             den = fmaf(expf(mlv.x - M), mlv.y, den);
         }
@@ -233,8 +291,8 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     }
 #pragma unroll
     for (int qi = 0; qi < GTB; ++qi) acc[qi] = 0.f;
-    for (int cb = 0; cb < nsplit; cb += PST) {               // chunks in passes of PST
-        const int nc = min(PST, nsplit - cb);
+    for (int cb = 0; cb < nmerge; cb += PST) {               // chunks in passes of PST
+        const int nc = min(PST, nmerge - cb);
         __syncthreads();                                     // ml_s ready / previous pass done with w_s
         for (int idx = tid; idx < GT * nc; idx += AT_THREADS) {
             const int qi = idx / nc, c = idx - qi * nc;
@@ -242,11 +300,19 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
         }
         __syncthreads();
         if (tid < HD) {
-#pragma unroll 4
-            for (int c = 0; c < nc; ++c) {
-                const float *src = pa0 + (size_t)(cb + c) * HS_MAX_GT * HD + tid;
+            constexpr int MB = 64 / GTB < 1 ? 1 : 64 / GTB;       // chunks whose partials are fetched together
+            for (int c = 0; c < nc; c += MB) {
+                float v[MB][GTB];
 #pragma unroll
-                for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc[qi] = fmaf(w_s[qi * PST + c], __ldcg(src + qi * HD), acc[qi]);
+                for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+                    for (int qi = 0; qi < GTB; ++qi)
+                        v[mb][qi] = (c + mb < nc && qi < GT) ? __ldcg(pa0 + ((size_t)(cb + c + mb) * HS_MAX_GT + qi) * HD + tid) : 0.f;
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+                    for (int qi = 0; qi < GTB; ++qi)
+                        if (c + mb < nc && qi < GT) acc[qi] = fmaf(w_s[qi * PST + c + mb], v[mb][qi], acc[qi]);
             }
         }
     }
@@ -262,8 +328,8 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
 
 template <int HD, int GTB>
 cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
-    dim3 grid(a.nch, a.kvh, a.nb);
-    return launch_pdl(attn_kernel<HD, GTB>, grid, dim3(AT_THREADS), AttnSmem<HD>::total(a.chunk), s, a);
+    dim3 grid((a.nch + AT_CL - 1) / AT_CL * AT_CL, a.kvh, a.nb);
+    return launch_pdl_cluster(attn_kernel<HD, GTB>, grid, dim3(AT_THREADS), AttnSmem<HD>::total(a.chunk), s, AT_CL, a);
 }
 
 template <int HD, int GTB>
