@@ -1,20 +1,25 @@
 // Verify-mode attention: the T = k+1 new positions of a sequence attend over its KV cache plus the
 // new rows themselves (causal among the new ones), grouped-query heads, split over the cache length.
 //
-// grid = (max splits, kv heads, sequences); one CTA = one chunk of CK cached keys for the G*T query
-// rows that share its KV head (G = q heads per KV head).
-//  * Before the programmatic-dependent-launch wait the CTA reads kv_len (written at least two
-//    kernels earlier), starts two bulk asynchronous copies - its K chunk and its V chunk, each one
-//    contiguous piece of the cache - and fetches the RoPE rows of the new positions.
-//  * After the wait it rotates and scales the queries into shared memory; the CTA of the last chunk
-//    also rotates the T new K rows, rounds K and V to bf16 exactly as they are cached, appends them to
-//    the cache and keeps them in shared memory behind the cached keys, so nothing written by this
-//    launch is read back from global memory by another block.
-//  * Scores: lane = key, each warp takes a subset of the query rows; the dense key rows are read in a
-//    per-lane rotated chunk order so that the 128-bit reads do not collide on a bank.  One softmax per
-//    chunk (the whole chunk is resident), then P V with thread = output dimension.
-//  * Several chunks: every CTA publishes an un-normalised partial (m, l, acc); the CTA that arrives
-//    last (ticket counter, no spinning) merges them in chunk order, so the result is reproducible.
+// grid = (chunks rounded up to clusters of 8, kv heads, sequences); one CTA = one chunk of CK cached
+// keys for the G*T query rows that share its KV head (G = q heads per KV head).
+//  * Before the programmatic-dependent-launch wait the CTA reads kv_len (written at least two kernels
+//    earlier), starts the asynchronous copies of its K and V chunk into padded shared-memory rows and
+//    fetches the RoPE rows of the new positions.
+//  * After the wait it rotates and scales the queries; the CTA of the last chunk also rotates the T new
+//    K rows, rounds K and V to bf16 exactly as they are cached, appends them to the cache and keeps them
+//    in shared memory behind the cached keys, so nothing written by this launch is read back from
+//    global memory by another block.
+//  * Q K^T and P V run on the tensor cores (mma.sync m16n8k16, bf16 operands, fp32 accumulation).  K and
+//    V are bf16 in the cache and enter exactly; the fp32 queries and probabilities are split into a
+//    bf16 head and a bf16 remainder (two MMAs), which keeps the products exact to 2^-17 - the
+//    comparison with the CPU oracle allows 1e-3 on states fed by this output.
+//    Scores: a warp takes 32 keys at a time for all query rows; one softmax per chunk (the whole chunk is
+//    resident); P V: a warp takes a quarter of the head dimension over all keys.
+//  * The up to eight chunks of a cluster leave (m, l, acc) in their own shared memory and combine them
+//    through distributed shared memory, rank r summing an eighth of the output dimensions.  Longer
+//    caches span several clusters: each publishes one partial and the CTA that arrives last (ticket
+//    counter, no spinning) merges them in order, so the result is reproducible.
 #include "hs_internal.h"
 #include "hs_device.cuh"
 #include <cooperative_groups.h>
@@ -27,37 +32,78 @@ constexpr int AT_THREADS = 128;
 constexpr int AT_WARPS = 4;
 constexpr int AT_CL = 8;               // CTAs (chunks) per thread-block cluster
 
-template <int HD>
-struct AttnSmem {
-    // offsets in bytes for a chunk capacity of ck cached keys (+ up to 16 new ones)
-    static __host__ __device__ int keys(int ck) { return ck + 16; }
-    static __host__ __device__ size_t k_off() { return 128; }
-    static __host__ __device__ size_t v_off(int ck) { return k_off() + (size_t)keys(ck) * HD * 2; }
-    static __host__ __device__ size_t q_off(int ck) { return v_off(ck) + (size_t)keys(ck) * HD * 2; }
-    static __host__ __device__ size_t p_off(int ck) { return q_off(ck) + (size_t)HS_MAX_GT * HD * 4; }
-    static __host__ __device__ size_t ml_off(int ck) { return p_off(ck) + (size_t)HS_MAX_GT * keys(ck) * 4; }
-    static __host__ __device__ size_t rope_off(int ck) { return ml_off(ck) + (size_t)HS_MAX_GT * 2 * 4; }
-    static __host__ __device__ size_t total(int ck) { return rope_off(ck) + (size_t)HS_MAX_T * (HD / 2) * 8; }
+struct AttnLayout {
+    int kstr, keys, mrows, pstr, sstr;
+    size_t k_off, v_off, q_off, s_off, p_off, ml_off, rope_off, red_off, total;
 };
+// shared-memory carve-up for head dim hd, chunk ck, gt query rows
+__host__ __device__ inline AttnLayout attn_layout(int hd, int ck, int gt) {
+    AttnLayout L;
+    L.kstr = hd + 8;                       // padded bf16 row: 16-byte aligned, conflict-free ldmatrix
+    L.keys = ck + 16;                      // cached keys + the new rows, rounded to the MMA k step
+    L.mrows = (gt + 15) / 16 * 16;
+    L.pstr = L.keys + 8;
+    L.sstr = L.keys + 4;
+    size_t o = 128;
+    L.k_off = o; o += (size_t)L.keys * L.kstr * 2;
+    L.v_off = o; o += (size_t)L.keys * L.kstr * 2;
+    L.q_off = o; o += (size_t)2 * L.mrows * L.kstr * 2;       // bf16 head | remainder; later the fp32 partial acc
+    L.s_off = o; o += (size_t)L.mrows * L.sstr * 4;           // raw scores fp32
+    L.p_off = o; o += (size_t)2 * L.mrows * L.pstr * 2;       // probabilities: bf16 head | remainder
+    L.ml_off = o; o += (size_t)HS_MAX_GT * 2 * 4;
+    L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
+    L.red_off = o; o += (size_t)(AT_CL * HS_MAX_GT * 3 + HS_MAX_GT * 2) * 4;
+    L.total = (o + 127) / 128 * 128;
+    return L;
+}
 
-template <int HD, int GTB>      // GTB: compile-time bound of G*T (16, 32 or 48)
+__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// x = head + remainder, both bf16 (round to nearest): exact to 2^-17 relative
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &h, __nv_bfloat16 &l) {
+    h = __float2bfloat16_rn(x);
+    l = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+template <int HD, int MT>       // MT: 16-row tiles of query rows (G*T <= 16 * MT)
 __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
-    using L = AttnSmem<HD>;
-    constexpr int NC = HD / 8;             // 16-byte chunks per key row
     extern __shared__ __align__(128) unsigned char smraw[];
     const int CK = a.chunk;
-    uint64_t *bar = reinterpret_cast<uint64_t *>(smraw);
-    __nv_bfloat16 *K_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L::k_off());      // [CK + 16][HD]
-    __nv_bfloat16 *V_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L::v_off(CK));
-    float *q_s = reinterpret_cast<float *>(smraw + L::q_off(CK));                    // [GT][HD] rotated, pre-scaled
-    float *p_s = reinterpret_cast<float *>(smraw + L::p_off(CK));                    // [GT][CK + 16]
-    float *ml_s = reinterpret_cast<float *>(smraw + L::ml_off(CK));                  // [GT][2]
-    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L::rope_off(CK));            // [T][HD/2]
+    const int G = a.qh / a.kvh, T = a.T, GT = G * T;
+    const AttnLayout L = attn_layout(HD, CK, GT);
+    const int KSTR = L.kstr, PSTR = L.pstr, SSTR = L.sstr;
+    __nv_bfloat16 *K_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.k_off);         // [keys][KSTR]
+    __nv_bfloat16 *V_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.v_off);
+    __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.q_off);        // [mrows][KSTR] rotated, pre-scaled
+    __nv_bfloat16 *Ql_s = Qh_s + (size_t)L.mrows * KSTR;
+    float *s_s = reinterpret_cast<float *>(smraw + L.s_off);                         // [mrows][SSTR]
+    __nv_bfloat16 *Ph_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.p_off);        // [mrows][PSTR]
+    __nv_bfloat16 *Pl_s = Ph_s + (size_t)L.mrows * PSTR;
+    float *ml_s = reinterpret_cast<float *>(smraw + L.ml_off);                       // [GT][2]
+    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);                 // [T][HD/2]
+    float *red_s = reinterpret_cast<float *>(smraw + L.red_off);
     __shared__ int ticket_s;
 
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = a.qh / a.kvh, T = a.T, GT = G * T, PST = L::keys(CK);
+    const uint32_t tinv = (65536u + T - 1) / T;      // x / T == (x * tinv) >> 16 for the small x used here
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
     // ---- before the wait: kv_len, the cached chunk, the RoPE rows
@@ -70,55 +116,54 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     // takes its share of the cluster's reduction
     const bool last = split == nsplit - 1;
     const int c0 = split * CK, ncache = max(0, min(len, c0 + CK) - c0);
-    const bool overflow = len + T > a.cap;       // never write past the cache; the host reports the status word
-    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    if (tid == 0) { mbar_init(bar, 1); mbar_fence_init(); }
-    __syncthreads();
-    if (tid == 0 && ncache > 0 && !overflow) {
-        const uint32_t bytes = (uint32_t)ncache * HD * 2;
-        mbar_expect_tx(bar, 2 * bytes);
-        bulk_g2s(K_s, Kb + (size_t)c0 * HD, bytes, bar);
-        bulk_g2s(V_s, Vb + (size_t)c0 * HD, bytes, bar);
-    }
-    if (!overflow)
-        for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
-            const int i = idx / (HD / 2), e = idx - i * (HD / 2);
-            rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
-        }
-    pdl_wait();
-    if (overflow) {
+    if (len + T > a.cap) {                        // never write past the cache; the host reports the status word
         if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
         return;
     }
+    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    for (int idx = tid; idx < ncache * (HD / 8); idx += AT_THREADS) {
+        const int j = idx / (HD / 8), c = idx - j * (HD / 8);
+        cp_async16(K_s + (size_t)j * KSTR + 8 * c, Kb + (size_t)(c0 + j) * HD + 8 * c);
+        cp_async16(V_s + (size_t)j * KSTR + 8 * c, Vb + (size_t)(c0 + j) * HD + 8 * c);
+    }
+    cp_async_commit();
+    for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
+        const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+        rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
+    }
+    pdl_wait();
     __syncthreads();                        // rope_s complete
 
-    // ---- queries: RoPE at position len + i, pre-multiplied by 1/sqrt(hd)
+    // ---- queries: RoPE at position len + i, pre-multiplied by 1/sqrt(hd), split into bf16 head + remainder
     const int rowbase = lb * T;
     const float scale = rsqrtf((float)HD);
-    for (int base = 0; base < GT * (HD / 2); base += AT_THREADS * 6) {
-        // six elements per thread and sweep: all twelve loads are issued before the first is used
-        float x0[6], x1[6];
+    {
+        // thread = (rotation pair e, half of the query rows); all loads of a thread are issued before the first use
+        constexpr int HP = HD / 2, NH = AT_THREADS / HP;      // 64 pairs x 2 halves (hd 128) or 32 x 4 (hd 64)
+        constexpr int QPT = (HS_MAX_GT + NH - 1) / NH;        // query rows per thread
+        const int e = tid % HP, part = tid / HP;
+        float x0[QPT], x1[QPT];
 #pragma unroll
-        for (int u = 0; u < 6; ++u) {
-            const int idx = base + u * AT_THREADS + tid;
+        for (int u = 0; u < QPT; ++u) {
+            const int qi = part + u * NH;
             x0[u] = x1[u] = 0.f;
-            if (idx < GT * (HD / 2)) {
-                const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
-                const int gq = qi / T, i = qi - gq * T;
-                const float *src = a.zx + (size_t)(rowbase + i) * a.in_ld + a.q_off + (kh * G + gq) * HD;
-                x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HD / 2);
+            if (qi < GT) {
+                const int gq = (int)((qi * tinv) >> 16);
+                const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
             }
         }
 #pragma unroll
-        for (int u = 0; u < 6; ++u) {
-            const int idx = base + u * AT_THREADS + tid;
-            if (idx < GT * (HD / 2)) {
-                const int qi = idx / (HD / 2), e = idx - qi * (HD / 2);
-                const int i = qi % T;
-                const float2 cs = rope_s[i * (HD / 2) + e];
-                q_s[qi * HD + e] = (x0[u] * cs.x - x1[u] * cs.y) * scale;
-                q_s[qi * HD + e + HD / 2] = (x1[u] * cs.x + x0[u] * cs.y) * scale;
+        for (int u = 0; u < QPT; ++u) {
+            const int qi = part + u * NH;
+            if (qi < GT) {
+                const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
+                __nv_bfloat16 h, l;
+                split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
+                Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
+                Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
             }
         }
     }
@@ -135,133 +180,157 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
             const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
             const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
             const int j = ncache + i;
-            K_s[j * HD + e] = k0; K_s[j * HD + e + HD / 2] = k1;
-            V_s[j * HD + e] = v0; V_s[j * HD + e + HD / 2] = v1;
+            K_s[j * KSTR + e] = k0; K_s[j * KSTR + e + HD / 2] = k1;
+            V_s[j * KSTR + e] = v0; V_s[j * KSTR + e + HD / 2] = v1;
             Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
             Vb[(size_t)(len + i) * HD + e] = v0; Vb[(size_t)(len + i) * HD + e + HD / 2] = v1;
         }
         nkeys += T;
     }
-    bool landed = true;
-    if (ncache > 0) landed = mbar_wait(bar, 0);
-    if (!__syncthreads_and(landed)) {             // a copy never landed: report it, contribute nothing, keep the barriers
-        if (tid == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
-        nkeys = 0;
+    const int nkp = (nkeys + 15) & ~15;            // keys rounded to the MMA k step
+    // V rows of the padding keys must be finite: their probabilities are zero, and 0 * NaN is not
+    for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += AT_THREADS) {
+        const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4 *>(V_s + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
     }
+    cp_async_wait_all();
+    __syncthreads();
 
-    // ---- scores: lane = key (tiles of 32), warp w takes query rows w, w + 4, ...
-    for (int j0 = 0; j0 < nkeys; j0 += 32) {
-        const int j = j0 + lane;
-        const bool kvalid = j < nkeys;
-        const uint4 *krow = reinterpret_cast<const uint4 *>(K_s + (size_t)min(j, nkeys - 1) * HD);
-        for (int qb = warp; qb < GT; qb += AT_WARPS * 4) {
-            // up to four query rows per pass: qb, qb + 4, qb + 8, qb + 12
-            float d[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-            for (int c = 0; c < NC; ++c) {
-                const int cc = (c + lane) & (NC - 1);          // rotated chunk order: conflict-free key reads
-                const uint4 w = krow[cc];
-                const float k0 = bf_lo(w.x), k1 = bf_hi(w.x), k2 = bf_lo(w.y), k3 = bf_hi(w.y);
-                const float k4 = bf_lo(w.z), k5 = bf_hi(w.z), k6 = bf_lo(w.w), k7 = bf_hi(w.w);
+    // ---- scores S = Q K^T on the tensor cores: a warp takes 32 keys at a time for all query rows
+    const int g8 = lane >> 2, t4 = lane & 3;
+    for (int grp = warp; grp * 32 < nkp; grp += AT_WARPS) {
+        const int kb = grp * 32;
+        float S[MT][4][4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int qi = qb + u * AT_WARPS;
-                    if (qi < GT) {
-                        const float4 qa = *reinterpret_cast<const float4 *>(q_s + qi * HD + cc * 8);
-                        const float4 qc = *reinterpret_cast<const float4 *>(q_s + qi * HD + cc * 8 + 4);
-                        d[u] = fmaf(k0, qa.x, fmaf(k1, qa.y, fmaf(k2, qa.z, fmaf(k3, qa.w, d[u]))));
-                        d[u] = fmaf(k4, qc.x, fmaf(k5, qc.y, fmaf(k6, qc.z, fmaf(k7, qc.w, d[u]))));
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) { S[mt][nt][0] = S[mt][nt][1] = S[mt][nt][2] = S[mt][nt][3] = 0.f; }
+#pragma unroll 2
+        for (int ks = 0; ks < HD / 16; ++ks) {
+            uint32_t bk[2][4];
+#pragma unroll
+            for (int p = 0; p < 2; ++p)
+                ldsm_x4(bk[p], K_s + (size_t)(kb + p * 16 + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                uint32_t ah[4], al[4];
+                const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
+                ldsm_x4(ah, Qh_s + qo);
+                ldsm_x4(al, Ql_s + qo);
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], ah, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], al, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+            }
+        }
+        // raw scores to shared memory; keys beyond the chunk and, among the new rows, later positions are masked
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int row = mt * 16 + g8 + (e >> 1) * 8, key = kb + nt * 8 + 2 * t4 + (e & 1);
+                    if (row < GT && key < nkp) {
+                        const bool masked = key >= nkeys || (last && key >= ncache && (key - ncache) > (row - (int)((row * tinv) >> 16) * T));
+                        s_s[row * SSTR + key] = masked ? -INFINITY : S[mt][nt][e];
                     }
                 }
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int qi = qb + u * AT_WARPS;
-                if (qi < GT && kvalid) {
-                    const int i = qi % T;
-                    const bool masked = last && j >= ncache && (j - ncache) > i;     // causal among the new rows
-                    p_s[qi * PST + j] = masked ? -INFINITY : d[u];
-                }
-            }
-        }
     }
     __syncthreads();
-    // ---- softmax statistics of the chunk: one warp per query row
-    for (int qi = warp; qi < GT; qi += AT_WARPS) {
+    // ---- softmax of the chunk: one warp per query row; probabilities as bf16 head + remainder
+    for (int q0 = 0; q0 < GT; q0 += AT_THREADS / 8) {        // eight lanes per query row, sixteen rows per pass
+        const int qi = q0 + (tid >> 3), sub = tid & 7;
+        const bool rv = qi < GT;
         float mx = -INFINITY;
-        for (int j = lane; j < nkeys; j += 32) mx = fmaxf(mx, p_s[qi * PST + j]);
-        mx = warp_max(mx);
+        if (rv) for (int j = sub; j < nkp; j += 8) mx = fmaxf(mx, s_s[qi * SSTR + j]);
+#pragma unroll
+        for (int o = 4; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float sum = 0.f;
-        for (int j = lane; j < nkeys; j += 32) {
-            const float p = expf(p_s[qi * PST + j] - mx);        // expf(-inf) = 0 for masked keys
-            p_s[qi * PST + j] = p;
-            sum += p;
-        }
-        sum = warp_sum(sum);
-        if (lane == 0) { ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = sum; }
+        if (rv)
+            for (int j = sub; j < nkp; j += 8) {
+                const float p = expf(s_s[qi * SSTR + j] - mx);   // expf(-inf) = 0 for masked keys
+                __nv_bfloat16 h, l;
+                split_bf16(p, h, l);
+                Ph_s[qi * PSTR + j] = h; Pl_s[qi * PSTR + j] = l;
+                sum += p;
+            }
+#pragma unroll
+        for (int o = 4; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (rv && sub == 0) { ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = sum; }
     }
     __syncthreads();
-    // ---- acc = P V : thread = output dimension
-    float acc[GTB];
+    // ---- acc = P V on the tensor cores: a warp takes a quarter of the head dimension over all keys
+    constexpr int DW = HD / AT_WARPS, NTW = DW / 8;
+    float O[MT][NTW][4];
 #pragma unroll
-    for (int qi = 0; qi < GTB; ++qi) acc[qi] = 0.f;
-    if (tid < HD) {
-        for (int j = 0; j < nkeys; ++j) {
-            const float v = __bfloat162float(V_s[(size_t)j * HD + tid]);
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc[qi] = fmaf(p_s[qi * PST + j], v, acc[qi]);
+        for (int nt = 0; nt < NTW; ++nt) { O[mt][nt][0] = O[mt][nt][1] = O[mt][nt][2] = O[mt][nt][3] = 0.f; }
+    for (int kk = 0; kk < nkp / 16; ++kk) {
+        uint32_t bv[NTW / 2][4];
+#pragma unroll
+        for (int p = 0; p < NTW / 2; ++p)
+            ldsm_x4_t(bv[p], V_s + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + warp * DW + p * 16 + (lane >> 4) * 8);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            uint32_t ah[4], al[4];
+            const size_t po = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PSTR + kk * 16 + (lane >> 4) * 8;
+            ldsm_x4(ah, Ph_s + po);
+            ldsm_x4(al, Pl_s + po);
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], ah, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], al, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
         }
     }
+    // ---- this CTA's partial into its own shared memory (the query tiles are no longer needed)
+    float *acc_s = reinterpret_cast<float *>(Qh_s);          // [GT][HD] fp32
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int row = mt * 16 + g8 + hh * 8, d = warp * DW + nt * 8 + 2 * t4;
+                if (row < GT) *reinterpret_cast<float2 *>(acc_s + row * HD + d) = make_float2(O[mt][nt][2 * hh], O[mt][nt][2 * hh + 1]);
+            }
     float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
-    // ---- combine the chunks of this cluster through distributed shared memory: every CTA leaves its partial
-    //      (m, l, acc) in its own shared memory, rank r then sums output dims [r * DS, (r + 1) * DS) over all ranks
+    // ---- combine the chunks of this cluster through distributed shared memory: rank r sums output dims
+    //      [r * DS, (r + 1) * DS) over all ranks
     constexpr int DS = HD / AT_CL;
-    float *acc_s = q_s;                                      // [GT][HD]; the queries are no longer needed
-    if (tid < HD) {
-#pragma unroll
-        for (int qi = 0; qi < GTB; ++qi) if (qi < GT) acc_s[qi * HD + tid] = acc[qi];
-    }
     cluster.sync();
-    float *mlr_s = p_s;                                      // [AT_CL][GT][2] copies of every rank's (m, l)
-    float *wr_s = mlr_s + AT_CL * HS_MAX_GT * 2;             // [AT_CL][GT] merge weights
-    float *Md_s = wr_s + AT_CL * HS_MAX_GT;                  // [GT][2] merged (M, den)
-    for (int idx = tid; idx < AT_CL * GT * 2; idx += AT_THREADS) {
-        const int r = idx / (GT * 2), rem = idx - r * (GT * 2);
-        mlr_s[idx] = cluster.map_shared_rank(ml_s, r)[rem];
-    }
-    __syncthreads();
-    if (tid < GT) {
-        float M = -INFINITY;
-#pragma unroll
-        for (int r = 0; r < AT_CL; ++r) M = fmaxf(M, mlr_s[(r * GT + tid) * 2]);
-        float den = 0.f;
-#pragma unroll
-        for (int r = 0; r < AT_CL; ++r) {
-            const float mr = mlr_s[(r * GT + tid) * 2];
-            const float w = mr == -INFINITY ? 0.f : expf(mr - M);
-            wr_s[r * GT + tid] = w;
-            den = fmaf(w, mlr_s[(r * GT + tid) * 2 + 1], den);
-        }
-        Md_s[2 * tid] = M; Md_s[2 * tid + 1] = den;
-    }
-    __syncthreads();
     const int nclus = (nsplit + AT_CL - 1) / AT_CL;
     const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
+    float *Md_s = red_s;                                     // [GT][2] merged (M, den), for the cluster partial
     for (int idx = tid; idx < GT * DS; idx += AT_THREADS) {
-        const int qi = idx / DS, d = crank * DS + (idx - qi * DS);
+        const int qi = idx / DS, dd = idx - qi * DS, d = crank * DS + dd;
+        float2 mlr[AT_CL];
         float v[AT_CL];
 #pragma unroll
-        for (int r = 0; r < AT_CL; ++r) v[r] = cluster.map_shared_rank(acc_s, r)[qi * HD + d];
-        float sum = 0.f;
+        for (int r = 0; r < AT_CL; ++r) {                    // all remote reads are independent: one round trip
+            mlr[r] = *reinterpret_cast<const float2 *>(cluster.map_shared_rank(ml_s, r) + 2 * qi);
+            v[r] = cluster.map_shared_rank(acc_s, r)[qi * HD + d];
+        }
+        float M = -INFINITY;
 #pragma unroll
-        for (int r = 0; r < AT_CL; ++r) sum = fmaf(wr_s[r * GT + qi], v[r], sum);
+        for (int r = 0; r < AT_CL; ++r) M = fmaxf(M, mlr[r].x);
+        float den = 0.f, sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < AT_CL; ++r) {
+            const float w = mlr[r].x == -INFINITY ? 0.f : expf(mlr[r].x - M);
+            den = fmaf(w, mlr[r].y, den);
+            sum = fmaf(w, v[r], sum);
+        }
         if (nclus == 1) {
             const int gq = qi / T, i = qi - gq * T;
-            o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d] = sum / Md_s[2 * qi + 1];
+            o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d] = sum / den;
         } else {
             a.part_acc[(pbase + cl) * HS_MAX_GT * HD + qi * HD + d] = sum;
+            if (crank == 0 && dd == 0) { Md_s[2 * qi] = M; Md_s[2 * qi + 1] = den; }
         }
     }
+    if (nclus > 1) __syncthreads();
     if (nclus > 1 && crank == 0 && tid < 2 * GT) a.part_ml[(pbase + cl) * HS_MAX_GT * 2 + tid] = Md_s[tid];
     cluster.sync();                                          // peers may still be reading this CTA's shared memory
     if (nclus == 1) return;
@@ -273,34 +342,35 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     if (ticket_s != nclus * AT_CL - 1) return;
     __threadfence();
     if (tid == 0) a.counters[b * a.kvh + kh] = 0;          // ready for the next launch
-    const int nmerge = nclus;
+    constexpr int GTB = MT * 16;
     const float *pa0 = a.part_acc + pbase * HS_MAX_GT * HD;
     const float *pm0 = a.part_ml + pbase * HS_MAX_GT * 2;
-    float *w_s = p_s;                                        // [GT][PST]: merge weights of PST chunks per pass
+    float *w_s = s_s;                                        // [GT][SSTR]: merge weights of SSTR clusters per pass
     for (int qi = warp; qi < GT; qi += AT_WARPS) {
         float M = -INFINITY;
-        for (int c = lane; c < nmerge; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+        for (int c = lane; c < nclus; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
         M = warp_max(M);
         float den = 0.f;
-        for (int c = lane; c < nmerge; c += 32) {
+        for (int c = lane; c < nclus; c += 32) {
             const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
             den = fmaf(expf(mlv.x - M), mlv.y, den);
         }
         den = warp_sum(den);
         if (lane == 0) { ml_s[2 * qi] = M; ml_s[2 * qi + 1] = den; }
     }
+    float acc[GTB];
 #pragma unroll
     for (int qi = 0; qi < GTB; ++qi) acc[qi] = 0.f;
-    for (int cb = 0; cb < nmerge; cb += PST) {               // chunks in passes of PST
-        const int nc = min(PST, nmerge - cb);
+    for (int cb = 0; cb < nclus; cb += SSTR) {               // clusters in passes of SSTR
+        const int nc = min(SSTR, nclus - cb);
         __syncthreads();                                     // ml_s ready / previous pass done with w_s
         for (int idx = tid; idx < GT * nc; idx += AT_THREADS) {
             const int qi = idx / nc, c = idx - qi * nc;
-            w_s[qi * PST + c] = expf(__ldcg(pm0 + ((size_t)(cb + c) * HS_MAX_GT + qi) * 2) - ml_s[2 * qi]);
+            w_s[qi * SSTR + c] = expf(__ldcg(pm0 + ((size_t)(cb + c) * HS_MAX_GT + qi) * 2) - ml_s[2 * qi]);
         }
         __syncthreads();
         if (tid < HD) {
-            constexpr int MB = 64 / GTB < 1 ? 1 : 64 / GTB;       // chunks whose partials are fetched together
+            constexpr int MB = 64 / GTB < 1 ? 1 : 64 / GTB;       // clusters whose partials are fetched together
             for (int c = 0; c < nc; c += MB) {
                 float v[MB][GTB];
 #pragma unroll
@@ -312,7 +382,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
                 for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
                     for (int qi = 0; qi < GTB; ++qi)
-                        if (c + mb < nc && qi < GT) acc[qi] = fmaf(w_s[qi * PST + c + mb], v[mb][qi], acc[qi]);
+                        if (c + mb < nc && qi < GT) acc[qi] = fmaf(w_s[qi * SSTR + c + mb], v[mb][qi], acc[qi]);
             }
         }
     }
@@ -326,37 +396,38 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     }
 }
 
-template <int HD, int GTB>
+template <int HD, int MT>
 cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
     dim3 grid((a.nch + AT_CL - 1) / AT_CL * AT_CL, a.kvh, a.nb);
-    return launch_pdl_cluster(attn_kernel<HD, GTB>, grid, dim3(AT_THREADS), AttnSmem<HD>::total(a.chunk), s, AT_CL, a);
+    const size_t smem = attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
+    return launch_pdl_cluster(attn_kernel<HD, MT>, grid, dim3(AT_THREADS), smem, s, AT_CL, a);
 }
 
-template <int HD, int GTB>
+template <int HD, int MT>
 cudaError_t configure_t() {
-    cudaError_t e = cudaFuncSetAttribute(attn_kernel<HD, GTB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnSmem<HD>::total(128));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<HD, GTB>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+    cudaError_t e = cudaFuncSetAttribute(attn_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_layout(HD, 128, MT * 16).total);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<HD, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     return e;
 }
 
 }  // namespace
 
 cudaError_t configure_attn() {
-    cudaError_t e = configure_t<128, 16>();
-    if (e == cudaSuccess) e = configure_t<128, 32>();
-    if (e == cudaSuccess) e = configure_t<128, 48>();
-    if (e == cudaSuccess) e = configure_t<64, 16>();
-    if (e == cudaSuccess) e = configure_t<64, 32>();
-    if (e == cudaSuccess) e = configure_t<64, 48>();
+    cudaError_t e = configure_t<128, 1>();
+    if (e == cudaSuccess) e = configure_t<128, 2>();
+    if (e == cudaSuccess) e = configure_t<128, 3>();
+    if (e == cudaSuccess) e = configure_t<64, 1>();
+    if (e == cudaSuccess) e = configure_t<64, 2>();
+    if (e == cudaSuccess) e = configure_t<64, 3>();
     return e;
 }
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     const int GT = (a.qh / a.kvh) * a.T;
     if (GT > HS_MAX_GT || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128)) return cudaErrorInvalidValue;
-    const int gtb = GT <= 16 ? 16 : GT <= 32 ? 32 : 48;
-#define CASE(hd_, g_) if (a.hd == hd_ && gtb == g_) return launch_t<hd_, g_>(a, s)
-    CASE(128, 16); CASE(128, 32); CASE(128, 48); CASE(64, 16); CASE(64, 32); CASE(64, 48);
+    const int mt = (GT + 15) / 16;
+#define CASE(hd_, m_) if (a.hd == hd_ && mt == m_) return launch_t<hd_, m_>(a, s)
+    CASE(128, 1); CASE(128, 2); CASE(128, 3); CASE(64, 1); CASE(64, 2); CASE(64, 3);
 #undef CASE
     return cudaErrorInvalidValue;
 }
