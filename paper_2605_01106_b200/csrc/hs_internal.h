@@ -88,6 +88,7 @@ struct hs_model {
 // Every kernel of a step is launched with programmatic stream serialization: it may start while its
 // predecessor still runs and synchronises with griddepcontrol.wait (see hs_device.cuh).
 extern bool g_hs_pdl;
+extern bool g_hs_gemm_mma;     // projections with 2..16 activation rows on the tensor cores (default) or the CUDA cores
 // cluster_x > 1 launches thread-block clusters of that many CTAs along x (grid.x must be a multiple).
 template <class... KArgs, class... Args>
 inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

