@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libhs.so")
-SOURCES = ["hs_api.cu", "kernels_gemv.cu", "kernels_mixer.cu", "kernels_attn.cu", "kernels_misc.cu"]
+SOURCES = ["hs_api.cu", "kernels_gemv.cu", "kernels_gemm_tc.cu", "kernels_mixer.cu", "kernels_attn.cu", "kernels_misc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

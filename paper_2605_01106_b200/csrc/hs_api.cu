@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <algorithm>
 
 namespace {
 
@@ -120,7 +121,7 @@ Derived derive(const hs_config &c) {
 // layout of the work buffer; base may be null to only measure
 struct WorkLayout {
     int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters;
-    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, am_part, total;
+    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, am_part, xb, total;
 };
 
 WorkLayout work_layout(const hs_config &c, const Derived &v) {
@@ -141,6 +142,10 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.att_acc = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * c.hd);
     w.att_ml = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * 2);
     w.am_part = take((int64_t)16 * v.R * HS_ARGMAX_CHUNKS);
+    {   // packed bf16 activation operand of the many-row projection kernel: [2][rows][widest reduction]
+        const int64_t kmax = std::max<int64_t>(std::max<int64_t>(c.d, c.ff), (int64_t)v.gw + c.qh * c.hd);
+        w.xb = take(v.R > 16 ? (int64_t)2 * 2 * gemm_tc_rows(v.R) * kmax : 0);
+    }
     w.total = off;
     return w;
 }
@@ -216,6 +221,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         ga.early_trigger = 0;
         ga.pf_ptr = ly.type == HS_LAYER_ATT ? ly.W_o : ly.W_out;
         ga.pf_bytes = 2 * (int64_t)d * (ly.type == HS_LAYER_ATT ? c.qh * c.hd : m->gw);
+        ga.xb = m->xb; ga.xb_rows = m->xb_rows;
         PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, st_w, s, &m->launches, nullptr), "in_proj");
         // (2) recurrent mixer
         if (ly.type != HS_LAYER_ATT) {
@@ -281,6 +287,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             go.W0 = ly.W_o; go.ldw0 = c.qh * c.hd; go.K0 = c.qh * c.hd; go.x0 = m->obuf; go.ldx0 = c.qh * c.hd;
         }
         go.early_trigger = 1; go.pf_ptr = ly.W_gu; go.pf_bytes = 2 * (int64_t)2 * c.ff * d;
+        go.xb = m->xb; go.xb_rows = m->xb_rows;
         PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, st_w, s, &m->launches, &hparts), "out_proj");
         cur ^= 1;
         // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
@@ -289,6 +296,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         gu.norm_w = ly.norm2; gu.eps = c.eps;
         gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
         gu.early_trigger = 1; gu.pf_ptr = ly.W_down; gu.pf_bytes = 2 * (int64_t)d * c.ff;
+        gu.xb = m->xb; gu.xb_rows = m->xb_rows;
         PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, st_w, s, &m->launches, nullptr), "gate_up");
         GemvArgs gdn{};
         gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff; gdn.xparts = 1;
@@ -301,6 +309,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             if (nl < c.L) { gdn.pf_ptr = m->layers[nl].W_in; gdn.pf_bytes = 2 * (int64_t)d * (draft ? m->layers[nl].in_rows_draft : m->layers[nl].in_rows_full); }
             else { gdn.pf_ptr = m->lm_head; gdn.pf_bytes = 2 * (int64_t)c.V * d; }
         }
+        gdn.xb = m->xb; gdn.xb_rows = m->xb_rows;
         PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, st_w, s, &m->launches, &hparts), "down");
         cur ^= 1;
     }
@@ -310,6 +319,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     lm.norm_w = m->final_norm; lm.eps = c.eps;
     lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
     lm.early_trigger = 1;
+    lm.xb = m->xb; lm.xb_rows = m->xb_rows;
     PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
     if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, m->am_part, m->ctrl.am_counters, s), "argmax");
     else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, m->am_part, m->ctrl.am_counters, s), "argmax");
@@ -430,7 +440,7 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     m->rope = (float2 *)(w + wl.rope);
     m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
     m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits);
-    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part;
+    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part; m->xb = v.R > 16 ? (__nv_bfloat16 *)(w + wl.xb) : nullptr; m->xb_rows = gemm_tc_rows(v.R);
     // conv buffer: committed windows | verify history | draft ping-pong
     float *cv = (float *)bufs->conv;
     const size_t win = (size_t)v.n_rl * v.B * 3 * v.convd;
@@ -441,6 +451,7 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     *out = m;
     CK(configure_gemv(), "configure gemv");
     CK(configure_attn(), "configure attention");
+    if (configure_gemm_tc() != cudaSuccess) { g_hs_gemm_tc = false; cudaGetLastError(); }   // falls back to several 16-row launches
     // RoPE table (rotate-half pairing: pair (e, e + hd/2) turns by pos * theta^(-2e/hd)), computed in double
     std::vector<float2> tab((size_t)c.kv_capacity * (c.hd / 2));
     for (int e = 0; e < c.hd / 2; ++e) {

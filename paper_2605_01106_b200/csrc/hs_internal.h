@@ -63,6 +63,7 @@ struct hs_model {
     float *hbuf[2];            // residual stream, ping-pong; each [HS_H_PARTS][B*Tm][d] partial sums
     float *zx, *gbuf, *obuf, *abuf, *logits;
     float *att_acc, *att_ml;
+    __nv_bfloat16 *xb; int64_t xb_rows;   // packed activation operand of the many-row projection kernel
     void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
     // conv buffers
     float *cw, *hist, *dcw;
@@ -129,12 +130,18 @@ struct GemvArgs {
     int nrows;                // activation rows (batch * T), at most 16 per launch
     int epi;
     const void *pf_ptr; int64_t pf_bytes;   // optional: weights of the next projection, prefetched into L2
+    __nv_bfloat16 *xb; int64_t xb_rows;     // scratch for the packed activation operand of the many-row kernel: [2][xb_rows][K0+K1]
     int early_trigger;        // 1: let the next kernel start before this one has waited for its predecessor
                               // (allowed only if that kernel touches nothing but weights before its own wait)
 };
 // *oparts receives the number of parts written to `out` (1 unless EPI_RESID split the reduction).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
 cudaError_t configure_gemv();   // one-time kernel attributes; call outside stream capture
+// many activation rows (> 16): tcgen05 tensor-core contraction (kernels_gemm_tc.cu)
+extern bool g_hs_gemm_tc;
+cudaError_t configure_gemm_tc();
+int gemm_tc_rows(int nrows);
+cudaError_t launch_gemm_tc(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
 cudaError_t configure_attn();
 
 cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,

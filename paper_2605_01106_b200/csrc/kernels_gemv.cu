@@ -527,6 +527,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         return cudaSuccess;
     };
     const bool mma = g_hs_gemm_mma && a.nrows >= 2;
+    if (a.nrows > GV_MAXROWS && g_hs_gemm_tc && a.xb) return launch_gemm_tc(a, status, s, launches, oparts);   // a dense contraction: tcgen05
     if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     if (!mma && a.nrows > 4) {
         const int K = a.K0 > a.K1 ? a.K0 : a.K1;
