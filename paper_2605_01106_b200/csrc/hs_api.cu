@@ -218,7 +218,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
         // the mixer that follows reads its recurrent state before its own wait: keep it from starting
         // until this kernel has waited, i.e. until everything older is complete
-        ga.early_trigger = 0;
+        ga.early_trigger = 1;
         ga.pf_ptr = ly.type == HS_LAYER_ATT ? ly.W_o : ly.W_out;
         ga.pf_bytes = 2 * (int64_t)d * (ly.type == HS_LAYER_ATT ? c.qh * c.hd : m->gw);
         ga.xb = m->xb; ga.xb_rows = m->xb_rows;

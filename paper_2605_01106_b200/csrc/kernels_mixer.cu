@@ -30,21 +30,19 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
     const int rowbase = lb * T;
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
-    // ---- issue the state loads first: they do not depend on anything computed here
+    // ---- before the wait only parameters are read; the recurrent state (written by an earlier kernel of
+    //      the step or of the previous round) is merely pulled towards L2 and loaded after the wait, together
+    //      with the in-projection's outputs, so that this kernel may start as early as its predecessor allows
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
                         (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) +
                         ((size_t)h * a.P + p0 + warp * RPW) * N;
-    float s[RPW][EPL];
 #pragma unroll
     for (int r = 0; r < RPW; ++r)
 #pragma unroll
-        for (int v = 0; v < NVEC; ++v) {
-            const float *src = sin_ + r * N + v * (32 * VW) + lane * VW;
-            if (VW == 4) { float4 t = *reinterpret_cast<const float4 *>(src); s[r][v * 4] = t.x; s[r][v * 4 + 1] = t.y; s[r][v * 4 + 2] = t.z; s[r][v * 4 + 3] = t.w; }
-            else { float2 t = *reinterpret_cast<const float2 *>(src); s[r][0] = t.x; s[r][1] = t.y; }
-        }
-
-    // ---- still before the wait: everything of the conv that is a parameter or older state.
+        for (int v = 0; v < NVEC; ++v)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(sin_ + r * N + v * (32 * VW) + lane * VW));
+    float s[RPW][EPL];
+    // ---- still before the wait: the conv parameters.
     // A thread owns the channels tid, tid + 128, ... of this block's set: its x strip, all of B and C.
     constexpr int NCH = SSM_PR + 2 * N;
     constexpr int CPT = (NCH + SSM_THREADS - 1) / SSM_THREADS;
@@ -59,16 +57,29 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
             const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
             tap[q] = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
             bias[q] = a.conv_b[gc];
+        }
+    }
+    const float Aexp = expf(a.A_log[h]), dtb = a.dt_bias[h], Dh = a.D[h];
+    pdl_wait();
+
+    // ---- after the wait: the state rows and the conv window (L2 hits), in flight with the sweep below
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v) {
+            const float *src = sin_ + r * N + v * (32 * VW) + lane * VW;
+            if (VW == 4) { float4 t = __ldcg(reinterpret_cast<const float4 *>(src)); s[r][v * 4] = t.x; s[r][v * 4 + 1] = t.y; s[r][v * 4 + 2] = t.z; s[r][v * 4 + 3] = t.w; }
+            else { float2 t = __ldcg(reinterpret_cast<const float2 *>(src)); s[r][0] = t.x; s[r][1] = t.y; }
+        }
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
             const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
             w0[q] = __ldcg(win); w1[q] = __ldcg(win + a.convd); w2[q] = __ldcg(win + 2 * a.convd);
         }
     }
-    const float Aexp = expf(a.A_log[h]), dtb = a.dt_bias[h], Dh = a.D[h];
-    // The state and the conv window were written at least two kernels ago and the in-projection before
-    // this kernel only lets it start after its own wait, so everything older than that projection is
-    // complete: the loads above are safe.  Everything below reads the in-projection.
-    pdl_wait();
-
     // ---- raw conv inputs, gate inputs and dt of all T positions: one sweep of independent loads
     for (int idx = threadIdx.x; idx < T * NCH; idx += SSM_THREADS) {
         const int i = idx / NCH, c = idx - i * NCH;
@@ -172,12 +183,17 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
                         (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) + (size_t)h * dv * DK;
     float s[RPW][2];
     const bool rows_ok = warp * RPW < dv;
+    // before the wait the state is only pulled towards L2 (it was written by an earlier kernel); it is loaded
+    // after the wait, so this kernel may start as early as its predecessor allows
+    if (rows_ok)
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) asm volatile("prefetch.global.L2 [%0];" :: "l"(sin_ + (warp * RPW + r) * DK + 2 * lane));
+    pdl_wait();
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
-        float2 t = rows_ok ? *reinterpret_cast<const float2 *>(sin_ + (warp * RPW + r) * DK + 2 * lane) : make_float2(0.f, 0.f);
+        float2 t = rows_ok ? __ldcg(reinterpret_cast<const float2 *>(sin_ + (warp * RPW + r) * DK + 2 * lane)) : make_float2(0.f, 0.f);
         s[r][0] = t.x; s[r][1] = t.y;
     }
-    pdl_wait();
     // conv + SiLU on this head's q, k, v channels
     for (int c = threadIdx.x; c < 2 * DK + dv; c += GDN_THREADS) {
         const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
