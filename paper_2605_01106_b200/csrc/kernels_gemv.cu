@@ -102,9 +102,14 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
         const int buf = t % D;
         if (lane == 0) mbar_expect_tx(&mybar[buf], (uint32_t)rows_in * cw * 2);
         __syncwarp();
-        if (lane < rows_in)
+        if (ld == kc && cw == kc) {
+            // whole rows of an unsplit matrix: the tile is one contiguous piece of memory, one large request
+            if (lane == 0)
+                bulk_g2s(mybuf + (size_t)buf * WR * kc, W + (size_t)row0 * ld, (uint32_t)rows_in * cw * 2, &mybar[buf]);
+        } else if (lane < rows_in) {
             bulk_g2s(mybuf + ((size_t)buf * WR + lane) * kc, W + (size_t)(row0 + lane) * ld + k0 + ch * kc,
                      (uint32_t)cw * 2, &mybar[buf]);
+        }
     };
 
     // ---- prologue, independent of the previous kernel: start the weight stream
@@ -561,7 +566,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (g.NR > units) g.NR = units;
     const int nrow_max = ceil_div(units, g.NR) * g.unit;
     // tile: 4 weight rows per warp when that already gives every warp a tile, else 8
-    const int WR = mma ? 8 : (nrow_max <= 4 * GV_WARPS ? 4 : 8);
+    // (wide K ranges: 4-row tiles of whole rows - requests of several KB stream best)
+    const int WR = mma ? 8 : ((nrow_max <= 4 * GV_WARPS || g.krmax > 1280) ? 4 : 8);
     const int NG = a.nrows <= 8 ? 1 : 2;                       // tensor-core kernel: groups of 8 activation rows
     const int tpad = mma ? 8 : 0;                              // its tile rows are padded by 16 bytes
     // chunk of at most 1280 columns, as even as possible; narrower if the ring would not fit
@@ -571,7 +577,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     g.off_ring = g.off_nw + (a.norm_w ? g.krmax * 4 : 0);
     const int ring_warps = ceil_div(nrow_max, WR) < GV_WARPS ? ceil_div(nrow_max, WR) : GV_WARPS;
     size_t tile = 0;
-    for (int nch = ceil_div(g.krmax, 1280);; ++nch) {
+    for (int nch = mma ? ceil_div(g.krmax, 1280) : 1;; ++nch) {
         g.kc = ceil_div(ceil_div(g.krmax, nch), 256) * 256;
         tile = (size_t)WR * (g.kc + tpad) * 2;
         if (g.off_ring + tile * ring_warps <= GV_SMEM_MAX || g.kc == 256) break;
@@ -580,7 +586,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (!mma && a.nrows > 4 && nchunks > 1) return rows_launch(4);   // passes need every chunk of a row group resident
     const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * nchunks;
     int D = 1;
-    while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= GV_SMEM_PAIR) ++D;
+    const size_t budget = g.off_ring + tile * GV_WARPS > GV_SMEM_PAIR ? GV_SMEM_MAX : GV_SMEM_PAIR;   // no room for a neighbour anyway: go deep
+    while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= budget) ++D;
     g.D = D;
     const size_t smem = g.off_ring + tile * ring_warps * D;
     if (smem > GV_SMEM_MAX) return a.nrows > 1 ? rows_launch((a.nrows + 1) / 2) : cudaErrorInvalidValue;
