@@ -19,7 +19,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy", "hs_argmax_static"]
+           "hs_set_attn_geometry", "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
 class HsError(RuntimeError):
@@ -71,6 +71,7 @@ def load_library(path: str | None = None):
     L.hs_get_round.argtypes = [vp, vp, vp, vp]
     L.hs_launch_count.restype = i64
     L.hs_launch_count.argtypes = [vp]
+    L.hs_set_attn_geometry.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     L.hs_profile.argtypes = [vp, ctypes.c_int]
     L.hs_profile_read.argtypes = [vp, vp, vp, vp]
     L.hs_device_status.argtypes = [vp]
@@ -279,6 +280,10 @@ class Engine:
         return c, g, m
 
     PROF_NAMES = ("gemv", "mixer", "attention", "argmax", "embed", "accept")
+
+    def set_attn_geometry(self, chunk, tiles=1):
+        """Fix the KV split of verify-mode attention (chunk keys x tiles per CTA); chunk = 0: automatic."""
+        self._ck(lib().hs_set_attn_geometry(self.h, int(chunk), int(tiles)))
 
     def profile(self, enable):
         self._ck(lib().hs_profile(self.h, int(enable)))

@@ -183,19 +183,33 @@ double gemv_bytes(const GemvArgs &a) {
 //   draft = false: full model M_H (verify);  draft = true: draft model M_S, one position,
 //   reading candidate column `col` and, for step > 0, the scratch state of the previous step.
 // ------------------------------------------------------------------------------------------------
-// keys per attention CTA for this launch: small enough to spread a short context over the eight CTAs of one
-// cluster (which combine their partials in shared memory), never below the size the partial buffers were
-// laid out for
-int attn_chunk(const hs_model *m, int T, int b0, int nb) {
+// Attention geometry of this launch.  Keys per tile: small enough to spread a short context over the eight
+// CTAs of one cluster (which combine their partials in shared memory), never below the size the partial
+// buffers were laid out for.  Tiles per CTA: one, unless the launch would have far more CTAs than the GPU
+// runs at once (long caches at large batch) - then a CTA walks up to sixteen 64-key tiles, so that staging
+// the queries and combining the partials is paid once per 1024 keys.
+struct AttnGeom {
+    int chunk, tiles;
+    int code() const { return (chunk == 32 ? 0 : chunk == 64 ? 1 : 2) * 64 + tiles - 1; }   // < 256, part of the graph key
+};
+AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
+    if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles};
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
     const int want = maxlen + T <= 256 ? 32 : maxlen + T <= 512 ? 64 : 128;
-    return want > m->att_chunk ? want : m->att_chunk;
+    AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1};
+    const int64_t ctas64 = (int64_t)nb * m->c.kvh * ((maxlen + T + 63) / 64);
+    const int64_t fill = 148 * 8;             // CTAs that keep every SM busy for several rounds
+    if (g.chunk == 128 && ctas64 >= 4 * fill) {
+        g.chunk = 64;
+        g.tiles = ctas64 / fill >= 16 ? 16 : ctas64 / fill >= 8 ? 8 : ctas64 / fill >= 4 ? 4 : 2;
+    }
+    return g;
 }
 
 int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     const hs_config &c = m->c;
-    const int at_chunk = draft ? m->att_chunk : attn_chunk(m, T, b0, nb);
+    const AttnGeom at_geom = draft ? AttnGeom{m->att_chunk, 1} : attn_geom(m, T, b0, nb);
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
@@ -270,7 +284,8 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             aa.Kc = m->Kc + ly.al * per_layer; aa.Vc = m->Vc + ly.al * per_layer; aa.cap = c.kv_capacity;
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
-            aa.chunk = at_chunk; aa.nch = (c.kv_capacity + at_chunk - 1) / at_chunk; aa.T = T; aa.b0 = b0; aa.nb = nb;
+            aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles;
+            aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
             PROF(HS_PROF_ATTN, 0, launch_attn(aa, s), "attention");
             ++m->launches;
         }
@@ -408,7 +423,7 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     Derived v = derive(c);
     m->B = v.B; m->Tm = v.Tm; m->batch = 0; m->di = d_inner(c); m->convd = v.convd; m->gw = v.gw;
     m->n_rl = v.n_rl; m->n_al = v.n_al; m->state_elems = v.state_elems; m->in_rows_max = v.in_rows_max;
-    m->att_chunk = v.att_chunk; m->att_nch = v.att_nch;
+    m->att_chunk = v.att_chunk; m->att_nch = v.att_nch; m->att_force_chunk = m->att_force_tiles = 0;
     m->phase = 0; m->last_k = -1; m->last_rows = 0; m->launches = 0; m->prof = false;
     m->kv_upper.assign(v.B, 0);
     const char *wb = (const char *)bufs->weights;
@@ -536,7 +551,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
-    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_chunk(m, T, 0, nb) << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
+    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
     return HS_OK;
@@ -681,6 +696,15 @@ int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin
 }
 
 int64_t hs_launch_count(const hs_model *m) { return m ? m->launches : -1; }
+
+int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    if (chunk == 0) { m->att_force_chunk = m->att_force_tiles = 0; return HS_OK; }
+    if ((chunk != 32 && chunk != 64 && chunk != 128) || tiles < 1 || tiles > 64 || chunk * tiles < m->att_chunk)
+        return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk 32/64/128, tiles 1..64, chunk * tiles >= workspace chunk");
+    m->att_force_chunk = chunk; m->att_force_tiles = tiles;
+    return HS_OK;
+}
 
 int hs_profile(hs_model *m, int enable) {
     if (!m) return HS_ERR_INVALID_ARG;

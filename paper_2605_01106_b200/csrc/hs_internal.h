@@ -54,6 +54,7 @@ struct hs_model {
     int64_t state_elems;      // floats of one (layer, seq) recurrent state
     int in_rows_max;
     int att_chunk, att_nch;   // keys per split, max splits
+    int att_force_chunk, att_force_tiles;   // 0: automatic
     std::vector<HsLayer> layers;
     const __nv_bfloat16 *embed, *lm_head;
     const float *final_norm;
@@ -186,7 +187,7 @@ struct AttnArgs {
     const int32_t *kv_len;
     float *o;                           // [rows][qh*hd]
     float *part_acc, *part_ml; int32_t *counters; int32_t *status;
-    int chunk, nch;
+    int chunk, tiles, nch;              // keys per tile, tiles per CTA, CTAs (key ranges) that cover the cache capacity
     int T, b0, nb;
 };
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);

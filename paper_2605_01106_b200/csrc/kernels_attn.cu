@@ -1,11 +1,14 @@
 // Verify-mode attention: the T = k+1 new positions of a sequence attend over its KV cache plus the
 // new rows themselves (causal among the new ones), grouped-query heads, split over the cache length.
 //
-// grid = (chunks rounded up to clusters of 8, kv heads, sequences); one CTA = one chunk of CK cached
-// keys for the G*T query rows that share its KV head (G = q heads per KV head).
+// grid = (key ranges rounded up to clusters of 8, kv heads, sequences); one CTA = a range of `tiles`
+// tiles of CK cached keys each for the G*T query rows that share its KV head (G = q heads per KV head).
+// Long caches at large batch use several tiles per CTA: the queries are staged and the partial combined
+// once per range, and the tiles are folded into a running (max, sum, acc) - the online softmax.
 //  * Before the programmatic-dependent-launch wait the CTA reads kv_len (written at least two kernels
-//    earlier), starts the asynchronous copies of its K and V chunk into padded shared-memory rows and
-//    fetches the RoPE rows of the new positions.
+//    earlier), starts the asynchronous copies of its first K and V tile into padded shared-memory rows
+//    and fetches the RoPE rows of the new positions.  Later tiles are fetched while the previous one is
+//    still in use: K for tile t+1 as soon as the scores of tile t are out, V after P V of tile t.
 //  * After the wait it rotates and scales the queries; the CTA of the last chunk also rotates the T new
 //    K rows, rounds K and V to bf16 exactly as they are cached, appends them to the cache and keeps them
 //    in shared memory behind the cached keys, so nothing written by this launch is read back from
@@ -14,8 +17,8 @@
 //    V are bf16 in the cache and enter exactly; the fp32 queries and probabilities are split into a
 //    bf16 head and a bf16 remainder (two MMAs), which keeps the products exact to 2^-17 - the
 //    comparison with the CPU oracle allows 1e-3 on states fed by this output.
-//    Scores: a warp takes 32 keys at a time for all query rows; one softmax per chunk (the whole chunk is
-//    resident); P V: a warp takes a quarter of the head dimension over all keys.
+//    Scores: a warp takes 32 keys at a time for all query rows; one softmax per tile (the whole tile is
+//    resident); P V: a warp takes a quarter of the head dimension over all keys of the tile.
 //  * The up to eight chunks of a cluster leave (m, l, acc) in their own shared memory and combine them
 //    through distributed shared memory, rank r summing an eighth of the output dimensions.  Longer
 //    caches span several clusters: each publishes one partial and the CTA that arrives last (ticket
@@ -34,7 +37,7 @@ constexpr int AT_CL = 8;               // CTAs (chunks) per thread-block cluster
 
 struct AttnLayout {
     int kstr, keys, mrows, pstr, sstr;
-    size_t k_off, v_off, q_off, s_off, p_off, ml_off, rope_off, red_off, total;
+    size_t k_off, v_off, q_off, s_off, p_off, ml_off, corr_off, new_off, rope_off, red_off, total;
 };
 // shared-memory carve-up for head dim hd, chunk ck, gt query rows
 __host__ __device__ inline AttnLayout attn_layout(int hd, int ck, int gt) {
@@ -51,6 +54,8 @@ __host__ __device__ inline AttnLayout attn_layout(int hd, int ck, int gt) {
     L.s_off = o; o += (size_t)L.mrows * L.sstr * 4;           // raw scores fp32
     L.p_off = o; o += (size_t)2 * L.mrows * L.pstr * 2;       // probabilities: bf16 head | remainder
     L.ml_off = o; o += (size_t)HS_MAX_GT * 2 * 4;
+    L.corr_off = o; o += (size_t)HS_MAX_GT * 4;
+    L.new_off = o; o += (size_t)2 * HS_MAX_T * L.kstr * 2;    // the new K | V rows as they are cached
     L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
     L.red_off = o; o += (size_t)(AT_CL * HS_MAX_GT * 3 + HS_MAX_GT * 2) * 4;
     L.total = (o + 127) / 128 * 128;
@@ -62,6 +67,7 @@ __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
@@ -96,7 +102,10 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     float *s_s = reinterpret_cast<float *>(smraw + L.s_off);                         // [mrows][SSTR]
     __nv_bfloat16 *Ph_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.p_off);        // [mrows][PSTR]
     __nv_bfloat16 *Pl_s = Ph_s + (size_t)L.mrows * PSTR;
-    float *ml_s = reinterpret_cast<float *>(smraw + L.ml_off);                       // [GT][2]
+    float *ml_s = reinterpret_cast<float *>(smraw + L.ml_off);                       // [GT][2] running (max, sum)
+    float *corr_s = reinterpret_cast<float *>(smraw + L.corr_off);                   // [GT] rescale of acc for this tile
+    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.new_off);      // [T][KSTR] new K rows (last CTA)
+    __nv_bfloat16 *Vn_s = Kn_s + (size_t)HS_MAX_T * KSTR;
     float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);                 // [T][HD/2]
     float *red_s = reinterpret_cast<float *>(smraw + L.red_off);
     __shared__ int ticket_s;
@@ -106,28 +115,36 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     const uint32_t tinv = (65536u + T - 1) / T;      // x / T == (x * tinv) >> 16 for the small x used here
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
-    // ---- before the wait: kv_len, the cached chunk, the RoPE rows
+    // ---- before the wait: kv_len, the first cached tile, the RoPE rows
     const int len = __ldcg(a.kv_len + b);
-    const int nsplit = max(1, (len + CK - 1) / CK);
+    const int SPAN = CK * a.tiles;                // cached keys per CTA
+    const int nsplit = max(1, (len + SPAN - 1) / SPAN);
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank(), cl = split / AT_CL;
     if (cl * AT_CL >= nsplit) return;             // the whole cluster is beyond the cache: nobody reaches a barrier
-    // a CTA beyond the last chunk of a live cluster has no keys: it contributes (m, l) = (-inf, 0) and still
+    // a CTA beyond the last range of a live cluster has no keys: it contributes (m, l) = (-inf, 0) and still
     // takes its share of the cluster's reduction
     const bool last = split == nsplit - 1;
-    const int c0 = split * CK, ncache = max(0, min(len, c0 + CK) - c0);
+    const int c0 = split * SPAN, rc = max(0, min(len, c0 + SPAN) - c0);
+    const int ntile = last ? max(1, (rc + CK - 1) / CK) : (rc + CK - 1) / CK;
     if (len + T > a.cap) {                        // never write past the cache; the host reports the status word
         if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
         return;
     }
     __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
     __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    for (int idx = tid; idx < ncache * (HD / 8); idx += AT_THREADS) {
-        const int j = idx / (HD / 8), c = idx - j * (HD / 8);
-        cp_async16(K_s + (size_t)j * KSTR + 8 * c, Kb + (size_t)(c0 + j) * HD + 8 * c);
-        cp_async16(V_s + (size_t)j * KSTR + 8 * c, Vb + (size_t)(c0 + j) * HD + 8 * c);
-    }
-    cp_async_commit();
+    // asynchronous copy of the cached rows of tile t (one commit group per call, possibly empty)
+    auto fetch = [&](__nv_bfloat16 *dst, const __nv_bfloat16 *src, int t) {
+        const int n = t < ntile ? max(0, min(CK, rc - t * CK)) : 0;
+        const __nv_bfloat16 *from = src + (size_t)(c0 + t * CK) * HD;
+        for (int idx = tid; idx < n * (HD / 8); idx += AT_THREADS) {
+            const int j = idx / (HD / 8), c = idx - j * (HD / 8);
+            cp_async16(dst + (size_t)j * KSTR + 8 * c, from + (size_t)j * HD + 8 * c);
+        }
+        cp_async_commit();
+    };
+    fetch(K_s, Kb, 0);
+    fetch(V_s, Vb, 0);
     for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
         const int i = idx / (HD / 2), e = idx - i * (HD / 2);
         rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
@@ -167,9 +184,9 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
             }
         }
     }
-    int nkeys = ncache;
     if (last) {
-        // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached, behind the cached keys
+        // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached: appended to the cache and kept
+        // aside; they join the last tile behind its cached keys
         for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
             const int i = idx / (HD / 2), e = idx - i * (HD / 2);
             const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
@@ -179,111 +196,145 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
             const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
             const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
             const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
-            const int j = ncache + i;
-            K_s[j * KSTR + e] = k0; K_s[j * KSTR + e + HD / 2] = k1;
-            V_s[j * KSTR + e] = v0; V_s[j * KSTR + e + HD / 2] = v1;
+            Kn_s[i * KSTR + e] = k0; Kn_s[i * KSTR + e + HD / 2] = k1;
+            Vn_s[i * KSTR + e] = v0; Vn_s[i * KSTR + e + HD / 2] = v1;
             Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
             Vb[(size_t)(len + i) * HD + e] = v0; Vb[(size_t)(len + i) * HD + e + HD / 2] = v1;
         }
-        nkeys += T;
     }
-    const int nkp = (nkeys + 15) & ~15;            // keys rounded to the MMA k step
-    // V rows of the padding keys must be finite: their probabilities are zero, and 0 * NaN is not
-    for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += AT_THREADS) {
-        const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
-        *reinterpret_cast<uint4 *>(V_s + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
-    }
-    cp_async_wait_all();
-    __syncthreads();
-
-    // ---- scores S = Q K^T on the tensor cores: a warp takes 32 keys at a time for all query rows
+    if (tid < GT) { ml_s[2 * tid] = -INFINITY; ml_s[2 * tid + 1] = 0.f; }
     const int g8 = lane >> 2, t4 = lane & 3;
-    for (int grp = warp; grp * 32 < nkp; grp += AT_WARPS) {
-        const int kb = grp * 32;
-        float S[MT][4][4];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) { S[mt][nt][0] = S[mt][nt][1] = S[mt][nt][2] = S[mt][nt][3] = 0.f; }
-#pragma unroll 2
-        for (int ks = 0; ks < HD / 16; ++ks) {
-            uint32_t bk[2][4];
-#pragma unroll
-            for (int p = 0; p < 2; ++p)
-                ldsm_x4(bk[p], K_s + (size_t)(kb + p * 16 + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                uint32_t ah[4], al[4];
-                const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
-                ldsm_x4(ah, Qh_s + qo);
-                ldsm_x4(al, Ql_s + qo);
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], ah, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], al, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
-            }
-        }
-        // raw scores to shared memory; keys beyond the chunk and, among the new rows, later positions are masked
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int row = mt * 16 + g8 + (e >> 1) * 8, key = kb + nt * 8 + 2 * t4 + (e & 1);
-                    if (row < GT && key < nkp) {
-                        const bool masked = key >= nkeys || (last && key >= ncache && (key - ncache) > (row - (int)((row * tinv) >> 16) * T));
-                        s_s[row * SSTR + key] = masked ? -INFINITY : S[mt][nt][e];
-                    }
-                }
-    }
-    __syncthreads();
-    // ---- softmax of the chunk: one warp per query row; probabilities as bf16 head + remainder
-    for (int q0 = 0; q0 < GT; q0 += AT_THREADS / 8) {        // eight lanes per query row, sixteen rows per pass
-        const int qi = q0 + (tid >> 3), sub = tid & 7;
-        const bool rv = qi < GT;
-        float mx = -INFINITY;
-        if (rv) for (int j = sub; j < nkp; j += 8) mx = fmaxf(mx, s_s[qi * SSTR + j]);
-#pragma unroll
-        for (int o = 4; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float sum = 0.f;
-        if (rv)
-            for (int j = sub; j < nkp; j += 8) {
-                const float p = expf(s_s[qi * SSTR + j] - mx);   // expf(-inf) = 0 for masked keys
-                __nv_bfloat16 h, l;
-                split_bf16(p, h, l);
-                Ph_s[qi * PSTR + j] = h; Pl_s[qi * PSTR + j] = l;
-                sum += p;
-            }
-#pragma unroll
-        for (int o = 4; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        if (rv && sub == 0) { ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = sum; }
-    }
-    __syncthreads();
-    // ---- acc = P V on the tensor cores: a warp takes a quarter of the head dimension over all keys
     constexpr int DW = HD / AT_WARPS, NTW = DW / 8;
     float O[MT][NTW][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) { O[mt][nt][0] = O[mt][nt][1] = O[mt][nt][2] = O[mt][nt][3] = 0.f; }
-    for (int kk = 0; kk < nkp / 16; ++kk) {
-        uint32_t bv[NTW / 2][4];
-#pragma unroll
-        for (int p = 0; p < NTW / 2; ++p)
-            ldsm_x4_t(bv[p], V_s + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + warp * DW + p * 16 + (lane >> 4) * 8);
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            uint32_t ah[4], al[4];
-            const size_t po = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PSTR + kk * 16 + (lane >> 4) * 8;
-            ldsm_x4(ah, Ph_s + po);
-            ldsm_x4(al, Pl_s + po);
-#pragma unroll
-            for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], ah, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
-#pragma unroll
-            for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], al, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
+    __syncthreads();                        // queries, new rows, running stats in place
+
+    for (int t = 0; t < ntile; ++t) {
+        const int ncache = max(0, min(CK, rc - t * CK));
+        const bool lastt = last && t == ntile - 1;     // the tile that also holds the new rows
+        const int nkeys = ncache + (lastt ? T : 0);
+        const int nkp = (nkeys + 15) & ~15;            // keys rounded to the MMA k step
+        if (lastt) {
+            for (int idx = tid; idx < T * (HD / 8); idx += AT_THREADS) {
+                const int i = idx / (HD / 8), c = idx - i * (HD / 8);
+                *reinterpret_cast<uint4 *>(K_s + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Kn_s + (size_t)i * KSTR + 8 * c);
+                *reinterpret_cast<uint4 *>(V_s + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Vn_s + (size_t)i * KSTR + 8 * c);
+            }
+            // V rows of the padding keys must be finite: their probabilities are zero, and 0 * NaN is not
+            for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += AT_THREADS) {
+                const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
+                *reinterpret_cast<uint4 *>(V_s + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+            }
         }
+        cp_async_wait_but_one();            // K of this tile has landed (V may still be in flight)
+        __syncthreads();
+
+        // ---- scores S = Q K^T on the tensor cores: a warp takes 32 keys at a time for all query rows
+        for (int grp = warp; grp * 32 < nkp; grp += AT_WARPS) {
+            const int kb = grp * 32;
+            float S[MT][4][4];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) { S[mt][nt][0] = S[mt][nt][1] = S[mt][nt][2] = S[mt][nt][3] = 0.f; }
+#pragma unroll 2
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                uint32_t bk[2][4];
+#pragma unroll
+                for (int p = 0; p < 2; ++p)
+                    ldsm_x4(bk[p], K_s + (size_t)(kb + p * 16 + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    uint32_t ah[4], al[4];
+                    const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
+                    ldsm_x4(ah, Qh_s + qo);
+                    ldsm_x4(al, Ql_s + qo);
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], ah, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], al, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+                }
+            }
+            // raw scores to shared memory; keys beyond the tile and, among the new rows, later positions are masked
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int row = mt * 16 + g8 + (e >> 1) * 8, key = kb + nt * 8 + 2 * t4 + (e & 1);
+                        if (row < GT && key < nkp) {
+                            const bool masked = key >= nkeys || (lastt && key >= ncache && (key - ncache) > (row - (int)((row * tinv) >> 16) * T));
+                            s_s[row * SSTR + key] = masked ? -INFINITY : S[mt][nt][e];
+                        }
+                    }
+        }
+        __syncthreads();
+        fetch(K_s, Kb, t + 1);              // the K buffer is free: next tile's keys arrive during softmax and P V
+        // ---- softmax of the tile folded into the running (max, sum): eight lanes per query row, sixteen rows
+        //      per pass; probabilities as bf16 head + remainder
+        for (int q0 = 0; q0 < GT; q0 += AT_THREADS / 8) {
+            const int qi = q0 + (tid >> 3), sub = tid & 7;
+            const bool rv = qi < GT;
+            const float m_old = rv ? ml_s[2 * qi] : -INFINITY, l_old = rv ? ml_s[2 * qi + 1] : 0.f;
+            float mx = m_old;
+            if (rv) for (int j = sub; j < nkp; j += 8) mx = fmaxf(mx, s_s[qi * SSTR + j]);
+#pragma unroll
+            for (int o = 4; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float sum = 0.f;
+            if (rv)
+                for (int j = sub; j < nkp; j += 8) {
+                    const float sv = s_s[qi * SSTR + j];
+                    const float p = sv == -INFINITY ? 0.f : expf(sv - mx);
+                    __nv_bfloat16 h, l;
+                    split_bf16(p, h, l);
+                    Ph_s[qi * PSTR + j] = h; Pl_s[qi * PSTR + j] = l;
+                    sum += p;
+                }
+#pragma unroll
+            for (int o = 4; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (rv && sub == 0) {
+                const float corr = m_old == -INFINITY ? 0.f : expf(m_old - mx);
+                ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = fmaf(l_old, corr, sum);
+                corr_s[qi] = corr;
+            }
+        }
+        cp_async_wait_but_one();            // V of this tile has landed (the next K may still be in flight)
+        __syncthreads();
+        // ---- acc = acc * corr + P V on the tensor cores: a warp takes a quarter of the head dimension
+        if (t > 0) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const int r0 = mt * 16 + g8, r1 = r0 + 8;
+                const float c0r = r0 < GT ? corr_s[r0] : 1.f, c1r = r1 < GT ? corr_s[r1] : 1.f;
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt) { O[mt][nt][0] *= c0r; O[mt][nt][1] *= c0r; O[mt][nt][2] *= c1r; O[mt][nt][3] *= c1r; }
+            }
+        }
+        for (int kk = 0; kk < nkp / 16; ++kk) {
+            uint32_t bv[NTW / 2][4];
+#pragma unroll
+            for (int p = 0; p < NTW / 2; ++p)
+                ldsm_x4_t(bv[p], V_s + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + warp * DW + p * 16 + (lane >> 4) * 8);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                uint32_t ah[4], al[4];
+                const size_t po = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PSTR + kk * 16 + (lane >> 4) * 8;
+                ldsm_x4(ah, Ph_s + po);
+                ldsm_x4(al, Pl_s + po);
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], ah, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
+#pragma unroll
+                for (int nt = 0; nt < NTW; ++nt) mma_bf16(O[mt][nt], al, bv[nt >> 1][(nt & 1) * 2], bv[nt >> 1][(nt & 1) * 2 + 1]);
+            }
+        }
+        __syncthreads();                    // everybody is done with V, P and the scores of this tile
+        fetch(V_s, Vb, t + 1);
     }
+    cp_async_wait_all();                    // only empty groups can be left
     // ---- this CTA's partial into its own shared memory (the query tiles are no longer needed)
     float *acc_s = reinterpret_cast<float *>(Qh_s);          // [GT][HD] fp32
 #pragma unroll
@@ -424,7 +475,7 @@ cudaError_t configure_attn() {
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     const int GT = (a.qh / a.kvh) * a.T;
-    if (GT > HS_MAX_GT || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128)) return cudaErrorInvalidValue;
+    if (GT > HS_MAX_GT || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128) || a.tiles < 1) return cudaErrorInvalidValue;
     const int mt = (GT + 15) / 16;
 #define CASE(hd_, m_) if (a.hd == hd_ && mt == m_) return launch_t<hd_, m_>(a, s)
     CASE(128, 1); CASE(128, 2); CASE(128, 3); CASE(64, 1); CASE(64, 2); CASE(64, 3);

@@ -59,6 +59,26 @@ def test_cfg2_full_size_real_acceptance(env):
     assert eng.device_status() == 0
 
 
+def test_cfg2_attention_geometries(env):
+    # the split of the KV cache over CTAs (keys per tile x tiles per CTA) is a launch-time choice: every
+    # setting, including several tiles per CTA (running softmax), ragged last tiles and more than one
+    # cluster per sequence, must reproduce the oracle on two sequences of different context length
+    s, eng, model, seqs = make(env, "cfg2_0p5b", 2, 4, 1024, {0, 1}, [700, 333])
+    with pytest.raises(RuntimeError):
+        eng.set_attn_geometry(48, 1)
+    rep = None
+    for chunk, tiles in ((32, 2), (32, 4), (64, 2), (64, 8), (128, 2), (128, 1), (0, 0)):
+        seqs = [model.new_seq(), model.new_seq()]
+        for b, n in enumerate((700, 333)):
+            env["harness"].inject_context(eng, seqs[b], s, b, n, 11 + b)
+        eng.set_batch(2)
+        eng.set_attn_geometry(chunk, tiles)
+        rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=[[2], [4]], rep=rep)
+        assert eng.device_status() == 0, (chunk, tiles)
+    print(rep)
+    assert rep.rounds == 7
+
+
 def test_cfg4_sequential_full_size(env):
     s, eng, model, seqs = make(env, "cfg4_seq", 1, 4, 1100, {0}, [1024])
     rep = env["harness"].run_rounds(eng, seqs, s, 2, 2, forced=[hi.forced_accept(2, 2, seq=1)])
