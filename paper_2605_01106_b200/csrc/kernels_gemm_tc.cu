@@ -154,12 +154,18 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
 template <int EPI>
 __device__ __forceinline__ void tc_finish8(const TcArgs &a, float (&v)[8], int r0, int nvalid, int row) {
     if (EPI == EPI_SWIGLU) {
-        const bool st = row + 1 < a.O && !(row & 1);
+        // weight rows come in (gate, up) pairs held by neighbouring lanes.  The even lane finishes the even
+        // columns of the pair, the odd lane the odd ones, so both lanes work and each evaluates one SiLU per two
+        // columns: lanes swap what the other needs (even sends its gate of column j + 1, odd its up of column j).
+        const bool odd = row & 1;
+        const bool st = (row | 1) < a.O;
         float *p = a.out + (size_t)r0 * a.ldo + (row >> 1);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float up = __shfl_down_sync(0xffffffffu, v[j], 1);           // the odd row of the pair
-            if (st && j < nvalid) p[(size_t)j * a.ldo] = silu_f(v[j]) * up;
+        for (int j = 0; j < 8; j += 2) {
+            const float got = __shfl_xor_sync(0xffffffffu, odd ? v[j] : v[j + 1], 1);
+            const float gate = odd ? got : v[j], up = odd ? v[j + 1] : got;
+            const int jj = j + (odd ? 1 : 0);
+            if (st && jj < nvalid) p[(size_t)jj * a.ldo] = gate / (1.f + __expf(-gate)) * up;
         }
     } else {
         const bool st = row < a.O;
