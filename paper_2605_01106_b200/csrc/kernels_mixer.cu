@@ -13,10 +13,12 @@
 namespace {
 using namespace hsd;
 
-constexpr int SSM_PR = 16;       // state rows (of P) per block
-constexpr int SSM_THREADS = 128; // 4 warps x 4 rows
+constexpr int SSM_THREADS = 128; // 4 warps x PR / 4 rows
 
-template <int EPL>               // floats of one state row held by a lane; N = 32 * EPL
+// EPL: floats of one state row held by a lane (N = 32 * EPL).  SSM_PR: state rows (of P) per block - 16
+// spreads one sequence over many blocks; 64 (a whole head) is for large batches, where the conv of the
+// shared B and C channels, redone by every block, would otherwise outweigh the state traffic.
+template <int EPL, int SSM_PR>
 __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(SsmArgs a) {
     constexpr int N = 32 * EPL;
     constexpr int VW = EPL < 4 ? EPL : 4;       // vector width of the state loads
@@ -273,10 +275,13 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
 }  // namespace
 
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
-    dim3 grid(a.P / SSM_PR, a.H, a.nb);
-    if (a.N == 64) return launch_pdl(ssm_kernel<2>, grid, dim3(SSM_THREADS), 0, s, a);
-    if (a.N == 128) return launch_pdl(ssm_kernel<4>, grid, dim3(SSM_THREADS), 0, s, a);
-    if (a.N == 256) return launch_pdl(ssm_kernel<8>, grid, dim3(SSM_THREADS), 0, s, a);
+    // a whole head per block once blocks of 16 rows would already fill the GPU several times over
+    const bool wide = a.P % 64 == 0 && (int64_t)(a.P / 16) * a.H * a.nb >= 148 * 32;
+    const dim3 grid(a.P / (wide ? 64 : 16), a.H, a.nb);
+#define CASE(n_, e_) if (a.N == n_) return wide ? launch_pdl(ssm_kernel<e_, 64>, grid, dim3(SSM_THREADS), 0, s, a) \
+                                                 : launch_pdl(ssm_kernel<e_, 16>, grid, dim3(SSM_THREADS), 0, s, a)
+    CASE(64, 2); CASE(128, 4); CASE(256, 8);
+#undef CASE
     return cudaErrorInvalidValue;
 }
 
