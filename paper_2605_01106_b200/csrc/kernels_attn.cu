@@ -17,7 +17,7 @@
 //    V are bf16 in the cache and enter exactly; the fp32 queries and probabilities are split into a
 //    bf16 head and a bf16 remainder (two MMAs), which keeps the products exact to 2^-17 - the
 //    comparison with the CPU oracle allows 1e-3 on states fed by this output.
-//    Scores: a warp takes 32 keys at a time for all query rows; one softmax per tile (the whole tile is
+//    Scores: a warp takes 16 keys at a time for all query rows; one softmax per tile (the whole tile is
 //    resident); P V: a warp takes a quarter of the head dimension over all keys of the tile.
 //  * The up to eight chunks of a cluster leave (m, l, acc) in their own shared memory and combine them
 //    through distributed shared memory, rank r summing an eighth of the output dimensions.  Longer
@@ -232,20 +232,18 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
         cp_async_wait_but_one();            // K of this tile has landed (V may still be in flight)
         __syncthreads();
 
-        // ---- scores S = Q K^T on the tensor cores: a warp takes 32 keys at a time for all query rows
-        for (int grp = warp; grp * 32 < nkp; grp += AT_WARPS) {
-            const int kb = grp * 32;
-            float S[MT][4][4];
+        // ---- scores S = Q K^T on the tensor cores: a warp takes 16 keys at a time for all query rows
+        for (int grp = warp; grp * 16 < nkp; grp += AT_WARPS) {
+            const int kb = grp * 16;
+            float S[MT][2][4];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt) { S[mt][nt][0] = S[mt][nt][1] = S[mt][nt][2] = S[mt][nt][3] = 0.f; }
-#pragma unroll 2
+                for (int nt = 0; nt < 2; ++nt) { S[mt][nt][0] = S[mt][nt][1] = S[mt][nt][2] = S[mt][nt][3] = 0.f; }
+#pragma unroll 4
             for (int ks = 0; ks < HD / 16; ++ks) {
-                uint32_t bk[2][4];
-#pragma unroll
-                for (int p = 0; p < 2; ++p)
-                    ldsm_x4(bk[p], K_s + (size_t)(kb + p * 16 + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
+                uint32_t bk[4];
+                ldsm_x4(bk, K_s + (size_t)(kb + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     uint32_t ah[4], al[4];
@@ -253,20 +251,20 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
                     ldsm_x4(ah, Qh_s + qo);
                     ldsm_x4(al, Ql_s + qo);
 #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], ah, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+                    for (int nt = 0; nt < 2; ++nt) mma_bf16(S[mt][nt], ah, bk[nt * 2], bk[nt * 2 + 1]);
 #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) mma_bf16(S[mt][nt], al, bk[nt >> 1][(nt & 1) * 2], bk[nt >> 1][(nt & 1) * 2 + 1]);
+                    for (int nt = 0; nt < 2; ++nt) mma_bf16(S[mt][nt], al, bk[nt * 2], bk[nt * 2 + 1]);
                 }
             }
             // raw scores to shared memory; keys beyond the tile and, among the new rows, later positions are masked
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt)
+                for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int row = mt * 16 + g8 + (e >> 1) * 8, key = kb + nt * 8 + 2 * t4 + (e & 1);
-                        if (row < GT && key < nkp) {
+                        if (row < GT) {
                             const bool masked = key >= nkeys || (lastt && key >= ncache && (key - ncache) > (row - (int)((row * tinv) >> 16) * T));
                             s_s[row * SSTR + key] = masked ? -INFINITY : S[mt][nt][e];
                         }
@@ -276,17 +274,18 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
         fetch(K_s, Kb, t + 1);              // the K buffer is free: next tile's keys arrive during softmax and P V
         // ---- softmax of the tile folded into the running (max, sum): eight lanes per query row, sixteen rows
         //      per pass; probabilities as bf16 head + remainder
-        for (int q0 = 0; q0 < GT; q0 += AT_THREADS / 8) {
-            const int qi = q0 + (tid >> 3), sub = tid & 7;
+        constexpr int LPR = MT == 1 ? 8 : 4;          // lanes per query row: one pass covers 16 (MT = 1) or 32 rows
+        for (int q0 = 0; q0 < GT; q0 += AT_THREADS / LPR) {
+            const int qi = q0 + tid / LPR, sub = tid % LPR;
             const bool rv = qi < GT;
             const float m_old = rv ? ml_s[2 * qi] : -INFINITY, l_old = rv ? ml_s[2 * qi + 1] : 0.f;
             float mx = m_old;
-            if (rv) for (int j = sub; j < nkp; j += 8) mx = fmaxf(mx, s_s[qi * SSTR + j]);
+            if (rv) for (int j = sub; j < nkp; j += LPR) mx = fmaxf(mx, s_s[qi * SSTR + j]);
 #pragma unroll
-            for (int o = 4; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            for (int o = LPR / 2; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             float sum = 0.f;
             if (rv)
-                for (int j = sub; j < nkp; j += 8) {
+                for (int j = sub; j < nkp; j += LPR) {
                     const float sv = s_s[qi * SSTR + j];
                     const float p = sv == -INFINITY ? 0.f : expf(sv - mx);
                     __nv_bfloat16 h, l;
@@ -295,7 +294,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
                     sum += p;
                 }
 #pragma unroll
-            for (int o = 4; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            for (int o = LPR / 2; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             if (rv && sub == 0) {
                 const float corr = m_old == -INFINITY ? 0.f : expf(m_old - mx);
                 ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = fmaf(l_old, corr, sum);
