@@ -238,6 +238,8 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         ga.xb = m->xb; ga.xb_rows = m->xb_rows;
         PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, st_w, s, &m->launches, nullptr), "in_proj");
         // (2) recurrent mixer
+        SsmArgs ssm_args{};
+        bool ssm_deferred = false;
         if (ly.type != HS_LAYER_ATT) {
             const size_t lrB = (size_t)ly.rl * m->B;
             const float *win_in; float *win_out = nullptr, *hist = nullptr;
@@ -260,7 +262,8 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
                 sa.state_in = st_in; sa.in_seq_stride = in_seq; sa.in_slot_stride = in_slot;
                 sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
                 sa.slot = m->ctrl.slot; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
-                PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
+                if (with_attn) { ssm_args = sa; ssm_deferred = true; }      // goes out together with the attention
+                else PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
             } else {
                 GdnArgs gd{};
                 gd.gh = c.gh; gd.dk = c.gdk; gd.dv = c.gdv; gd.convd = m->convd; gd.in_ld = m->in_rows_max;
@@ -271,7 +274,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
                 gd.slot = m->ctrl.slot; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
                 PROF(HS_PROF_MIXER, 0, launch_gdn(gd, s), "gdn");
             }
-            ++m->launches;
+            if (!ssm_deferred) ++m->launches;
         }
         // (3) attention over the cache + the new rows (full model only)
         if (with_attn) {
@@ -286,8 +289,17 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
             aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles;
             aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
-            PROF(HS_PROF_ATTN, 0, launch_attn(aa, s), "attention");
-            ++m->launches;
+            bool fused = false;
+            if (ssm_deferred) {
+                // a parallel block: mixer and attention are independent of each other - one launch for both
+                if (!ssm_wide(ssm_args)) PROF(HS_PROF_MIXER, 0, launch_ssm_attn(ssm_args, aa, s, &fused), "ssm + attention");
+                if (fused) ++m->launches;
+                else { PROF(HS_PROF_MIXER, 0, launch_ssm(ssm_args, s), "ssm"); ++m->launches; }
+            }
+            if (!fused) {
+                PROF(HS_PROF_ATTN, 0, launch_attn(aa, s), "attention");
+                ++m->launches;
+            }
         }
         // (4) out-projection(s) + residual:  h += W_out rmsnorm_gated(g)  (+ W_o o)
         GemvArgs go{};

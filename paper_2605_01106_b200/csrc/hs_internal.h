@@ -191,6 +191,9 @@ struct AttnArgs {
     int T, b0, nb;
 };
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);
+// mixer + attention of a parallel block in one launch (verify pass); *fused = false: not applicable, nothing launched
+cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s, bool *fused);
+bool ssm_wide(const SsmArgs &a);    // the mixer runs a whole head per block (large batch)
 
 // part: scratch of HS_ARGMAX_CHUNKS * 16 bytes per logits row (row slot b * Tm + i); counters: one int32 per
 // row slot, zero between launches

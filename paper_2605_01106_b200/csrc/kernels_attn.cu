@@ -25,6 +25,7 @@
 //    counter, no spinning) merges them in order, so the result is reproducible.
 #include "hs_internal.h"
 #include "hs_device.cuh"
+#include "ssm_body.cuh"
 #include <cooperative_groups.h>
 
 namespace {
@@ -88,9 +89,12 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &h, __nv_bfloa
     l = __float2bfloat16_rn(x - __bfloat162float(h));
 }
 
-template <int HD, int MT>       // MT: 16-row tiles of query rows (G*T <= 16 * MT)
-__global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
-    extern __shared__ __align__(128) unsigned char smraw[];
+// MT: 16-row tiles of query rows (G*T <= 16 * MT).  The body takes its block coordinates as arguments
+// (key range within the sequence, KV head, local sequence): it runs as a kernel of its own and as one of the
+// two roles of the fused mixer + attention launch.  `split` must be the CTA's x index within a cluster-aligned
+// row of the grid, so that split / 8 is the cluster and split % 8 the rank inside it.
+template <int HD, int MT>
+__device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, const int kh, const int lb, unsigned char *smraw) {
     const int CK = a.chunk;
     const int G = a.qh / a.kvh, T = a.T, GT = G * T;
     const AttnLayout L = attn_layout(HD, CK, GT);
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     float *red_s = reinterpret_cast<float *>(smraw + L.red_off);
     __shared__ int ticket_s;
 
-    const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
+    const int b = a.b0 + lb;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t tinv = (65536u + T - 1) / T;      // x / T == (x * tinv) >> 16 for the small x used here
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
@@ -447,10 +451,53 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
 }
 
 template <int HD, int MT>
+__global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    attn_body<HD, MT>(a, blockIdx.x, blockIdx.y, blockIdx.z, smraw);
+}
+
+// Verify pass of a parallel hybrid block: the Mamba-2 mixer and the attention read the same in-projection
+// output and feed the same out-projection, so they run as ONE launch - the first `attn_ctas` blocks (whole
+// clusters) are attention CTAs, the rest mixer CTAs - and the dependent-launch chain is one kernel shorter.
+struct FusedGeo { int attn_nx, attn_ctas, ssm_nx, ssm_ctas; };
+
+template <int EPL, int HD, int MT>
+__global__ void __launch_bounds__(AT_THREADS) ssm_attn_kernel(const SsmArgs sa, const AttnArgs aa, const FusedGeo g) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    const int id = blockIdx.x;
+    if (id < g.attn_ctas) {
+        const int split = id % g.attn_nx, t = id / g.attn_nx;
+        attn_body<HD, MT>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
+    } else if (id - g.attn_ctas < g.ssm_ctas) {
+        const int j = id - g.attn_ctas, bx = j % g.ssm_nx, t = j / g.ssm_nx;
+        ssm_body<EPL, 16>(sa, bx, t % sa.H, t / sa.H);
+    }
+}
+
+template <int HD, int MT>
 cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
     dim3 grid((a.nch + AT_CL - 1) / AT_CL * AT_CL, a.kvh, a.nb);
     const size_t smem = attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
     return launch_pdl_cluster(attn_kernel<HD, MT>, grid, dim3(AT_THREADS), smem, s, AT_CL, a);
+}
+
+template <int EPL, int HD, int MT>
+cudaError_t launch_fused_t(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s) {
+    FusedGeo g;
+    g.attn_nx = (a.nch + AT_CL - 1) / AT_CL * AT_CL;
+    g.attn_ctas = g.attn_nx * a.kvh * a.nb;
+    g.ssm_nx = sa.P / 16;
+    g.ssm_ctas = g.ssm_nx * sa.H * sa.nb;
+    const int total = (g.attn_ctas + g.ssm_ctas + AT_CL - 1) / AT_CL * AT_CL;
+    const size_t smem = attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_layout(HD, 128, MT * 16).total);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_pdl_cluster(ssm_attn_kernel<EPL, HD, MT>, dim3(total), dim3(AT_THREADS), smem, s, AT_CL, sa, a, g);
 }
 
 template <int HD, int MT>
@@ -480,4 +527,19 @@ cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     CASE(128, 1); CASE(128, 2); CASE(128, 3); CASE(64, 1); CASE(64, 2); CASE(64, 3);
 #undef CASE
     return cudaErrorInvalidValue;
+}
+
+// Fused launch for a parallel block of the verify pass; `fused` reports whether it applies (mixer blocks of
+// 16 state rows, 128 threads in both roles) - otherwise nothing is launched and the caller issues the two
+// kernels one after the other.
+cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s, bool *fused) {
+    const int GT = (a.qh / a.kvh) * a.T, mt = (GT + 15) / 16;
+    *fused = false;
+    if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128) || sa.P % 16) return cudaSuccess;
+#define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return launch_fused_t<e_, hd_, m_>(sa, a, s); }
+#define CASES(n_, e_) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)
+    CASES(64, 2) CASES(128, 4) CASES(256, 8)
+#undef CASES
+#undef CASE
+    return cudaSuccess;
 }

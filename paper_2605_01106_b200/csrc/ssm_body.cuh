@@ -1,0 +1,168 @@
+// Mamba-2 mixer block body (conv + SiLU + softplus + state recurrence + gate), shared by the stand-alone
+// mixer kernel and the fused mixer + attention kernel of the verify pass.
+#pragma once
+#include "hs_internal.h"
+#include "hs_device.cuh"
+
+namespace hsd {
+
+constexpr int SSM_THREADS = 128; // 4 warps x PR / 4 rows
+
+// EPL: floats of one state row held by a lane (N = 32 * EPL).  SSM_PR: state rows (of P) per block - 16
+// spreads one sequence over many blocks; 64 (a whole head) is for large batches, where the conv of the
+// shared B and C channels, redone by every block, would otherwise outweigh the state traffic.
+// The body takes its block coordinates as arguments: (row strip, head, local sequence); it is also one of the
+// two roles of the fused mixer + attention launch of the verify pass.
+template <int EPL, int SSM_PR>
+__device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const int by, const int bz) {
+    constexpr int N = 32 * EPL;
+    constexpr int VW = EPL < 4 ? EPL : 4;       // vector width of the state loads
+    constexpr int NVEC = EPL / VW;
+    constexpr int RPW = SSM_PR / (SSM_THREADS / 32);
+    __shared__ __align__(16) float Bs[HS_MAX_T][N], Cs[HS_MAX_T][N];
+    __shared__ float xs[HS_MAX_T][SSM_PR], dt_s[HS_MAX_T], a_s[HS_MAX_T];
+
+    const int p0 = bx * SSM_PR, h = by, lb = bz, b = a.b0 + lb;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, T = a.T;
+    const int rowbase = lb * T;
+    pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
+
+    // ---- before the wait only parameters are read; the recurrent state (written by an earlier kernel of
+    //      the step or of the previous round) is merely pulled towards L2 and loaded after the wait, together
+    //      with the in-projection's outputs, so that this kernel may start as early as its predecessor allows
+    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
+                        (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) +
+                        ((size_t)h * a.P + p0 + warp * RPW) * N;
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(sin_ + r * N + v * (32 * VW) + lane * VW));
+    float s[RPW][EPL];
+    // ---- still before the wait: the conv parameters.
+    // A thread owns the channels tid, tid + 128, ... of this block's set: its x strip, all of B and C.
+    constexpr int NCH = SSM_PR + 2 * N;
+    constexpr int CPT = (NCH + SSM_THREADS - 1) / SSM_THREADS;
+    __shared__ float zs[HS_MAX_T][SSM_PR];
+    const bool owner = (bx == 0 && by == 0);   // writes the shared B|C channels' history
+    float4 tap[CPT];
+    float bias[CPT], w0[CPT], w1[CPT], w2[CPT];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+            tap[q] = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
+            bias[q] = a.conv_b[gc];
+        }
+    }
+    const float Aexp = expf(a.A_log[h]), dtb = a.dt_bias[h], Dh = a.D[h];
+    pdl_wait();
+
+    // ---- after the wait: the state rows and the conv window (L2 hits), in flight with the sweep below
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v) {
+            const float *src = sin_ + r * N + v * (32 * VW) + lane * VW;
+            if (VW == 4) { float4 t = __ldcg(reinterpret_cast<const float4 *>(src)); s[r][v * 4] = t.x; s[r][v * 4 + 1] = t.y; s[r][v * 4 + 2] = t.z; s[r][v * 4 + 3] = t.w; }
+            else { float2 t = __ldcg(reinterpret_cast<const float2 *>(src)); s[r][0] = t.x; s[r][1] = t.y; }
+        }
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+            const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
+            w0[q] = __ldcg(win); w1[q] = __ldcg(win + a.convd); w2[q] = __ldcg(win + 2 * a.convd);
+        }
+    }
+    // ---- raw conv inputs, gate inputs and dt of all T positions: one sweep of independent loads
+    for (int idx = threadIdx.x; idx < T * NCH; idx += SSM_THREADS) {
+        const int i = idx / NCH, c = idx - i * NCH;
+        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+        const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc);
+        if (c < SSM_PR) xs[i][c] = raw;
+        else if (c < SSM_PR + N) Bs[i][c - SSM_PR] = raw;
+        else Cs[i][c - SSM_PR - N] = raw;
+    }
+    for (int idx = threadIdx.x; idx < T * SSM_PR; idx += SSM_THREADS) {
+        const int i = idx / SSM_PR, c = idx - i * SSM_PR;
+        zs[i][c] = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c);
+    }
+    if (threadIdx.x < T) {
+        const float dt = softplus_f(__ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) + dtb);
+        dt_s[threadIdx.x] = dt;
+        a_s[threadIdx.x] = expf(-dt * Aexp);
+    }
+    __syncthreads();
+    // ---- causal conv + SiLU in place (one thread walks the positions of its channel)
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
+        if (c < NCH) {
+            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+            float *col = c < SSM_PR ? &xs[0][c] : c < SSM_PR + N ? &Bs[0][c - SSM_PR] : &Cs[0][c - SSM_PR - N];
+            const int stride = c < SSM_PR ? SSM_PR : N;
+            const bool wr = c < SSM_PR || owner;
+            float v0 = w0[q], v1 = w1[q], v2 = w2[q];
+            for (int i = 0; i < T; ++i) {
+                const float raw = col[i * stride];
+                col[i * stride] = silu_f(bias[q] + tap[q].x * v0 + tap[q].y * v1 + tap[q].z * v2 + tap[q].w * raw);
+                v0 = v1; v1 = v2; v2 = raw;
+                if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+            }
+            if (wr && a.win_out) {
+                float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
+                wo[0] = v0; wo[a.convd] = v1; wo[2 * a.convd] = v2;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- recurrence over the T positions
+    float *sout = a.state_out + (size_t)b * a.out_seq_stride + ((size_t)h * a.P + p0 + warp * RPW) * N;
+    for (int i = 0; i < T; ++i) {
+        const float dec = a_s[i], dt = dt_s[i];
+        float Bv[EPL], Cv[EPL];
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v)
+#pragma unroll
+            for (int j = 0; j < VW; ++j) {
+                Bv[v * VW + j] = Bs[i][v * (32 * VW) + lane * VW + j];
+                Cv[v * VW + j] = Cs[i][v * (32 * VW) + lane * VW + j];
+            }
+        float acc[RPW];
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const float dtx = dt * xs[i][warp * RPW + r];
+            float t = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                s[r][e] = fmaf(dec, s[r][e], dtx * Bv[e]);
+                t = fmaf(s[r][e], Cv[e], t);
+            }
+            acc[r] = t;
+        }
+        const float y = xreduce<RPW>(acc, lane);           // lanes l with l / (32/RPW) == r hold row r
+        constexpr int LPV = 32 / RPW;
+        if ((lane & (LPV - 1)) == 0) {
+            const int r = lane / LPV, col = h * a.P + p0 + warp * RPW + r;
+            const float z = zs[i][warp * RPW + r];
+            a.g[(size_t)(rowbase + i) * a.di + col] = (y + Dh * xs[i][warp * RPW + r]) * silu_f(z);
+        }
+        // state after position i (verify: snapshot i; draft: the scratch state)
+        float *dst = sout + (size_t)i * a.out_slot_stride;
+#pragma unroll
+        for (int r = 0; r < RPW; ++r)
+#pragma unroll
+            for (int v = 0; v < NVEC; ++v) {
+                float *p = dst + r * N + v * (32 * VW) + lane * VW;
+                if (VW == 4) *reinterpret_cast<float4 *>(p) = make_float4(s[r][v * 4], s[r][v * 4 + 1], s[r][v * 4 + 2], s[r][v * 4 + 3]);
+                else *reinterpret_cast<float2 *>(p) = make_float2(s[r][0], s[r][1]);
+            }
+    }
+}
+
+
+}  // namespace hsd
