@@ -117,3 +117,20 @@ def test_cfg5_batch64_ragged_sampled(env):
         kv, _ = eng.get_context(b)
         assert kv == lens[b] + int((np.array(forced[b]) + 1).sum())
     assert len(rep.n_hist) >= 2 and eng.device_status() == 0
+
+
+def test_cfg5_batch64_two_sequences_128_tokens(env):
+    # the long run of the batch-64 workload: 64 ragged sequences decode 128 tokens each (k = 4, seeded accept
+    # pattern, about 48 rounds); two of them carry their full context on the CPU side as well and are compared
+    # round by round over the whole generation, states every eighth round
+    s = hi.CONFIGS["cfg5_b64"]
+    lens = hi.context_lengths(64, 4096, 16384)
+    rounds = 48
+    s, eng, model, seqs = make(env, "cfg5_b64", 64, 4, 16384 + 5 * (rounds + 2), {5, 41}, lens)
+    forced = [hi.forced_accept(4, rounds, seq=100 + b) for b in range(64)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, rounds, forced=forced, check_states_every=8)
+    print(rep)
+    assert rep.tokens >= 2 * 110 and eng.device_status() == 0
+    for b in (5, 41):
+        kv, _ = eng.get_context(b)
+        assert kv == lens[b] + int((np.array(forced[b]) + 1).sum())
