@@ -470,7 +470,7 @@ __global__ void __launch_bounds__(AT_THREADS) ssm_attn_kernel(const SsmArgs sa, 
         attn_body<HD, MT>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
     } else if (id - g.attn_ctas < g.ssm_ctas) {
         const int j = id - g.attn_ctas, bx = j % g.ssm_nx, t = j / g.ssm_nx;
-        ssm_body<EPL, 16>(sa, bx, t % sa.H, t / sa.H);
+        ssm_body<EPL, 16, HS_MAX_T>(sa, bx, t % sa.H, t / sa.H);
     }
 }
 

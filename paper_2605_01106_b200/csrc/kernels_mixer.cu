@@ -14,9 +14,9 @@
 namespace {
 using namespace hsd;
 
-template <int EPL, int SSM_PR>
+template <int EPL, int SSM_PR, int TMAX>
 __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(const SsmArgs a) {
-    ssm_body<EPL, SSM_PR>(a, blockIdx.x, blockIdx.y, blockIdx.z);
+    ssm_body<EPL, SSM_PR, TMAX>(a, blockIdx.x, blockIdx.y, blockIdx.z);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -130,8 +130,10 @@ bool ssm_wide(const SsmArgs &a) { return a.P % 64 == 0 && (int64_t)(a.P / 16) * 
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
     const bool wide = ssm_wide(a);
     const dim3 grid(a.P / (wide ? 64 : 16), a.H, a.nb);
-#define CASE(n_, e_) if (a.N == n_) return wide ? launch_pdl(ssm_kernel<e_, 64>, grid, dim3(SSM_THREADS), 0, s, a) \
-                                                 : launch_pdl(ssm_kernel<e_, 16>, grid, dim3(SSM_THREADS), 0, s, a)
+#define CASE(n_, e_) if (a.N == n_) return a.T == 1 ? (wide ? launch_pdl(ssm_kernel<e_, 64, 1>, grid, dim3(SSM_THREADS), 0, s, a)     \
+                                                         : launch_pdl(ssm_kernel<e_, 16, 1>, grid, dim3(SSM_THREADS), 0, s, a))    \
+                                              : (wide ? launch_pdl(ssm_kernel<e_, 64, HS_MAX_T>, grid, dim3(SSM_THREADS), 0, s, a) \
+                                                      : launch_pdl(ssm_kernel<e_, 16, HS_MAX_T>, grid, dim3(SSM_THREADS), 0, s, a))
     CASE(64, 2); CASE(128, 4); CASE(256, 8);
 #undef CASE
     return cudaErrorInvalidValue;

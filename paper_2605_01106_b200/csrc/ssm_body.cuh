@@ -13,17 +13,19 @@ constexpr int SSM_THREADS = 128; // 4 warps x PR / 4 rows
 // shared B and C channels, redone by every block, would otherwise outweigh the state traffic.
 // The body takes its block coordinates as arguments: (row strip, head, local sequence); it is also one of the
 // two roles of the fused mixer + attention launch of the verify pass.
-template <int EPL, int SSM_PR>
+// TMAX: most positions this instance handles (1 for the draft step: a much shorter program, which matters
+// because every launch of a step starts with a cold instruction cache).
+template <int EPL, int SSM_PR, int TMAX>
 __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const int by, const int bz) {
     constexpr int N = 32 * EPL;
     constexpr int VW = EPL < 4 ? EPL : 4;       // vector width of the state loads
     constexpr int NVEC = EPL / VW;
     constexpr int RPW = SSM_PR / (SSM_THREADS / 32);
-    __shared__ __align__(16) float Bs[HS_MAX_T][N], Cs[HS_MAX_T][N];
-    __shared__ float xs[HS_MAX_T][SSM_PR], dt_s[HS_MAX_T], a_s[HS_MAX_T];
+    __shared__ __align__(16) float Bs[TMAX][N], Cs[TMAX][N];
+    __shared__ float xs[TMAX][SSM_PR], dt_s[TMAX], a_s[TMAX];
 
     const int p0 = bx * SSM_PR, h = by, lb = bz, b = a.b0 + lb;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, T = a.T;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, T = TMAX == 1 ? 1 : a.T;
     const int rowbase = lb * T;
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
@@ -43,7 +45,7 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
     // A thread owns the channels tid, tid + 128, ... of this block's set: its x strip, all of B and C.
     constexpr int NCH = SSM_PR + 2 * N;
     constexpr int CPT = (NCH + SSM_THREADS - 1) / SSM_THREADS;
-    __shared__ float zs[HS_MAX_T][SSM_PR];
+    __shared__ float zs[TMAX][SSM_PR];
     const bool owner = (bx == 0 && by == 0);   // writes the shared B|C channels' history
     float4 tap[CPT];
     float bias[CPT], w0[CPT], w1[CPT], w2[CPT];
@@ -77,26 +79,26 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
             w0[q] = __ldcg(win); w1[q] = __ldcg(win + a.convd); w2[q] = __ldcg(win + 2 * a.convd);
         }
     }
-    // ---- raw conv inputs, gate inputs and dt of all T positions: one sweep of independent loads
-    for (int idx = threadIdx.x; idx < T * NCH; idx += SSM_THREADS) {
-        const int i = idx / NCH, c = idx - i * NCH;
+    // ---- raw conv inputs of this thread's own channels for all T positions, gate inputs and dt: every load is
+    //      issued before the first value is used, so the whole phase costs one trip to L2
+    float raw[CPT][TMAX];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) {
+        const int c = threadIdx.x + q * SSM_THREADS;
         const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
-        const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc);
-        if (c < SSM_PR) xs[i][c] = raw;
-        else if (c < SSM_PR + N) Bs[i][c - SSM_PR] = raw;
-        else Cs[i][c - SSM_PR - N] = raw;
+#pragma unroll
+        for (int i = 0; i < TMAX; ++i)
+            raw[q][i] = (c < NCH && i < T) ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc) : 0.f;
     }
-    for (int idx = threadIdx.x; idx < T * SSM_PR; idx += SSM_THREADS) {
-        const int i = idx / SSM_PR, c = idx - i * SSM_PR;
-        zs[i][c] = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c);
+    constexpr int ZPT = (TMAX * SSM_PR + SSM_THREADS - 1) / SSM_THREADS;
+    float zraw[ZPT];
+#pragma unroll
+    for (int u = 0; u < ZPT; ++u) {
+        const int idx = threadIdx.x + u * SSM_THREADS, i = idx / SSM_PR, c = idx - i * SSM_PR;
+        zraw[u] = idx < T * SSM_PR ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c) : 0.f;
     }
-    if (threadIdx.x < T) {
-        const float dt = softplus_f(__ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) + dtb);
-        dt_s[threadIdx.x] = dt;
-        a_s[threadIdx.x] = expf(-dt * Aexp);
-    }
-    __syncthreads();
-    // ---- causal conv + SiLU in place (one thread walks the positions of its channel)
+    const float dtraw = threadIdx.x < T ? __ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) : 0.f;
+    // ---- causal conv + SiLU in registers (a thread walks the positions of its channels); results to shared memory
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
         const int c = threadIdx.x + q * SSM_THREADS;
@@ -106,17 +108,30 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
             const int stride = c < SSM_PR ? SSM_PR : N;
             const bool wr = c < SSM_PR || owner;
             float v0 = w0[q], v1 = w1[q], v2 = w2[q];
-            for (int i = 0; i < T; ++i) {
-                const float raw = col[i * stride];
-                col[i * stride] = silu_f(bias[q] + tap[q].x * v0 + tap[q].y * v1 + tap[q].z * v2 + tap[q].w * raw);
-                v0 = v1; v1 = v2; v2 = raw;
-                if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+#pragma unroll
+            for (int i = 0; i < TMAX; ++i) {
+                if (i < T) {
+                    const float r = raw[q][i];
+                    col[i * stride] = silu_f(bias[q] + tap[q].x * v0 + tap[q].y * v1 + tap[q].z * v2 + tap[q].w * r);
+                    v0 = v1; v1 = v2; v2 = r;
+                    if (wr && a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = r;
+                }
             }
             if (wr && a.win_out) {
                 float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
                 wo[0] = v0; wo[a.convd] = v1; wo[2 * a.convd] = v2;
             }
         }
+    }
+#pragma unroll
+    for (int u = 0; u < ZPT; ++u) {
+        const int idx = threadIdx.x + u * SSM_THREADS, i = idx / SSM_PR, c = idx - i * SSM_PR;
+        if (idx < T * SSM_PR) zs[i][c] = zraw[u];
+    }
+    if (threadIdx.x < T) {
+        const float dt = softplus_f(dtraw + dtb);
+        dt_s[threadIdx.x] = dt;
+        a_s[threadIdx.x] = expf(-dt * Aexp);
     }
     __syncthreads();
 
