@@ -39,6 +39,9 @@ struct GemvGeo {
     int D;               // tiles in flight per warp (depth of each warp's private ring)
     int krmax;           // max(kr0, kr1): row stride of the staged activations
     int off_x, off_nw, off_ring; // shared-memory carve-up (bytes)
+    int rq, rrem;        // row ranges: units / NR and units % NR
+    int nch;             // chunks of a full K range
+    long long pf_per;    // bytes of the next projection's weights each CTA pulls into L2
 };
 
 __device__ __forceinline__ float dot8(const uint4 &w, const float4 &a, const float4 &b, float acc) {
@@ -61,7 +64,11 @@ __device__ __forceinline__ int xs_pos(int c) {
 // A tile is WR weight rows x kc columns; warp w owns the row groups w, w + 8, ... of the CTA's row
 // range and walks each group's K chunks in order through a private ring of D tile buffers, so the
 // main loop needs no block-wide synchronisation.
-template <int R, int WR>
+// ONE = true is the single-row, single-segment instance of the draft step with the epilogue (EPI) and the
+// presence of a norm (NORMED) fixed at compile time: the same program with every unused path removed.  A step is
+// a chain of ~3 us kernels that each start with a cold instruction cache, so the length of the executed code
+// is a first-order cost there.  ONE = false (EPI = NORMED = -1: taken from the arguments) is the general form.
+template <int R, int WR, bool ONE = false, int EPI = -1, int NORMED = -1>
 __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
     constexpr int NV = pow2_ge(WR * R);
     constexpr int LPV = 32 / NV;
@@ -74,32 +81,34 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     __nv_bfloat16 *ring = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_ring);   // [8][D][WR][kc]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int S = g.S0 + g.S1;
-    const int ri = blockIdx.x / S, si = blockIdx.x - ri * S;
-    const bool seg1 = si >= g.S0;
+    const int si = blockIdx.x, ri = blockIdx.y;          // grid = (K splits, row ranges): no division to find them
+    const bool seg1 = ONE ? false : si >= g.S0;
     const __nv_bfloat16 *W = seg1 ? a.W1 : a.W0;
     const int ld = seg1 ? a.ldw1 : a.ldw0, Kseg = seg1 ? a.K1 : a.K0;
     const int krn = seg1 ? g.kr1 : g.kr0;
     const int k0 = (seg1 ? si - g.S0 : si) * krn;
     const int kr = min(krn, Kseg - k0);
-    const int units = a.O / g.unit;
-    const int r0 = (int)((long long)ri * units / g.NR) * g.unit;
-    const int r1 = (int)((long long)(ri + 1) * units / g.NR) * g.unit;
-    const int nrow = r1 - r0;
+    // row ranges: the first g.rrem ranges have g.rq + 1 units, the others g.rq (computed once on the host)
+    const int r0 = (ri * g.rq + min(ri, g.rrem)) * g.unit;
+    const int nrow = (g.rq + (ri < g.rrem ? 1 : 0)) * g.unit, r1 = r0 + nrow;
     const int kc = g.kc, D = g.D, krmax = g.krmax;
-    const int nch = (kr + kc - 1) / kc;
+    int nch = g.nch;                                      // chunks of a full K range; the last range may need fewer
+    while ((nch - 1) * kc >= kr) --nch;
     const int ngrp = (nrow + WR - 1) / WR;
     const int mygrps = warp < ngrp ? (ngrp - warp + GV_WARPS - 1) / GV_WARPS : 0;
     const int ntile = mygrps * nch;
     uint64_t *mybar = bars + warp * D;
     __nv_bfloat16 *mybuf = ring + (size_t)warp * D * WR * kc;
 
-    auto issue_tile = [&](int t) {         // whole warp
-        const int gi = t / nch, ch = t - gi * nch;
+    // tiles are requested strictly in order: (group, chunk, buffer) of the next request advance as counters
+    int i_gi = 0, i_ch = 0, i_buf = 0;
+    auto issue_tile = [&]() {              // whole warp
+        const int gi = i_gi, ch = i_ch, buf = i_buf;
+        if (++i_ch == nch) { i_ch = 0; ++i_gi; }
+        if (++i_buf == D) i_buf = 0;
         const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
         const int rows_in = min(WR, r1 - row0);
         const int cw = min(kc, kr - ch * kc);
-        const int buf = t % D;
         if (lane == 0) mbar_expect_tx(&mybar[buf], (uint32_t)rows_in * cw * 2);
         __syncwarp();
         if (ld == kc && cw == kc) {
@@ -118,19 +127,23 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     __syncthreads();
     {
         const int pre = min(D, ntile);
-        for (int t = 0; t < pre; ++t) issue_tile(t);
+#pragma unroll 1
+        for (int t = 0; t < pre; ++t) issue_tile();
     }
     // pull the next projection's weights towards L2: by the time its own kernel asks for them the
     // HBM latency is already paid
     if (a.pf_bytes > 0 && warp == GV_WARPS - 1) {
-        const long long per = ((a.pf_bytes / gridDim.x) + 15) & ~15ll;
-        const long long lo = (long long)blockIdx.x * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+        const long long per = g.pf_per;                   // bytes per CTA, a multiple of 16
+        const long long lo = (long long)(ri * gridDim.x + si) * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+#pragma unroll 1
         for (long long o = lo + (long long)lane * 8192; o < hi; o += 32 * 8192)
             prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
     }
     // the norm weights are parameters too: fetch them now, they would otherwise miss in L2 after the wait
-    const bool normed = a.norm_w != nullptr && !seg1;
+    const bool normed = NORMED >= 0 ? (NORMED != 0) : (a.norm_w != nullptr && !seg1);
+    const int epi = EPI >= 0 ? EPI : a.epi;
     if (normed)
+#pragma unroll 1
         for (int c = tid * 4; c < kr; c += GV_THREADS * 4)
             *reinterpret_cast<float4 *>(nw_s + c) = *reinterpret_cast<const float4 *>(a.norm_w + k0 + c);
     pdl_wait();
@@ -138,33 +151,41 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     __syncthreads();                       // nw_s complete
 
     // ---- stage the activation rows of this K range (parts summed, norm weight folded in)
-    const int nrows = a.nrows;
+    const int nrows = ONE ? 1 : a.nrows;
     {
         const float *xsrc = seg1 ? a.x1 : a.x0;
         const int ldx = seg1 ? a.ldx1 : a.ldx0;
         const int parts = seg1 ? 1 : a.xparts;
         const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
-        for (int rbase = 0; rbase < nrows; rbase += 4) {
-            float ss[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
-                float4 v[4];
+        constexpr int SR = ONE ? 1 : 4;                     // activation rows staged per sweep
+#pragma unroll 1
+        for (int rbase = 0; rbase < nrows; rbase += SR) {
+            float ss[SR];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {              // all loads of the four rows are in flight together
+            for (int j = 0; j < SR; ++j) ss[j] = 0.f;
+#pragma unroll 1
+            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
+                float4 v[SR];
+#pragma unroll
+                for (int j = 0; j < SR; ++j) {             // all loads of the rows of a sweep are in flight together
                     v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (rbase + j < nrows) {
                         const float *p = xsrc + (size_t)(rbase + j) * ldx + c;
                         v[j] = __ldcg(reinterpret_cast<const float4 *>(p));
-                        for (int q = 1; q < parts; ++q) {
-                            const float4 u = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
-                            v[j].x += u.x; v[j].y += u.y; v[j].z += u.z; v[j].w += u.w;
-                        }
+                        float4 u[HS_H_PARTS - 1];           // all parts in flight together, added in order
+#pragma unroll
+                        for (int q = 1; q < HS_H_PARTS; ++q)
+                            if (q < parts) u[q - 1] = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
+#pragma unroll
+                        for (int q = 1; q < HS_H_PARTS; ++q)
+                            if (q < parts) { v[j].x += u[q - 1].x; v[j].y += u[q - 1].y; v[j].z += u[q - 1].z; v[j].w += u[q - 1].w; }
                     }
                 }
                 const bool inside = c >= k0 && c < k0 + kr;
                 float4 nw = make_float4(1.f, 1.f, 1.f, 1.f);
                 if (normed && inside) nw = *reinterpret_cast<const float4 *>(nw_s + (c - k0));
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SR; ++j) {
                     if (rbase + j >= nrows) continue;
                     ss[j] = fmaf(v[j].x, v[j].x, fmaf(v[j].y, v[j].y, fmaf(v[j].z, v[j].z, fmaf(v[j].w, v[j].w, ss[j]))));
                     if (inside)
@@ -174,7 +195,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
             }
             if (normed) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SR; ++j) {
                     const float t = warp_sum(ss[j]);
                     if (lane == 0 && rbase + j < nrows) ss_s[warp * GV_MAXROWS + rbase + j] = t;
                 }
@@ -187,24 +208,38 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     const int vidx = lane / LPV, vr = vidx / WR, vw = vidx - vr * WR;
     const bool holder = (lane & (LPV - 1)) == 0 && vidx < WR * R;
     bool bad = false;
+    int g_buf = 0; uint32_t g_phase = 0;   // buffer and barrier phase of the first tile of the current row group
+    int t_next = min(D, ntile);            // tiles requested so far
+#pragma unroll 1
     for (int gi = 0; gi < mygrps; ++gi) {
         const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
         const int rows_in = min(WR, r1 - row0);
+        int c_buf = g_buf; uint32_t c_phase = g_phase;
+#pragma unroll 1
         for (int p0 = 0; p0 < nrows; p0 += R) {
+            c_buf = g_buf; c_phase = g_phase;               // every pass walks the group's tiles from its first buffer
             // residual of the value this lane will own: in flight while the tile is reduced
             float res = 0.f;
             const bool live = holder && p0 + vr < nrows && vw < rows_in;
             const size_t oi = (size_t)(p0 + vr) * a.ldo + row0 + vw;
-            if (a.epi == EPI_RESID && si == 0 && live)
-                for (int q = 0; q < a.rparts; ++q) res += __ldcg(a.resid + (size_t)q * a.rpstride + oi);
+            if (epi == EPI_RESID && si == 0 && live)
+            {
+                float rq[HS_H_PARTS];
+#pragma unroll
+                for (int q = 0; q < HS_H_PARTS; ++q) rq[q] = q < a.rparts ? __ldcg(a.resid + (size_t)q * a.rpstride + oi) : 0.f;
+#pragma unroll
+                for (int q = 0; q < HS_H_PARTS; ++q) res += rq[q];
+            }
             float acc[NV];
 #pragma unroll
             for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+#pragma unroll 1
             for (int ch = 0; ch < nch; ++ch) {
-                const int t = gi * nch + ch, buf = t % D;
-                if (p0 == 0 && !__all_sync(0xffffffffu, mbar_wait(&mybar[buf], (uint32_t)(t / D) & 1u))) { bad = true; break; }
+                const int buf = c_buf;
+                if (p0 == 0 && !__all_sync(0xffffffffu, mbar_wait(&mybar[buf], c_phase))) { bad = true; break; }
                 const __nv_bfloat16 *tile = mybuf + (size_t)buf * WR * kc;
                 const int nb = min(kc, kr - ch * kc) >> 8;
+#pragma unroll 2
                 for (int blk = 0; blk < nb; ++blk) {
                     const int col = (blk << 8) + lane * 8;
                     uint4 wv[WR];
@@ -222,8 +257,9 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
                 // last pass over the activation rows: this buffer is free, refill it D tiles ahead
                 if (p0 + R >= nrows) {
                     __syncwarp();
-                    if (t + D < ntile) issue_tile(t + D);
+                    if (t_next < ntile) { issue_tile(); ++t_next; }
                 }
+                if (++c_buf == D) { c_buf = 0; c_phase ^= 1u; }
             }
             if (bad) break;
             float tot = xreduce<NV>(acc, lane);
@@ -233,15 +269,16 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
                 for (int w = 0; w < GV_WARPS; ++w) t += ss_s[w * GV_MAXROWS + min(p0 + vr, nrows - 1)];
                 tot *= rsqrtf(t / (float)Kseg + a.eps);
             }
-            if (a.epi == EPI_SWIGLU) {
+            if (epi == EPI_SWIGLU) {
                 const float up = __shfl_down_sync(0xffffffffu, tot, LPV);    // value v + 1 = the up row of the pair
                 if (live && !(vw & 1)) a.out[(size_t)(p0 + vr) * a.ldo + ((row0 + vw) >> 1)] = silu_f(tot) * up;
             } else if (live) {
-                if (a.epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = tot + res;
+                if (epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = tot + res;
                 else a.out[oi] = tot;
             }
         }
         if (bad) break;
+        g_buf = c_buf; g_phase = c_phase;
     }
     if (bad) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);     // a copy never landed
 }
@@ -264,7 +301,8 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int NG>
+// EPI / NORMED >= 0 fix the epilogue and the presence of a norm at compile time (shorter program, see above).
+template <int NG, int EPI = -1, int NORMED = -1>
 __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
     constexpr int WR = 8;
     extern __shared__ __align__(128) unsigned char smraw[];
@@ -275,32 +313,32 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
     __nv_bfloat16 *ring = reinterpret_cast<__nv_bfloat16 *>(smraw + g.off_ring);   // [8][D][WR][kc + 8]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int S = g.S0 + g.S1;
-    const int ri = blockIdx.x / S, si = blockIdx.x - ri * S;
+    const int si = blockIdx.x, ri = blockIdx.y;          // grid = (K splits, row ranges)
     const bool seg1 = si >= g.S0;
     const __nv_bfloat16 *W = seg1 ? a.W1 : a.W0;
     const int ld = seg1 ? a.ldw1 : a.ldw0, Kseg = seg1 ? a.K1 : a.K0;
     const int krn = seg1 ? g.kr1 : g.kr0;
     const int k0 = (seg1 ? si - g.S0 : si) * krn;
     const int kr = min(krn, Kseg - k0);
-    const int units = a.O / g.unit;
-    const int r0 = (int)((long long)ri * units / g.NR) * g.unit;
-    const int r1 = (int)((long long)(ri + 1) * units / g.NR) * g.unit;
-    const int nrow = r1 - r0;
+    const int r0 = (ri * g.rq + min(ri, g.rrem)) * g.unit;
+    const int nrow = (g.rq + (ri < g.rrem ? 1 : 0)) * g.unit, r1 = r0 + nrow;
     const int kc = g.kc, D = g.D, krmax = g.krmax, TS = kc + 8, KP = krmax + 8;
-    const int nch = (kr + kc - 1) / kc;
+    int nch = g.nch;                                      // chunks of a full K range; the last range may need fewer
+    while ((nch - 1) * kc >= kr) --nch;
     const int ngrp = (nrow + WR - 1) / WR;
     const int mygrps = warp < ngrp ? (ngrp - warp + GV_WARPS - 1) / GV_WARPS : 0;
     const int ntile = mygrps * nch;
     uint64_t *mybar = bars + warp * D;
     __nv_bfloat16 *mybuf = ring + (size_t)warp * D * WR * TS;
 
-    auto issue_tile = [&](int t) {         // whole warp
-        const int gi = t / nch, ch = t - gi * nch;
+    int i_gi = 0, i_ch = 0, i_buf = 0;     // (group, chunk, buffer) of the next request
+    auto issue_tile = [&]() {              // whole warp
+        const int gi = i_gi, ch = i_ch, buf = i_buf;
+        if (++i_ch == nch) { i_ch = 0; ++i_gi; }
+        if (++i_buf == D) i_buf = 0;
         const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
         const int rows_in = min(WR, r1 - row0);
         const int cw = min(kc, kr - ch * kc);
-        const int buf = t % D;
         if (lane == 0) mbar_expect_tx(&mybar[buf], (uint32_t)rows_in * cw * 2);
         __syncwarp();
         if (lane < rows_in)
@@ -314,25 +352,32 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
     __syncthreads();
     {
         const int pre = min(D, ntile);
-        for (int t = 0; t < pre; ++t) issue_tile(t);
+#pragma unroll 1
+        for (int t = 0; t < pre; ++t) issue_tile();
     }
     if (a.pf_bytes > 0 && warp == GV_WARPS - 1) {
-        const long long per = ((a.pf_bytes / gridDim.x) + 15) & ~15ll;
-        const long long lo = (long long)blockIdx.x * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+        const long long per = g.pf_per;
+        const long long lo = (long long)(ri * gridDim.x + si) * per, hi = min(lo + per, (long long)a.pf_bytes & ~15ll);
+#pragma unroll 1
         for (long long o = lo + (long long)lane * 8192; o < hi; o += 32 * 8192)
             prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
     }
-    const bool normed = a.norm_w != nullptr && !seg1;
+    const bool normed = NORMED >= 0 ? (NORMED != 0 && !seg1) : (a.norm_w != nullptr && !seg1);
+    const int epi = EPI >= 0 ? EPI : a.epi;
     if (normed)
+#pragma unroll 1
         for (int c = tid * 4; c < kr; c += GV_THREADS * 4)
             *reinterpret_cast<float4 *>(nw_s + c) = *reinterpret_cast<const float4 *>(a.norm_w + k0 + c);
     const int nrows = a.nrows;
     // activation rows that do not exist are zero in both halves of their group
-    for (int idx = tid; idx < (NG * 8 - nrows) * (kr / 8); idx += GV_THREADS) {
-        const int r = nrows + idx / (kr / 8), c = (idx % (kr / 8)) * 8;
-        __nv_bfloat16 *p = xa_s + ((size_t)(r >> 3) * 16 + (r & 7)) * KP + c;
-        *reinterpret_cast<uint4 *>(p) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4 *>(p + 8 * KP) = make_uint4(0, 0, 0, 0);
+#pragma unroll 1
+    for (int r = nrows; r < NG * 8; ++r) {
+        __nv_bfloat16 *p = xa_s + ((size_t)(r >> 3) * 16 + (r & 7)) * KP;
+#pragma unroll 1
+        for (int c = tid * 8; c < kr; c += GV_THREADS * 8) {
+            *reinterpret_cast<uint4 *>(p + c) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(p + 8 * KP + c) = make_uint4(0, 0, 0, 0);
+        }
     }
     pdl_wait();
     if (!a.early_trigger) pdl_trigger();
@@ -344,6 +389,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
         const int ldx = seg1 ? a.ldx1 : a.ldx0;
         const int parts = seg1 ? 1 : a.xparts;
         const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
+#pragma unroll 1
         for (int rbase = 0; rbase < nrows; rbase += 4) {
             float ss[4] = {0.f, 0.f, 0.f, 0.f};
             for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
@@ -354,10 +400,13 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
                     if (rbase + j < nrows) {
                         const float *p = xsrc + (size_t)(rbase + j) * ldx + c;
                         v[j] = __ldcg(reinterpret_cast<const float4 *>(p));
-                        for (int q = 1; q < parts; ++q) {
-                            const float4 u = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
-                            v[j].x += u.x; v[j].y += u.y; v[j].z += u.z; v[j].w += u.w;
-                        }
+                        float4 u[HS_H_PARTS - 1];           // all parts in flight together, added in order
+#pragma unroll
+                        for (int q = 1; q < HS_H_PARTS; ++q)
+                            if (q < parts) u[q - 1] = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)q * a.xpstride));
+#pragma unroll
+                        for (int q = 1; q < HS_H_PARTS; ++q)
+                            if (q < parts) { v[j].x += u[q - 1].x; v[j].y += u[q - 1].y; v[j].z += u[q - 1].z; v[j].w += u[q - 1].w; }
                     }
                 }
                 const bool inside = c >= k0 && c < k0 + kr;
@@ -395,6 +444,9 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
     // this lane's results: activation row g * 8 + g8, weight rows 2 * t4 and 2 * t4 + 1 of the tile
     const int g8 = lane >> 2, t4 = lane & 3;
     bool bad = false;
+    int c_buf = 0; uint32_t c_phase = 0;   // buffer and barrier phase of the next tile to consume
+    int t_next = min(D, ntile);            // tiles requested so far
+#pragma unroll 1
     for (int gi = 0; gi < mygrps && !bad; ++gi) {
         const int row0 = r0 + (warp + gi * GV_WARPS) * WR;
         const int rows_in = min(WR, r1 - row0);
@@ -404,7 +456,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
         for (int gq = 0; gq < NG; ++gq) {
             res[gq][0] = res[gq][1] = 0.f;
             const int xr = gq * 8 + g8;
-            if (a.epi == EPI_RESID && si == 0 && xr < nrows)
+            if (epi == EPI_RESID && si == 0 && xr < nrows)
 #pragma unroll
                 for (int e = 0; e < 2; ++e)
                     if (2 * t4 + e < rows_in)
@@ -415,9 +467,10 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
         for (int gq = 0; gq < NG; ++gq)
 #pragma unroll
             for (int j = 0; j < 4; ++j) { acc[gq][j][0] = acc[gq][j][1] = acc[gq][j][2] = acc[gq][j][3] = 0.f; }
+#pragma unroll 1
         for (int ch = 0; ch < nch; ++ch) {
-            const int t = gi * nch + ch, buf = t % D;
-            if (!__all_sync(0xffffffffu, mbar_wait(&mybar[buf], (uint32_t)(t / D) & 1u))) { bad = true; break; }
+            const int buf = c_buf;
+            if (!__all_sync(0xffffffffu, mbar_wait(&mybar[buf], c_phase))) { bad = true; break; }
             const __nv_bfloat16 *tile = mybuf + (size_t)buf * WR * TS;
             const int cw = min(kc, kr - ch * kc);
             const __nv_bfloat16 *brow = tile + (size_t)(lane & 7) * TS + (lane >> 3) * 8;
@@ -436,7 +489,8 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
                     }
             }
             __syncwarp();
-            if (t + D < ntile) issue_tile(t + D);                // this buffer is free: refill it D tiles ahead
+            if (t_next < ntile) { issue_tile(); ++t_next; }     // this buffer is free: refill it D tiles ahead
+            if (++c_buf == D) { c_buf = 0; c_phase ^= 1u; }
         }
         if (bad) break;
 #pragma unroll
@@ -455,14 +509,14 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
                 v[0] *= rs; v[1] *= rs;
             }
             if (xr >= nrows) continue;
-            if (a.epi == EPI_SWIGLU) {
+            if (epi == EPI_SWIGLU) {
                 if (2 * t4 + 1 < rows_in) a.out[(size_t)xr * a.ldo + (wrow >> 1)] = silu_f(v[0]) * v[1];
             } else {
 #pragma unroll
                 for (int e = 0; e < 2; ++e)
                     if (2 * t4 + e < rows_in) {
                         const size_t oi = (size_t)xr * a.ldo + wrow + e;
-                        if (a.epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = v[e] + res[gq][e];
+                        if (epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = v[e] + res[gq][e];
                         else a.out[oi] = v[e];
                     }
             }
@@ -480,12 +534,21 @@ constexpr size_t GV_SMEM_PAIR = 127 * 1024;   // below this the CTA of the next 
 
 template <int NG>
 cudaError_t launch_mma(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
-    return launch_pdl(gemm_mma_kernel<NG>, dim3(g.NR * (g.S0 + g.S1)), dim3(GV_THREADS), smem, s, a, g, status);
+    const dim3 grid(g.S0 + g.S1, g.NR), block(GV_THREADS);
+    const int nm = a.norm_w ? 1 : 0;
+#define MM(ep, n) if (a.epi == ep && nm == n) return launch_pdl(gemm_mma_kernel<NG, ep, n>, grid, block, smem, s, a, g, status)
+    MM(EPI_STORE, 1); MM(EPI_STORE, 0); MM(EPI_RESID, 1); MM(EPI_RESID, 0); MM(EPI_SWIGLU, 1); MM(EPI_SWIGLU, 0);
+#undef MM
+    return cudaErrorInvalidValue;
 }
 
 template <int R, int WR>
 cudaError_t launch_rw(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
-    return launch_pdl(gemv_kernel<R, WR>, dim3(g.NR * (g.S0 + g.S1)), dim3(GV_THREADS), smem, s, a, g, status);
+    return launch_pdl(gemv_kernel<R, WR>, dim3(g.S0 + g.S1, g.NR), dim3(GV_THREADS), smem, s, a, g, status);
+}
+template <int WR, int EPI, int NORMED>
+cudaError_t launch_one(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
+    return launch_pdl(gemv_kernel<1, WR, true, EPI, NORMED>, dim3(g.S0, g.NR), dim3(GV_THREADS), smem, s, a, g, status);
 }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -504,9 +567,18 @@ cudaError_t configure_gemv() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<r, w>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
     CFG(1, 4); CFG(2, 4); CFG(3, 4); CFG(4, 4); CFG(1, 8); CFG(2, 8); CFG(3, 8); CFG(4, 8);
 #undef CFG
-#define CFGM(n) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
-    CFGM(1); CFGM(2);
+#define CFG1(w, ep, n) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<1, w, true, e_##ep, n>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<1, w, true, e_##ep, n>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+    constexpr int e_STORE = EPI_STORE, e_RESID = EPI_RESID, e_SWIGLU = EPI_SWIGLU;
+    CFG1(4, STORE, 1); CFG1(8, STORE, 1); CFG1(4, STORE, 0); CFG1(8, STORE, 0);
+    CFG1(4, RESID, 1); CFG1(8, RESID, 1); CFG1(4, RESID, 0); CFG1(8, RESID, 0);
+    CFG1(4, SWIGLU, 1); CFG1(8, SWIGLU, 1); CFG1(4, SWIGLU, 0); CFG1(8, SWIGLU, 0);
+#undef CFG1
+#define CFGM(n, ep, nm) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, ep, nm>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, ep, nm>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+#define CFGM6(n) CFGM(n, EPI_STORE, 1); CFGM(n, EPI_STORE, 0); CFGM(n, EPI_RESID, 1); CFGM(n, EPI_RESID, 0); CFGM(n, EPI_SWIGLU, 1); CFGM(n, EPI_SWIGLU, 0)
+    CFGM6(1); CFGM6(2);
+#undef CFGM6
 #undef CFGM
     return e;
 }
@@ -583,6 +655,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         if (g.off_ring + tile * ring_warps <= GV_SMEM_MAX || g.kc == 256) break;
     }
     const int nchunks = ceil_div(g.krmax, g.kc);
+    g.nch = nchunks; g.rq = units / g.NR; g.rrem = units % g.NR;
+    g.pf_per = ((a.pf_bytes / ((int64_t)g.NR * S)) + 15) & ~15ll;
     if (!mma && a.nrows > 4 && nchunks > 1) return rows_launch(4);   // passes need every chunk of a row group resident
     const int tiles_per_warp = ceil_div(ceil_div(nrow_max, WR), GV_WARPS) * nchunks;
     int D = 1;
@@ -594,6 +668,15 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
     if (launches) ++*launches;
     if (mma) return NG == 1 ? launch_mma<1>(a, g, smem, status, s) : launch_mma<2>(a, g, smem, status, s);
+    if (a.nrows == 1 && g.S1 == 0) {
+        // the draft step's projections: the pruned single-row instances
+        const int nm = a.norm_w ? 1 : 0;
+#define ONE(w, ep, n) if (WR == w && a.epi == ep && nm == n) return launch_one<w, ep, n>(a, g, smem, status, s)
+        ONE(4, EPI_STORE, 1); ONE(8, EPI_STORE, 1); ONE(4, EPI_STORE, 0); ONE(8, EPI_STORE, 0);
+        ONE(4, EPI_RESID, 1); ONE(8, EPI_RESID, 1); ONE(4, EPI_RESID, 0); ONE(8, EPI_RESID, 0);
+        ONE(4, EPI_SWIGLU, 1); ONE(8, EPI_SWIGLU, 1); ONE(4, EPI_SWIGLU, 0); ONE(8, EPI_SWIGLU, 0);
+#undef ONE
+    }
     // rows held in registers per pass: as even as possible over ceil(nrows / 4) passes
     const int npass = ceil_div(a.nrows, 4), R = ceil_div(a.nrows, npass);
 #define CASE(r, w) if (R == r && WR == w) return launch_rw<r, w>(a, g, smem, status, s)
