@@ -141,6 +141,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     auto fetch = [&](__nv_bfloat16 *dst, const __nv_bfloat16 *src, int t) {
         const int n = t < ntile ? max(0, min(CK, rc - t * CK)) : 0;
         const __nv_bfloat16 *from = src + (size_t)(c0 + t * CK) * HD;
+#pragma unroll 2
         for (int idx = tid; idx < n * (HD / 8); idx += AT_THREADS) {
             const int j = idx / (HD / 8), c = idx - j * (HD / 8);
             cp_async16(dst + (size_t)j * KSTR + 8 * c, from + (size_t)j * HD + 8 * c);
@@ -149,6 +150,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     };
     fetch(K_s, Kb, 0);
     fetch(V_s, Vb, 0);
+#pragma unroll 1
     for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
         const int i = idx / (HD / 2), e = idx - i * (HD / 2);
         rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
@@ -160,37 +162,41 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     const int rowbase = lb * T;
     const float scale = rsqrtf((float)HD);
     {
-        // thread = (rotation pair e, half of the query rows); all loads of a thread are issued before the first use
-        constexpr int HP = HD / 2, NH = AT_THREADS / HP;      // 64 pairs x 2 halves (hd 128) or 32 x 4 (hd 64)
-        constexpr int QPT = (HS_MAX_GT + NH - 1) / NH;        // query rows per thread
+        // thread = (rotation pair e, one of NH interleaved sets of query rows); four rows per round, whose loads
+        // are all issued before the first use
+        constexpr int HP = HD / 2, NH = AT_THREADS / HP;      // 64 pairs x 2 sets (hd 128) or 32 x 4 (hd 64)
         const int e = tid % HP, part = tid / HP;
-        float x0[QPT], x1[QPT];
+#pragma unroll 1
+        for (int q0 = part; q0 < GT; q0 += 4 * NH) {
+            float x0[4], x1[4];
 #pragma unroll
-        for (int u = 0; u < QPT; ++u) {
-            const int qi = part + u * NH;
-            x0[u] = x1[u] = 0.f;
-            if (qi < GT) {
-                const int gq = (int)((qi * tinv) >> 16);
-                const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
-                x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                x0[u] = x1[u] = 0.f;
+                if (qi < GT) {
+                    const int gq = (int)((qi * tinv) >> 16);
+                    const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                    x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
+                }
             }
-        }
 #pragma unroll
-        for (int u = 0; u < QPT; ++u) {
-            const int qi = part + u * NH;
-            if (qi < GT) {
-                const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
-                __nv_bfloat16 h, l;
-                split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
-                Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
-                split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
-                Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                if (qi < GT) {
+                    const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
+                    __nv_bfloat16 h, l;
+                    split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                    split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
+                }
             }
         }
     }
     if (last) {
         // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached: appended to the cache and kept
         // aside; they join the last tile behind its cached keys
+#pragma unroll 1
         for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
             const int i = idx / (HD / 2), e = idx - i * (HD / 2);
             const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
@@ -216,18 +222,21 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         for (int nt = 0; nt < NTW; ++nt) { O[mt][nt][0] = O[mt][nt][1] = O[mt][nt][2] = O[mt][nt][3] = 0.f; }
     __syncthreads();                        // queries, new rows, running stats in place
 
+#pragma unroll 1
     for (int t = 0; t < ntile; ++t) {
         const int ncache = max(0, min(CK, rc - t * CK));
         const bool lastt = last && t == ntile - 1;     // the tile that also holds the new rows
         const int nkeys = ncache + (lastt ? T : 0);
         const int nkp = (nkeys + 15) & ~15;            // keys rounded to the MMA k step
         if (lastt) {
+#pragma unroll 1
             for (int idx = tid; idx < T * (HD / 8); idx += AT_THREADS) {
                 const int i = idx / (HD / 8), c = idx - i * (HD / 8);
                 *reinterpret_cast<uint4 *>(K_s + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Kn_s + (size_t)i * KSTR + 8 * c);
                 *reinterpret_cast<uint4 *>(V_s + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Vn_s + (size_t)i * KSTR + 8 * c);
             }
             // V rows of the padding keys must be finite: their probabilities are zero, and 0 * NaN is not
+#pragma unroll 1
             for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += AT_THREADS) {
                 const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
                 *reinterpret_cast<uint4 *>(V_s + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
@@ -237,6 +246,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         __syncthreads();
 
         // ---- scores S = Q K^T on the tensor cores: a warp takes 16 keys at a time for all query rows
+#pragma unroll 1
         for (int grp = warp; grp * 16 < nkp; grp += AT_WARPS) {
             const int kb = grp * 16;
             float S[MT][2][4];
@@ -279,19 +289,23 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         // ---- softmax of the tile folded into the running (max, sum): eight lanes per query row, sixteen rows
         //      per pass; probabilities as bf16 head + remainder
         constexpr int LPR = MT == 1 ? 8 : 4;          // lanes per query row: one pass covers 16 (MT = 1) or 32 rows
+#pragma unroll 1
         for (int q0 = 0; q0 < GT; q0 += AT_THREADS / LPR) {
             const int qi = q0 + tid / LPR, sub = tid % LPR;
             const bool rv = qi < GT;
             const float m_old = rv ? ml_s[2 * qi] : -INFINITY, l_old = rv ? ml_s[2 * qi + 1] : 0.f;
             float mx = m_old;
-            if (rv) for (int j = sub; j < nkp; j += LPR) mx = fmaxf(mx, s_s[qi * SSTR + j]);
+            if (rv)
+#pragma unroll 4
+                for (int j = sub; j < nkp; j += LPR) mx = fmaxf(mx, s_s[qi * SSTR + j]);
 #pragma unroll
             for (int o = LPR / 2; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             float sum = 0.f;
             if (rv)
+#pragma unroll 2
                 for (int j = sub; j < nkp; j += LPR) {
                     const float sv = s_s[qi * SSTR + j];
-                    const float p = sv == -INFINITY ? 0.f : expf(sv - mx);
+                    const float p = sv == -INFINITY ? 0.f : __expf(sv - mx);
                     __nv_bfloat16 h, l;
                     split_bf16(p, h, l);
                     Ph_s[qi * PSTR + j] = h; Pl_s[qi * PSTR + j] = l;
@@ -300,7 +314,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
 #pragma unroll
             for (int o = LPR / 2; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             if (rv && sub == 0) {
-                const float corr = m_old == -INFINITY ? 0.f : expf(m_old - mx);
+                const float corr = m_old == -INFINITY ? 0.f : __expf(m_old - mx);
                 ml_s[2 * qi] = mx; ml_s[2 * qi + 1] = fmaf(l_old, corr, sum);
                 corr_s[qi] = corr;
             }
@@ -317,6 +331,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
                 for (int nt = 0; nt < NTW; ++nt) { O[mt][nt][0] *= c0r; O[mt][nt][1] *= c0r; O[mt][nt][2] *= c1r; O[mt][nt][3] *= c1r; }
             }
         }
+#pragma unroll 2
         for (int kk = 0; kk < nkp / 16; ++kk) {
             uint32_t bv[NTW / 2][4];
 #pragma unroll
@@ -357,6 +372,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     const int nclus = (nsplit + AT_CL - 1) / AT_CL;
     const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
     float *Md_s = red_s;                                     // [GT][2] merged (M, den), for the cluster partial
+#pragma unroll 1
     for (int idx = tid; idx < GT * DS; idx += AT_THREADS) {
         const int qi = idx / DS, dd = idx - qi * DS, d = crank * DS + dd;
         float2 mlr[AT_CL];
@@ -372,7 +388,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         float den = 0.f, sum = 0.f;
 #pragma unroll
         for (int r = 0; r < AT_CL; ++r) {
-            const float w = mlr[r].x == -INFINITY ? 0.f : expf(mlr[r].x - M);
+            const float w = mlr[r].x == -INFINITY ? 0.f : __expf(mlr[r].x - M);
             den = fmaf(w, mlr[r].y, den);
             sum = fmaf(w, v[r], sum);
         }
@@ -407,7 +423,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         float den = 0.f;
         for (int c = lane; c < nclus; c += 32) {
             const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
-            den = fmaf(expf(mlv.x - M), mlv.y, den);
+            den = fmaf(__expf(mlv.x - M), mlv.y, den);
         }
         den = warp_sum(den);
         if (lane == 0) { ml_s[2 * qi] = M; ml_s[2 * qi + 1] = den; }
@@ -420,7 +436,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         __syncthreads();                                     // ml_s ready / previous pass done with w_s
         for (int idx = tid; idx < GT * nc; idx += AT_THREADS) {
             const int qi = idx / nc, c = idx - qi * nc;
-            w_s[qi * SSTR + c] = expf(__ldcg(pm0 + ((size_t)(cb + c) * HS_MAX_GT + qi) * 2) - ml_s[2 * qi]);
+            w_s[qi * SSTR + c] = __expf(__ldcg(pm0 + ((size_t)(cb + c) * HS_MAX_GT + qi) * 2) - ml_s[2 * qi]);
         }
         __syncthreads();
         if (tid < HD) {
@@ -461,7 +477,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
 // clusters) are attention CTAs, the rest mixer CTAs - and the dependent-launch chain is one kernel shorter.
 struct FusedGeo { int attn_nx, attn_ctas, ssm_nx, ssm_ctas; };
 
-template <int EPL, int HD, int MT>
+template <int EPL, int HD, int MT, int TMAX>
 __global__ void __launch_bounds__(AT_THREADS) ssm_attn_kernel(const SsmArgs sa, const AttnArgs aa, const FusedGeo g) {
     extern __shared__ __align__(128) unsigned char smraw[];
     const int id = blockIdx.x;
@@ -470,7 +486,7 @@ __global__ void __launch_bounds__(AT_THREADS) ssm_attn_kernel(const SsmArgs sa, 
         attn_body<HD, MT>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
     } else if (id - g.attn_ctas < g.ssm_ctas) {
         const int j = id - g.attn_ctas, bx = j % g.ssm_nx, t = j / g.ssm_nx;
-        ssm_body<EPL, 16, HS_MAX_T>(sa, bx, t % sa.H, t / sa.H);
+        ssm_body<EPL, 16, TMAX>(sa, bx, t % sa.H, t / sa.H);
     }
 }
 
@@ -481,7 +497,7 @@ cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
     return launch_pdl_cluster(attn_kernel<HD, MT>, grid, dim3(AT_THREADS), smem, s, AT_CL, a);
 }
 
-template <int EPL, int HD, int MT>
+template <int EPL, int HD, int MT, int TMAX>
 cudaError_t launch_fused_t(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s) {
     FusedGeo g;
     g.attn_nx = (a.nch + AT_CL - 1) / AT_CL * AT_CL;
@@ -492,12 +508,12 @@ cudaError_t launch_fused_t(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s)
     const size_t smem = attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_layout(HD, 128, MT * 16).total);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        cudaError_t e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT, TMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_layout(HD, 128, MT * 16).total);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT, TMAX>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_pdl_cluster(ssm_attn_kernel<EPL, HD, MT>, dim3(total), dim3(AT_THREADS), smem, s, AT_CL, sa, a, g);
+    return launch_pdl_cluster(ssm_attn_kernel<EPL, HD, MT, TMAX>, dim3(total), dim3(AT_THREADS), smem, s, AT_CL, sa, a, g);
 }
 
 template <int HD, int MT>
@@ -536,7 +552,7 @@ cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s
     const int GT = (a.qh / a.kvh) * a.T, mt = (GT + 15) / 16;
     *fused = false;
     if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128) || sa.P % 16) return cudaSuccess;
-#define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return launch_fused_t<e_, hd_, m_>(sa, a, s); }
+#define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return a.T <= 3 ? launch_fused_t<e_, hd_, m_, 3>(sa, a, s) : launch_fused_t<e_, hd_, m_, HS_MAX_T>(sa, a, s); }
 #define CASES(n_, e_) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)
     CASES(64, 2) CASES(128, 4) CASES(256, 8)
 #undef CASES

@@ -130,12 +130,13 @@ bool ssm_wide(const SsmArgs &a) { return a.P % 64 == 0 && (int64_t)(a.P / 16) * 
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
     const bool wide = ssm_wide(a);
     const dim3 grid(a.P / (wide ? 64 : 16), a.H, a.nb);
-#define CASE(n_, e_) if (a.N == n_) return a.T == 1 ? (wide ? launch_pdl(ssm_kernel<e_, 64, 1>, grid, dim3(SSM_THREADS), 0, s, a)     \
-                                                         : launch_pdl(ssm_kernel<e_, 16, 1>, grid, dim3(SSM_THREADS), 0, s, a))    \
-                                              : (wide ? launch_pdl(ssm_kernel<e_, 64, HS_MAX_T>, grid, dim3(SSM_THREADS), 0, s, a) \
-                                                      : launch_pdl(ssm_kernel<e_, 16, HS_MAX_T>, grid, dim3(SSM_THREADS), 0, s, a))
+#define LAUNCH(e_, pr_, t_) launch_pdl(ssm_kernel<e_, pr_, t_>, grid, dim3(SSM_THREADS), 0, s, a)
+#define CASE(n_, e_) if (a.N == n_) return a.T == 1 ? (wide ? LAUNCH(e_, 64, 1) : LAUNCH(e_, 16, 1))               \
+                                         : a.T <= 3 ? (wide ? LAUNCH(e_, 64, 3) : LAUNCH(e_, 16, 3))               \
+                                                    : (wide ? LAUNCH(e_, 64, HS_MAX_T) : LAUNCH(e_, 16, HS_MAX_T))
     CASE(64, 2); CASE(128, 4); CASE(256, 8);
 #undef CASE
+#undef LAUNCH
     return cudaErrorInvalidValue;
 }
 
