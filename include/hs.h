@@ -178,8 +178,8 @@ int hs_get_round(hs_model *m, int32_t *cand_host, int32_t *g_host, float *margin
 int64_t hs_launch_count(const hs_model *m);
 /* Tuning hook for verify-mode attention (Sec. 3.3 verification pass): fix the split of the KV cache over
  * CTAs to `tiles` tiles of `chunk` keys per CTA for all following verify passes; chunk = 0 restores the
- * automatic choice (made per launch from the batch and the context lengths).  chunk is 32, 64 or 128,
- * tiles 1..64, and chunk * tiles must be at least the chunk the workspace was laid out for (128, or less
+ * automatic choice (made per launch from the batch and the context lengths).  chunk is a multiple of 16 up to 128,
+ * tiles 1..32, and chunk * tiles must be at least the chunk the workspace was laid out for (128, or less
  * for small batch * capacity): otherwise HS_ERR_INVALID_ARG and nothing changes.  Results do not depend on
  * the setting beyond fp32 summation order. */
 int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);

@@ -183,20 +183,22 @@ double gemv_bytes(const GemvArgs &a) {
 //   draft = false: full model M_H (verify);  draft = true: draft model M_S, one position,
 //   reading candidate column `col` and, for step > 0, the scratch state of the previous step.
 // ------------------------------------------------------------------------------------------------
-// Attention geometry of this launch.  Keys per tile: small enough to spread a short context over the eight
-// CTAs of one cluster (which combine their partials in shared memory), never below the size the partial
-// buffers were laid out for.  Tiles per CTA: one, unless the launch would have far more CTAs than the GPU
+// Attention geometry of this launch.  Keys per tile: the context is spread over the eight CTAs of one
+// cluster (which combine their partials in shared memory) - 32, 64, 96 or 128 keys each, whichever first
+// covers it - and never below the size the partial buffers were laid out for; longer contexts use 128-key
+// tiles over several clusters.  Tiles per CTA: one, unless the launch would have far more CTAs than the GPU
 // runs at once (long caches at large batch) - then a CTA walks up to sixteen 64-key tiles, so that staging
 // the queries and combining the partials is paid once per 1024 keys.
 struct AttnGeom {
     int chunk, tiles;
-    int code() const { return (chunk == 32 ? 0 : chunk == 64 ? 1 : 2) * 64 + tiles - 1; }   // < 256, part of the graph key
+    int code() const { return (chunk / 16 - 1) * 32 + tiles - 1; }   // < 256, part of the graph key
 };
 AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
     if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles};
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
-    const int want = maxlen + T <= 256 ? 32 : maxlen + T <= 512 ? 64 : 128;
+    int want = 32;
+    while (want < 128 && 8 * want < maxlen + T) want += 32;
     AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1};
     const int64_t ctas64 = (int64_t)nb * m->c.kvh * ((maxlen + T + 63) / 64);
     const int64_t fill = 148 * 8;             // CTAs that keep every SM busy for several rounds
@@ -712,8 +714,8 @@ int64_t hs_launch_count(const hs_model *m) { return m ? m->launches : -1; }
 int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
     if (!m) return HS_ERR_INVALID_ARG;
     if (chunk == 0) { m->att_force_chunk = m->att_force_tiles = 0; return HS_OK; }
-    if ((chunk != 32 && chunk != 64 && chunk != 128) || tiles < 1 || tiles > 64 || chunk * tiles < m->att_chunk)
-        return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk 32/64/128, tiles 1..64, chunk * tiles >= workspace chunk");
+    if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
+        return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk a multiple of 16 up to 128, tiles 1..32, chunk * tiles >= workspace chunk");
     m->att_force_chunk = chunk; m->att_force_tiles = tiles;
     return HS_OK;
 }

@@ -372,31 +372,36 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     const int nclus = (nsplit + AT_CL - 1) / AT_CL;
     const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
     float *Md_s = red_s;                                     // [GT][2] merged (M, den), for the cluster partial
+    constexpr int DV = DS / 4;                               // a thread takes four output dimensions of one query row
 #pragma unroll 1
-    for (int idx = tid; idx < GT * DS; idx += AT_THREADS) {
-        const int qi = idx / DS, dd = idx - qi * DS, d = crank * DS + dd;
+    for (int idx = tid; idx < GT * DV; idx += AT_THREADS) {
+        const int qi = idx / DV, dd = (idx - qi * DV) * 4, d = crank * DS + dd;
         float2 mlr[AT_CL];
-        float v[AT_CL];
+        float4 v[AT_CL];
 #pragma unroll
         for (int r = 0; r < AT_CL; ++r) {                    // all remote reads are independent: one round trip
             mlr[r] = *reinterpret_cast<const float2 *>(cluster.map_shared_rank(ml_s, r) + 2 * qi);
-            v[r] = cluster.map_shared_rank(acc_s, r)[qi * HD + d];
+            v[r] = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(acc_s, r) + qi * HD + d);
         }
         float M = -INFINITY;
 #pragma unroll
         for (int r = 0; r < AT_CL; ++r) M = fmaxf(M, mlr[r].x);
-        float den = 0.f, sum = 0.f;
+        float den = 0.f;
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int r = 0; r < AT_CL; ++r) {
             const float w = mlr[r].x == -INFINITY ? 0.f : __expf(mlr[r].x - M);
             den = fmaf(w, mlr[r].y, den);
-            sum = fmaf(w, v[r], sum);
+            sum.x = fmaf(w, v[r].x, sum.x); sum.y = fmaf(w, v[r].y, sum.y);
+            sum.z = fmaf(w, v[r].z, sum.z); sum.w = fmaf(w, v[r].w, sum.w);
         }
         if (nclus == 1) {
-            const int gq = qi / T, i = qi - gq * T;
-            o_base[(size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d] = sum / den;
+            const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
+            const float inv = 1.0f / den;
+            *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
+                make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
         } else {
-            a.part_acc[(pbase + cl) * HS_MAX_GT * HD + qi * HD + d] = sum;
+            *reinterpret_cast<float4 *>(a.part_acc + (pbase + cl) * HS_MAX_GT * HD + qi * HD + d) = sum;
             if (crank == 0 && dd == 0) { Md_s[2 * qi] = M; Md_s[2 * qi + 1] = den; }
         }
     }
@@ -537,7 +542,7 @@ cudaError_t configure_attn() {
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     const int GT = (a.qh / a.kvh) * a.T;
-    if (GT > HS_MAX_GT || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128) || a.tiles < 1) return cudaErrorInvalidValue;
+    if (GT > HS_MAX_GT || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || a.tiles < 1) return cudaErrorInvalidValue;
     const int mt = (GT + 15) / 16;
 #define CASE(hd_, m_) if (a.hd == hd_ && mt == m_) return launch_t<hd_, m_>(a, s)
     CASE(128, 1); CASE(128, 2); CASE(128, 3); CASE(64, 1); CASE(64, 2); CASE(64, 3);
@@ -551,7 +556,7 @@ cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
 cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s, bool *fused) {
     const int GT = (a.qh / a.kvh) * a.T, mt = (GT + 15) / 16;
     *fused = false;
-    if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || (a.chunk != 32 && a.chunk != 64 && a.chunk != 128) || sa.P % 16) return cudaSuccess;
+    if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || sa.P % 16) return cudaSuccess;
 #define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return a.T <= 3 ? launch_fused_t<e_, hd_, m_, 3>(sa, a, s) : launch_fused_t<e_, hd_, m_, HS_MAX_T>(sa, a, s); }
 #define CASES(n_, e_) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)
     CASES(64, 2) CASES(128, 4) CASES(256, 8)

@@ -65,9 +65,9 @@ def test_cfg2_attention_geometries(env):
     # cluster per sequence, must reproduce the oracle on two sequences of different context length
     s, eng, model, seqs = make(env, "cfg2_0p5b", 2, 4, 1024, {0, 1}, [700, 333])
     with pytest.raises(RuntimeError):
-        eng.set_attn_geometry(48, 1)
+        eng.set_attn_geometry(40, 1)
     rep = None
-    for chunk, tiles in ((32, 2), (32, 4), (64, 2), (64, 8), (128, 2), (128, 1), (0, 0)):
+    for chunk, tiles in ((32, 2), (32, 4), (48, 2), (64, 2), (64, 8), (96, 1), (128, 2), (128, 1), (0, 0)):
         seqs = [model.new_seq(), model.new_seq()]
         for b, n in enumerate((700, 333)):
             env["harness"].inject_context(eng, seqs[b], s, b, n, 11 + b)
@@ -76,7 +76,7 @@ def test_cfg2_attention_geometries(env):
         rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=[[2], [4]], rep=rep)
         assert eng.device_status() == 0, (chunk, tiles)
     print(rep)
-    assert rep.rounds == 7
+    assert rep.rounds == 9
 
 
 def test_cfg4_sequential_full_size(env):
