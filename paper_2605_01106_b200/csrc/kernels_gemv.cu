@@ -64,11 +64,12 @@ __device__ __forceinline__ int xs_pos(int c) {
 // A tile is WR weight rows x kc columns; warp w owns the row groups w, w + 8, ... of the CTA's row
 // range and walks each group's K chunks in order through a private ring of D tile buffers, so the
 // main loop needs no block-wide synchronisation.
-// ONE = true is the single-row, single-segment instance of the draft step with the epilogue (EPI) and the
-// presence of a norm (NORMED) fixed at compile time: the same program with every unused path removed.  A step is
-// a chain of ~3 us kernels that each start with a cold instruction cache, so the length of the executed code
-// is a first-order cost there.  ONE = false (EPI = NORMED = -1: taken from the arguments) is the general form.
-template <int R, int WR, bool ONE = false, int EPI = -1, int NORMED = -1>
+// ONE = true is the lean instance for exactly R activation rows (1: the draft step, 2 or 3: verify at k = 1, 2)
+// with the epilogue (EPI) and the presence of a norm (NORMED) fixed at compile time: the same program with every
+// unused path removed.  A step is a chain of ~3 us kernels, so the length of the executed code is a first-order
+// cost there.  ONE = false (EPI = NORMED = -1: taken from the arguments) is the general form.
+// SEG = false: the instance knows there is no second weight segment.
+template <int R, int WR, bool ONE = false, int EPI = -1, int NORMED = -1, bool SEG = true>
 __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
     constexpr int NV = pow2_ge(WR * R);
     constexpr int LPV = 32 / NV;
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int si = blockIdx.x, ri = blockIdx.y;          // grid = (K splits, row ranges): no division to find them
-    const bool seg1 = ONE ? false : si >= g.S0;
+    const bool seg1 = SEG ? si >= g.S0 : false;
     const __nv_bfloat16 *W = seg1 ? a.W1 : a.W0;
     const int ld = seg1 ? a.ldw1 : a.ldw0, Kseg = seg1 ? a.K1 : a.K0;
     const int krn = seg1 ? g.kr1 : g.kr0;
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
             prefetch_l2(reinterpret_cast<const char *>(a.pf_ptr) + o, (uint32_t)min(8192ll, hi - o));
     }
     // the norm weights are parameters too: fetch them now, they would otherwise miss in L2 after the wait
-    const bool normed = NORMED >= 0 ? (NORMED != 0) : (a.norm_w != nullptr && !seg1);
+    const bool normed = NORMED >= 0 ? (NORMED != 0 && !seg1) : (a.norm_w != nullptr && !seg1);
     const int epi = EPI >= 0 ? EPI : a.epi;
     if (normed)
 #pragma unroll 1
@@ -151,13 +152,13 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, c
     __syncthreads();                       // nw_s complete
 
     // ---- stage the activation rows of this K range (parts summed, norm weight folded in)
-    const int nrows = ONE ? 1 : a.nrows;
+    const int nrows = ONE ? R : a.nrows;
     {
         const float *xsrc = seg1 ? a.x1 : a.x0;
         const int ldx = seg1 ? a.ldx1 : a.ldx0;
         const int parts = seg1 ? 1 : a.xparts;
         const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
-        constexpr int SR = ONE ? 1 : 4;                     // activation rows staged per sweep
+        constexpr int SR = ONE ? R : 4;                     // activation rows staged per sweep
 #pragma unroll 1
         for (int rbase = 0; rbase < nrows; rbase += SR) {
             float ss[SR];
@@ -546,9 +547,16 @@ template <int R, int WR>
 cudaError_t launch_rw(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
     return launch_pdl(gemv_kernel<R, WR>, dim3(g.S0 + g.S1, g.NR), dim3(GV_THREADS), smem, s, a, g, status);
 }
-template <int WR, int EPI, int NORMED>
-cudaError_t launch_one(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
-    return launch_pdl(gemv_kernel<1, WR, true, EPI, NORMED>, dim3(g.S0, g.NR), dim3(GV_THREADS), smem, s, a, g, status);
+template <int R, int WR, int EPI, int NORMED, bool SEG>
+cudaError_t launch_lean(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_kernel<R, WR, true, EPI, NORMED, SEG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(224 * 1024));
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<R, WR, true, EPI, NORMED, SEG>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_pdl(gemv_kernel<R, WR, true, EPI, NORMED, SEG>, dim3(g.S0 + g.S1, g.NR), dim3(GV_THREADS), smem, s, a, g, status);
 }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -567,13 +575,6 @@ cudaError_t configure_gemv() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<r, w>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
     CFG(1, 4); CFG(2, 4); CFG(3, 4); CFG(4, 4); CFG(1, 8); CFG(2, 8); CFG(3, 8); CFG(4, 8);
 #undef CFG
-#define CFG1(w, ep, n) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<1, w, true, e_##ep, n>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemv_kernel<1, w, true, e_##ep, n>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
-    constexpr int e_STORE = EPI_STORE, e_RESID = EPI_RESID, e_SWIGLU = EPI_SWIGLU;
-    CFG1(4, STORE, 1); CFG1(8, STORE, 1); CFG1(4, STORE, 0); CFG1(8, STORE, 0);
-    CFG1(4, RESID, 1); CFG1(8, RESID, 1); CFG1(4, RESID, 0); CFG1(8, RESID, 0);
-    CFG1(4, SWIGLU, 1); CFG1(8, SWIGLU, 1); CFG1(4, SWIGLU, 0); CFG1(8, SWIGLU, 0);
-#undef CFG1
 #define CFGM(n, ep, nm) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, ep, nm>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, ep, nm>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
 #define CFGM6(n) CFGM(n, EPI_STORE, 1); CFGM(n, EPI_STORE, 0); CFGM(n, EPI_RESID, 1); CFGM(n, EPI_RESID, 0); CFGM(n, EPI_SWIGLU, 1); CFGM(n, EPI_SWIGLU, 0)
@@ -586,7 +587,7 @@ cudaError_t configure_gemv() {
 // Launches the projection.  a.max_oparts > 1 allows a K split for the residual epilogue; the number
 // of parts written is returned in *oparts (1 for the other epilogues).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts) {
-    // One activation row: the CUDA-core kernel.  2..16 rows: the tensor-core kernel.  More rows go in several
+    // One to three activation rows: the CUDA-core kernel.  4..16 rows: the tensor-core kernel.  More rows go in several
     // launches (the weights are streamed again for each).  g_hs_gemm_mma = false sends everything through the
     // CUDA-core kernel (passes of at most four rows over resident tiles; four rows per launch when a K range
     // needs more than one chunk).
@@ -603,7 +604,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         }
         return cudaSuccess;
     };
-    const bool mma = g_hs_gemm_mma && a.nrows >= 2;
+    const bool mma = g_hs_gemm_mma && a.nrows >= 4;       // up to three rows the pruned FMA instances are faster
     if (a.nrows > GV_MAXROWS && g_hs_gemm_tc && a.xb) return launch_gemm_tc(a, status, s, launches, oparts);   // a dense contraction: tcgen05
     if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     if (!mma && a.nrows > 4) {
@@ -668,14 +669,17 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
     if (launches) ++*launches;
     if (mma) return NG == 1 ? launch_mma<1>(a, g, smem, status, s) : launch_mma<2>(a, g, smem, status, s);
-    if (a.nrows == 1 && g.S1 == 0) {
-        // the draft step's projections: the pruned single-row instances
+    if (a.nrows <= 3) {
+        // one to three rows: the pruned instances (rows, tile height, epilogue, norm fixed at compile time)
         const int nm = a.norm_w ? 1 : 0;
-#define ONE(w, ep, n) if (WR == w && a.epi == ep && nm == n) return launch_one<w, ep, n>(a, g, smem, status, s)
-        ONE(4, EPI_STORE, 1); ONE(8, EPI_STORE, 1); ONE(4, EPI_STORE, 0); ONE(8, EPI_STORE, 0);
-        ONE(4, EPI_RESID, 1); ONE(8, EPI_RESID, 1); ONE(4, EPI_RESID, 0); ONE(8, EPI_RESID, 0);
-        ONE(4, EPI_SWIGLU, 1); ONE(8, EPI_SWIGLU, 1); ONE(4, EPI_SWIGLU, 0); ONE(8, EPI_SWIGLU, 0);
-#undef ONE
+#define LEAN(r, w, ep, n) if (a.nrows == r && WR == w && a.epi == ep && nm == n) {                                         \
+        if (ep == EPI_RESID && g.S1 > 0) return launch_lean<r, w, ep, n, ep == EPI_RESID>(a, g, smem, status, s);          \
+        if (g.S1 == 0) return launch_lean<r, w, ep, n, false>(a, g, smem, status, s); }
+#define LEAN6(r, w) LEAN(r, w, EPI_STORE, 1); LEAN(r, w, EPI_STORE, 0); LEAN(r, w, EPI_RESID, 1); LEAN(r, w, EPI_RESID, 0); \
+                    LEAN(r, w, EPI_SWIGLU, 1); LEAN(r, w, EPI_SWIGLU, 0)
+        LEAN6(1, 4); LEAN6(1, 8); LEAN6(2, 4); LEAN6(2, 8); LEAN6(3, 4); LEAN6(3, 8);
+#undef LEAN6
+#undef LEAN
     }
     // rows held in registers per pass: as even as possible over ceil(nrows / 4) passes
     const int npass = ceil_div(a.nrows, 4), R = ceil_div(a.nrows, npass);
