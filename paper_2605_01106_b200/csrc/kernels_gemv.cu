@@ -71,6 +71,7 @@ __device__ __forceinline__ int xs_pos(int c) {
 // SEG = false: the instance knows there is no second weight segment.
 template <int R, int WR, bool ONE = false, int EPI = -1, int NORMED = -1, bool SEG = true>
 __global__ void __launch_bounds__(GV_THREADS, 2) gemv_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
+    static_assert(WR * R <= 32, "a warp reduces at most 32 values");
     constexpr int NV = pow2_ge(WR * R);
     constexpr int LPV = 32 / NV;
     extern __shared__ __align__(128) unsigned char smraw[];
@@ -604,7 +605,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         }
         return cudaSuccess;
     };
-    const bool mma = g_hs_gemm_mma && a.nrows >= 4;       // up to three rows the pruned FMA instances are faster
+    const bool mma = g_hs_gemm_mma && a.nrows >= 4;       // measured: up to three rows the pruned FMA instances are faster
     if (a.nrows > GV_MAXROWS && g_hs_gemm_tc && a.xb) return launch_gemm_tc(a, status, s, launches, oparts);   // a dense contraction: tcgen05
     if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     if (!mma && a.nrows > 4) {
