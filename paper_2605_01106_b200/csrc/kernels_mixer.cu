@@ -22,11 +22,16 @@ __global__ void __launch_bounds__(SSM_THREADS) ssm_kernel(const SsmArgs a) {
 // ------------------------------------------------------------------------------------------------
 constexpr int GDN_THREADS = 256;   // 8 warps x 8 value rows; key dim 64 = 32 lanes x 2
 
-__global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
+// TMAX: most positions this instance handles (1 for the draft step, 3 for verify at k <= 2, else the maximum).
+// Everything the block needs from the in-projection - the raw conv inputs of a thread's own channel for all
+// positions, the gate inputs, the decay / write-strength inputs - is requested right after the wait, before the
+// first value is used: one trip to L2 for the whole kernel.
+template <int TMAX>
+__global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
     constexpr int DK = 64, RPW = 8;
-    __shared__ __align__(16) float qs[HS_MAX_T][DK], ks[HS_MAX_T][DK];
-    __shared__ float vs[HS_MAX_T][64], os[HS_MAX_T][64], al[HS_MAX_T], be[HS_MAX_T];
-    const int h = blockIdx.x, lb = blockIdx.y, b = a.b0 + lb, T = a.T, dv = a.dv;
+    __shared__ __align__(16) float qs[TMAX][DK], ks[TMAX][DK];
+    __shared__ float vs[TMAX][64], os[TMAX][64], zs[TMAX][64], al[TMAX], be[TMAX];
+    const int h = blockIdx.x, lb = blockIdx.y, b = a.b0 + lb, T = TMAX == 1 ? 1 : a.T, dv = a.dv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, rowbase = lb * T;
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
     const int nk = a.gh * DK, nv = a.gh * dv;
@@ -36,40 +41,65 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
     float s[RPW][2];
     const bool rows_ok = warp * RPW < dv;
     // before the wait the state is only pulled towards L2 (it was written by an earlier kernel); it is loaded
-    // after the wait, so this kernel may start as early as its predecessor allows
+    // after the wait, so this kernel may start as early as its predecessor allows.  Conv parameters are weights.
     if (rows_ok)
 #pragma unroll
         for (int r = 0; r < RPW; ++r) asm volatile("prefetch.global.L2 [%0];" :: "l"(sin_ + (warp * RPW + r) * DK + 2 * lane));
+    const int c = threadIdx.x;                        // this thread's channel of the head's q | k | v set
+    const bool chan = c < 2 * DK + dv;
+    const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
+    float4 tap = make_float4(0.f, 0.f, 0.f, 0.f);
+    float bias = 0.f;
+    if (chan) { tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc); bias = a.conv_b[gc]; }
     pdl_wait();
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
         float2 t = rows_ok ? __ldcg(reinterpret_cast<const float2 *>(sin_ + (warp * RPW + r) * DK + 2 * lane)) : make_float2(0.f, 0.f);
         s[r][0] = t.x; s[r][1] = t.y;
     }
-    // conv + SiLU on this head's q, k, v channels
-    for (int c = threadIdx.x; c < 2 * DK + dv; c += GDN_THREADS) {
-        const int gc = c < DK ? h * DK + c : c < 2 * DK ? nk + h * DK + (c - DK) : 2 * nk + h * dv + (c - 2 * DK);
-        const float4 tap = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
-        const float bias = a.conv_b[gc];
+    float w0 = 0.f, w1 = 0.f, w2 = 0.f, raw[TMAX];
+    if (chan) {
         const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
-        float w0 = __ldcg(win), w1 = __ldcg(win + a.convd), w2 = __ldcg(win + 2 * a.convd);
-        for (int i = 0; i < T; ++i) {
-            const float raw = __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + gc);
-            const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * raw);
-            w0 = w1; w1 = w2; w2 = raw;
-            if (c < DK) qs[i][c] = act; else if (c < 2 * DK) ks[i][c - DK] = act; else vs[i][c - 2 * DK] = act;
-            if (a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = raw;
+        w0 = __ldcg(win); w1 = __ldcg(win + a.convd); w2 = __ldcg(win + 2 * a.convd);
+    }
+#pragma unroll
+    for (int i = 0; i < TMAX; ++i) raw[i] = (chan && i < T) ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + gc) : 0.f;
+    constexpr int ZPT = (TMAX * 64 + GDN_THREADS - 1) / GDN_THREADS;
+    float zraw[ZPT];
+#pragma unroll
+    for (int u = 0; u < ZPT; ++u) {
+        const int idx = threadIdx.x + u * GDN_THREADS, i = idx >> 6, j = idx & 63;
+        zraw[u] = (i < T && j < dv) ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + 2 * nk + nv + h * dv + j) : 0.f;
+    }
+    float araw = 0.f, braw = 0.f;
+    if (threadIdx.x < T) {
+        const float *row = a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld;
+        araw = __ldcg(row + 2 * nk + 2 * nv + h);
+        braw = __ldcg(row + 2 * nk + 2 * nv + a.gh + h);
+    }
+    // conv + SiLU on this head's q, k, v channels, in registers
+    if (chan) {
+#pragma unroll
+        for (int i = 0; i < TMAX; ++i) {
+            if (i < T) {
+                const float r = raw[i];
+                const float act = silu_f(bias + tap.x * w0 + tap.y * w1 + tap.z * w2 + tap.w * r);
+                w0 = w1; w1 = w2; w2 = r;
+                if (c < DK) qs[i][c] = act; else if (c < 2 * DK) ks[i][c - DK] = act; else vs[i][c - 2 * DK] = act;
+                if (a.hist) a.hist[((size_t)b * a.Tm + i) * a.convd + gc] = r;
+            }
         }
         if (a.win_out) {
             float *wo = a.win_out + (size_t)b * 3 * a.convd + gc;
             wo[0] = w0; wo[a.convd] = w1; wo[2 * a.convd] = w2;
         }
     }
-    if (threadIdx.x < T) {
-        const float *row = a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld;
-        al[threadIdx.x] = sigmoid_f(__ldcg(row + 2 * nk + 2 * nv + h));
-        be[threadIdx.x] = sigmoid_f(__ldcg(row + 2 * nk + 2 * nv + a.gh + h));
+#pragma unroll
+    for (int u = 0; u < ZPT; ++u) {
+        const int idx = threadIdx.x + u * GDN_THREADS, i = idx >> 6, j = idx & 63;
+        if (i < T && j < dv) zs[i][j] = silu_f(zraw[u]);
     }
+    if (threadIdx.x < T) { al[threadIdx.x] = sigmoid_f(araw); be[threadIdx.x] = sigmoid_f(braw); }
     __syncthreads();
     // L2-normalise q and k of every position (one warp per vector)
     for (int t = warp; t < 2 * T; t += GDN_THREADS / 32) {
@@ -114,11 +144,8 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(GdnArgs a) {
         float ss = 0.f;
         for (int j = lane; j < dv; j += 32) ss = fmaf(os[i][j], os[i][j], ss);
         const float rstd = rsqrtf(warp_sum(ss) / (float)dv + a.eps);
-        const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
-        for (int j = lane; j < dv; j += 32) {
-            const float z = __ldcg(row + 2 * nk + nv + h * dv + j);
-            a.g[(size_t)(rowbase + i) * nv + h * dv + j] = os[i][j] * rstd * a.onorm[j] * silu_f(z);
-        }
+        for (int j = lane; j < dv; j += 32)
+            a.g[(size_t)(rowbase + i) * nv + h * dv + j] = os[i][j] * rstd * a.onorm[j] * zs[i][j];
     }
 }
 
@@ -142,5 +169,8 @@ cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s) {
 
 cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s) {
     if (a.dk != 64 || a.dv > 64 || (a.dv & 7)) return cudaErrorInvalidValue;
-    return launch_pdl(gdn_kernel, dim3(a.gh, a.nb), dim3(GDN_THREADS), 0, s, a);
+    const dim3 grid(a.gh, a.nb), block(GDN_THREADS);
+    if (a.T == 1) return launch_pdl(gdn_kernel<1>, grid, block, 0, s, a);
+    if (a.T <= 3) return launch_pdl(gdn_kernel<3>, grid, block, 0, s, a);
+    return launch_pdl(gdn_kernel<HS_MAX_T>, grid, block, 0, s, a);
 }
