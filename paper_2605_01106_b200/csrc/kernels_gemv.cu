@@ -391,13 +391,16 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
         const int ldx = seg1 ? a.ldx1 : a.ldx0;
         const int parts = seg1 ? 1 : a.xparts;
         const int c_lo = normed ? 0 : k0, c_hi = normed ? Kseg : k0 + kr;
+        constexpr int SR = 5;               // rows per sweep: k = 4 (five rows) is staged in one trip to L2
 #pragma unroll 1
-        for (int rbase = 0; rbase < nrows; rbase += 4) {
-            float ss[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
-                float4 v[4];
+        for (int rbase = 0; rbase < nrows; rbase += SR) {
+            float ss[SR];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {              // all loads of the four rows are in flight together
+            for (int j = 0; j < SR; ++j) ss[j] = 0.f;
+            for (int c = c_lo + tid * 4; c < c_hi; c += GV_THREADS * 4) {
+                float4 v[SR];
+#pragma unroll
+                for (int j = 0; j < SR; ++j) {             // all loads of the rows of a sweep are in flight together
                     v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (rbase + j < nrows) {
                         const float *p = xsrc + (size_t)(rbase + j) * ldx + c;
@@ -415,7 +418,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
                 float4 nw = make_float4(1.f, 1.f, 1.f, 1.f);
                 if (normed && inside) nw = *reinterpret_cast<const float4 *>(nw_s + (c - k0));
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SR; ++j) {
                     const int r = rbase + j;
                     if (r >= nrows) continue;
                     ss[j] = fmaf(v[j].x, v[j].x, fmaf(v[j].y, v[j].y, fmaf(v[j].z, v[j].z, fmaf(v[j].w, v[j].w, ss[j]))));
@@ -434,7 +437,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
             }
             if (normed) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SR; ++j) {
                     const float t = warp_sum(ss[j]);
                     if (lane == 0 && rbase + j < nrows) ss_s[warp * GV_MAXROWS + rbase + j] = t;
                 }
