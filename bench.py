@@ -297,7 +297,9 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": bytes_per_launch,
                 "isolated": {"avg_launch_us": 1e3 * g_ms / max(g_n, 1), "GBps": achieved_iso,
                              "note": "every launch bracketed by two events: no overlap with neighbours, event cost included"},
-                "time_share": {kk: v[0] / tot_iso for kk, v in prof.items()} if tot_iso > 0 else {}}
+                "time_share": {kk: v[0] / tot_iso for kk, v in prof.items()} if tot_iso > 0 else {},
+                "time_share_note": "in parallel hybrid blocks the verify attention runs inside the fused mixer launch "
+                                   "and is counted under 'mixer'"}
 
     if rank != 0:
         return
