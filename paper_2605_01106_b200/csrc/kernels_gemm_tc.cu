@@ -10,7 +10,7 @@
 // One elected thread issues the TMA copies, one issues tcgen05.mma (K = 16 per instruction, four per 64-column
 // stage) and releases stages with tcgen05.commit; all eight warps run the epilogue (thread = weight row, two
 // warps per lane quarter, each half of the columns).  Every wait is bounded.
-// No multicast: every CTA fetches its own tiles.
+// Every CTA fetches its own tiles (no copy is shared between CTAs).
 // The weights are the large operand, so the grid is filled by splitting K, not N: the CTAs of a thread-block
 // cluster (up to 8) take consecutive K ranges of the same tile, leave their fp32 partial tiles in shared
 // memory and add them up, in rank order, through distributed shared memory - every weight byte is fetched
