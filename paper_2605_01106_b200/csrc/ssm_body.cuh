@@ -49,15 +49,27 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
     const bool owner = (bx == 0 && by == 0);   // writes the shared B|C channels' history
     float4 tap[CPT];
     float bias[CPT], w0[CPT], w1[CPT], w2[CPT];
+    // addresses of everything read after the wait are formed here, so that the loads go out back to back
+    const float *raw_p[CPT], *win_p[CPT];
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
         const int c = threadIdx.x + q * SSM_THREADS;
+        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
+        raw_p[q] = a.zx + (size_t)rowbase * a.in_ld + a.di + gc;
+        win_p[q] = a.win_in + (size_t)b * 3 * a.convd + gc;
         if (c < NCH) {
-            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
             tap[q] = *reinterpret_cast<const float4 *>(a.conv_w + 4 * gc);
             bias[q] = a.conv_b[gc];
         }
     }
+    constexpr int ZPT = (TMAX * SSM_PR + SSM_THREADS - 1) / SSM_THREADS;
+    const float *z_p[ZPT];
+#pragma unroll
+    for (int u = 0; u < ZPT; ++u) {
+        const int idx = threadIdx.x + u * SSM_THREADS, i = idx / SSM_PR, c = idx - i * SSM_PR;
+        z_p[u] = a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c;
+    }
+    const float *dt_p = a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h;
     const float Aexp = expf(a.A_log[h]), dtb = a.dt_bias[h], Dh = a.D[h];
     pdl_wait();
 
@@ -73,11 +85,7 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
         const int c = threadIdx.x + q * SSM_THREADS;
-        if (c < NCH) {
-            const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
-            const float *win = a.win_in + (size_t)b * 3 * a.convd + gc;
-            w0[q] = __ldcg(win); w1[q] = __ldcg(win + a.convd); w2[q] = __ldcg(win + 2 * a.convd);
-        }
+        if (c < NCH) { w0[q] = __ldcg(win_p[q]); w1[q] = __ldcg(win_p[q] + a.convd); w2[q] = __ldcg(win_p[q] + 2 * a.convd); }
     }
     // ---- raw conv inputs of this thread's own channels for all T positions, gate inputs and dt: every load is
     //      issued before the first value is used, so the whole phase costs one trip to L2
@@ -85,19 +93,15 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
         const int c = threadIdx.x + q * SSM_THREADS;
-        const int gc = c < SSM_PR ? h * a.P + p0 + c : a.di + (c - SSM_PR);
 #pragma unroll
         for (int i = 0; i < TMAX; ++i)
-            raw[q][i] = (c < NCH && i < T) ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + a.di + gc) : 0.f;
+            raw[q][i] = (c < NCH && i < T) ? __ldcg(raw_p[q] + (size_t)i * a.in_ld) : 0.f;
     }
-    constexpr int ZPT = (TMAX * SSM_PR + SSM_THREADS - 1) / SSM_THREADS;
     float zraw[ZPT];
 #pragma unroll
-    for (int u = 0; u < ZPT; ++u) {
-        const int idx = threadIdx.x + u * SSM_THREADS, i = idx / SSM_PR, c = idx - i * SSM_PR;
-        zraw[u] = idx < T * SSM_PR ? __ldcg(a.zx + (size_t)(rowbase + i) * a.in_ld + h * a.P + p0 + c) : 0.f;
-    }
-    const float dtraw = threadIdx.x < T ? __ldcg(a.zx + (size_t)(rowbase + threadIdx.x) * a.in_ld + a.di + a.convd + h) : 0.f;
+    for (int u = 0; u < ZPT; ++u)
+        zraw[u] = threadIdx.x + u * SSM_THREADS < T * SSM_PR ? __ldcg(z_p[u]) : 0.f;
+    const float dtraw = threadIdx.x < T ? __ldcg(dt_p) : 0.f;
     // ---- causal conv + SiLU in registers (a thread walks the positions of its channels); results to shared memory
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
