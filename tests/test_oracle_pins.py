@@ -449,3 +449,94 @@ def test_gdn_layer_first_token_closed_form(tseq):
     q = oracle.Model(s1, b1, table, 8).new_seq()
     np.testing.assert_allclose(q.step(tok, mode=1), want, rtol=1e-9, atol=1e-11)
     np.testing.assert_allclose(q.gdn()[0], beta[:, None, None] * vv[:, :, None] * kn[:, None, :], rtol=1e-10, atol=1e-14)
+
+
+def test_second_token_ssm_decay_closed_form(tiny):
+    # two tokens through one parallel layer from zero state, attention and MLP silenced.  The second token is the
+    # first one whose state update has a non-zero previous state, so it is the one that fixes the decay term of the
+    # Mamba-2 recurrence inside the layer: S_2 = exp(dt_2 * (-exp(A_log_h))) S_1 + dt_2 x_2 (x) B_2 per head h -
+    # the sign, the exponential and the head index of A_log - and the conv window carrying the first raw input.
+    s, blob, table = tiny
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_O)[:] = 0
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    di, N, H, P = s.d_inner, s.N, s.H, s.P
+    E = _f(b1, table, -1, hi.G_EMBED)
+    Win = _f(b1, table, 0, hi.T_W_IN)
+    w1, wg = _f(b1, table, 0, hi.T_NORM1), _f(b1, table, 0, hi.T_GNORM)
+    cw, cb = _f(b1, table, 0, hi.T_CONV_W), _f(b1, table, 0, hi.T_CONV_B)
+    A_log, D, dtb = _f(b1, table, 0, hi.T_A_LOG), _f(b1, table, 0, hi.T_D), _f(b1, table, 0, hi.T_DT_BIAS)
+    Wout, Wlm, wf = _f(b1, table, 0, hi.T_W_OUT), _f(b1, table, -1, hi.G_LM_HEAD), _f(b1, table, -1, hi.G_FINAL_NORM)
+    assert len(set(np.round(A_log, 6))) == H              # distinct per head: a wrong head index cannot hide
+    toks = (123, 3001)
+    raws, S, want_logits = [], np.zeros((H, P, N)), None
+    for t, tok in enumerate(toks):
+        u = _rms(E[tok], w1, s.eps)
+        z, xbc, dtr = Win[:di] @ u, Win[di:2 * di + 2 * N] @ u, Win[2 * di + 2 * N: 2 * di + 2 * N + H] @ u
+        raws.append(xbc)
+        pre = cb + cw[:, 3] * raws[t] + (cw[:, 2] * raws[t - 1] if t >= 1 else 0.0)   # taps 0, 1 still see zeros
+        act = pre / (1 + np.exp(-pre))
+        x, B, C = act[:di].reshape(H, P), act[di:di + N], act[di + N:]
+        dt = np.log1p(np.exp(dtr + dtb))
+        decay = np.exp(dt * -np.exp(A_log))                                           # one scalar per head
+        S = decay[:, None, None] * S + dt[:, None, None] * x[:, :, None] * B[None, None, :]
+        y = (S @ C + D[:, None] * x).reshape(-1)
+        g = y * (z / (1 + np.exp(-z)))
+        h = E[tok] + Wout @ _rms(g, wg, s.eps)
+        want_logits = Wlm @ _rms(h, wf, s.eps)
+    q = oracle.Model(s1, b1, table, 8).new_seq()
+    q.step(toks[0], mode=1)
+    got = q.step(toks[1], mode=1)
+    np.testing.assert_allclose(q.ssm()[0], S, rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(got, want_logits, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(q.conv()[0, 1:], np.stack(raws), rtol=1e-12)
+    # the pin has teeth: the decay moves the state by far more than the tolerance (a dropped or mis-signed A would fail)
+    no_decay = S / decay[:, None, None]
+    assert np.abs(no_decay - S).max() > 1e-3 * np.abs(S).max()
+
+
+def test_second_token_gdn_alpha_closed_form(tseq):
+    # two tokens through one Gated DeltaNet layer from zero state, MLP silenced.  From a zero state the decay gate
+    # alpha never acts; the second token fixes alpha = sigmoid(W_a u) with its own row block of the in-projection:
+    # S_2 = alpha_2 S_1 + beta_2 (v_2 - alpha_2 S_1 k_2) k_2^T ,  o_2 = S_2 q_2 / sqrt(d_k)
+    s, blob, table = tseq
+    s1 = s.replace(L=1)
+    b1 = blob.copy()
+    hi.tensor_view(b1, table, 0, hi.T_W_DOWN)[:] = 0
+    nk, nv, gh, dk, dv = s.gh * s.gdk, s.gh * s.gdv, s.gh, s.gdk, s.gdv
+    E = _f(b1, table, -1, hi.G_EMBED)
+    Win = _f(b1, table, 0, hi.T_W_IN)
+    w1, wn = _f(b1, table, 0, hi.T_NORM1), _f(b1, table, 0, hi.T_GNORM)
+    cw, cb = _f(b1, table, 0, hi.T_CONV_W), _f(b1, table, 0, hi.T_CONV_B)
+    Wout, Wlm, wf = _f(b1, table, 0, hi.T_W_OUT), _f(b1, table, -1, hi.G_LM_HEAD), _f(b1, table, -1, hi.G_FINAL_NORM)
+    toks = (99, 1500)
+    raws, S, want_logits, alphas = [], np.zeros((gh, dv, dk)), None, None
+    for t, tok in enumerate(toks):
+        u = _rms(E[tok], w1, s.eps)
+        raw = Win[:2 * nk + nv] @ u
+        z = Win[2 * nk + nv:2 * nk + 2 * nv] @ u
+        ga = Win[2 * nk + 2 * nv:2 * nk + 2 * nv + gh] @ u          # decay-gate rows come before the beta rows
+        gb = Win[2 * nk + 2 * nv + gh:2 * nk + 2 * nv + 2 * gh] @ u
+        raws.append(raw)
+        pre = cb + cw[:, 3] * raws[t] + (cw[:, 2] * raws[t - 1] if t >= 1 else 0.0)
+        act = pre / (1 + np.exp(-pre))
+        qv, kv, vv = act[:nk].reshape(gh, dk), act[nk:2 * nk].reshape(gh, dk), act[2 * nk:].reshape(gh, dv)
+        qn = qv / np.sqrt((qv * qv).sum(1, keepdims=True) + 1e-6)
+        kn = kv / np.sqrt((kv * kv).sum(1, keepdims=True) + 1e-6)
+        alphas, beta = 1 / (1 + np.exp(-ga)), 1 / (1 + np.exp(-gb))
+        o = np.empty((gh, dv))
+        for h in range(gh):
+            Sd = alphas[h] * S[h]
+            S[h] = Sd + beta[h] * np.outer(vv[h] - Sd @ kn[h], kn[h])
+            o[h] = S[h] @ qn[h] / np.sqrt(dk)
+        o = np.stack([_rms(o[h], wn, s.eps) for h in range(gh)]) * (z / (1 + np.exp(-z))).reshape(gh, dv)
+        h1 = E[tok] + Wout @ o.reshape(-1)
+        want_logits = Wlm @ _rms(h1, wf, s.eps)
+    q = oracle.Model(s1, b1, table, 8).new_seq()
+    q.step(toks[0], mode=1)
+    got = q.step(toks[1], mode=1)
+    np.testing.assert_allclose(q.gdn()[0], S, rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(got, want_logits, rtol=1e-9, atol=1e-11)
+    # alpha acts visibly: with alpha = 1 (no decay) or with the beta rows used for alpha the state would differ
+    assert np.abs(alphas - 1.0).min() > 1e-3 and len(set(np.round(alphas, 6))) == gh
