@@ -177,7 +177,7 @@ class ModelShape:
 
 
 CONFIGS = {
-    # the five workloads, in the order the benchmark description lists them
+    # the five workloads (tiny, 0.5B-class, 3B-class, sequential, batch-64 long context)
     "cfg1_tiny": ModelShape("cfg1_tiny", ARCH_PARALLEL, L=2, d=256, V=4096, H=8, P=64, N=64,
                             qh=4, kvh=2, hd=64, ff=1024, batch=1, prompt_len=64, gen_tokens=32, ks=(2,)),
     "cfg2_0p5b": ModelShape("cfg2_0p5b", ARCH_PARALLEL, L=36, d=1024, V=32768, H=32, P=64, N=128,

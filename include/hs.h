@@ -112,36 +112,51 @@ enum { HS_G_EMBED = 0, HS_G_LM_HEAD = 1, HS_G_FINAL_NORM = 2 };
 int hs_query_sizes(const hs_config *cfg, hs_sizes *out);
 int64_t hs_weight_offset(const hs_config *cfg, int layer, int tensor);
 
-/* Build the host handle.  Requirements: conv_w == 4; d, ff, di, qh*hd, gh*gdv multiples of 256;
+/* Build the host handle for one hybrid model (paper Sec. 3.1: Eq. 2 parallel block / Eq. 3 sequential stack)
+ * and its two modes (Sec. 3.2).  Requirements: conv_w == 4; d, ff, di, qh*hd, gh*gdv multiples of 256;
  * P and gdv multiples of 16; N in {64,128,256}; hd in {64,128}; gdk == 64; qh % kvh == 0;
- * (qh/kvh)*(max_k+1) <= 48; max_k <= 8.  Enqueues (on `stream`, a cudaStream_t) the RoPE table
- * upload and the zeroing of the control block; does not read the other buffers.
- * The weights must already be in `bufs->weights` in the blob format. */
-int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs_model **out);
+ * (qh/kvh)*(max_k+1) <= 48; max_k <= 8.
+ * bufs: the six DEVICE buffers (caller-owned, 256-byte aligned, alive until hs_destroy); have: the number of
+ * bytes the caller really provides in each of them - HS_ERR_SIZE if any is smaller than hs_query_sizes reports.
+ * The weights must already be in `bufs->weights` in the blob format.  Enqueues (on `stream`, a cudaStream_t)
+ * the RoPE table upload and the zeroing of the control block, and synchronises; does not read the other buffers.
+ * On any error *out is set to NULL and nothing is left to destroy. */
+int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, const hs_sizes *have, void *stream, hs_model **out);
 
 /* Zero every sequence: recurrent state, conv windows, kv_len = 0, no pending token.  Async. */
 int hs_reset(hs_model *m);
 
-/* Consume prompts with the full model (paper Sec. 3.3 prefix x_{1:t}).  tokens_host: the prompts
- * back to back (sequence b starts at sum(lens_host[0..b-1])); lens_host[b] >= 1.  Sets the batch
+/* Consume prompts with the full model (paper Sec. 3.3 prefix x_{1:t}; M_H of Eq. 2 / Eq. 3).  tokens_host: the
+ * prompts back to back (sequence b starts at sum(lens_host[0..b-1])); lens_host[b] >= 1; every id in [0, V),
+ * otherwise HS_ERR_INVALID_ARG before anything is enqueued.  Sets the batch
  * size for the following rounds.  Afterwards kv_len[b] = lens[b] and pending[b] = the greedy choice
  * after the last prompt token (generated token #1).  Runs as repeated verify passes over chunks of
  * max_k+1 tokens with every candidate accepted.  Synchronises the stream before returning. */
 int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host, int batch);
 
-/* Draft phase: k draft-mode steps for every sequence; candidates cand[b][0..k] = [pending, d_1..d_k]
- * stay on the device.  0 <= k <= max_k; k = 0 does nothing.  Async. */
+/* Draft phase (paper Sec. 3.3, "Draft phase": M_S generates k tokens autoregressively; M_S is Eq. 4 for a
+ * parallel hybrid - attention output zeroed - and Eq. 5 for a sequential one - attention layers are the
+ * identity): k draft-mode steps for every sequence on scratch state; candidates
+ * cand[b][0..k] = [pending, d_1..d_k] stay on the device; the KV cache and the committed state are not touched.
+ * 0 <= k <= max_k; k = 0 does nothing.  HS_ERR_ORDER between hs_verify and hs_accept_rollback.  Async. */
 int hs_draft(hs_model *m, int k);
 
-/* Verification phase over k+1 candidates per sequence at positions kv_len[b]..kv_len[b]+k.
+/* Verification phase (paper Sec. 3.3, "Verification phase": M_H, Eq. 2 / Eq. 3, processes the prefix and the
+ * drafts in a single forward pass; here incrementally from the cached state) over k+1 candidates per sequence
+ * at positions kv_len[b]..kv_len[b]+k.  k is passed explicitly so that k = 0 (plain autoregressive decoding,
+ * the denominator of Eq. 1) and caller-supplied candidates need no preceding draft.
  * cand_dev: NULL to verify the candidates of the preceding hs_draft(k) (HS_ERR_ORDER if there was
  * none with this k, except k = 0), or int32 [batch][k+1] candidates to verify instead (cand[b][0]
  * replaces the pending token).  Produces g[b][i] = argmax of the logits after candidate i
- * (lowest id on ties), the top-2 margin, state snapshots and KV rows.  Async.
- * HS_ERR_CAPACITY if a sequence could exceed kv_capacity. */
+ * (lowest id on ties), the top-2 margin, state snapshots and KV rows.  Ids in cand_dev outside [0, V) are
+ * not used as addresses: token 0 is read instead and the device status word becomes HS_ERR_DEVICE.  Async.
+ * HS_ERR_CAPACITY if a sequence could exceed kv_capacity; HS_ERR_ORDER if the previous hs_verify has not been
+ * followed by hs_accept_rollback (its snapshots still hold the verified positions). */
 int hs_verify(hs_model *m, int k, const int32_t *cand_dev);
 
-/* Greedy acceptance + rollback after hs_verify.  Per sequence: n = number of leading drafts with
+/* Greedy acceptance + rollback after hs_verify (paper Sec. 3.3: under greedy decoding draft i is accepted iff
+ * argmax P_S = argmax P_H at position i, and all tokens up to the first rejection are accepted; Eq. 1's
+ * numerator counts the k+1 tokens a fully accepted round emits).  Per sequence: n = number of leading drafts with
  * cand[i+1] == g[i]; emitted = cand[1..n], g[n]; committed state <- snapshot n; kv_len += n+1;
  * pending <- g[n].  forced_n_dev (int32 [batch] on the device, or NULL) overrides n (0 <= n <= k) with
  * everything else unchanged; forced_next_dev (int32 [batch], entries < 0 ignored, or NULL) overrides
@@ -150,9 +165,10 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev);
 int hs_accept_rollback(hs_model *m, const int32_t *forced_n_dev, const int32_t *forced_next_dev,
                        int32_t *n_acc_host, int32_t *emitted_host);
 
-/* One whole round with HOST buffers: uploads forced_n_host / forced_next_host (either may be NULL),
- * runs draft(k), verify(k), accept/rollback, downloads n_acc_host [batch] and
- * emitted_host [batch][k+1] (either may be NULL) and synchronises. */
+/* One whole round of paper Sec. 3.3 with HOST buffers: uploads forced_n_host / forced_next_host (either may be
+ * NULL), runs draft(k), verify(k), accept/rollback, downloads n_acc_host [batch] and emitted_host [batch][k+1]
+ * (either may be NULL) and synchronises.  HS_ERR_INVALID_ARG (nothing enqueued) if a forced accept length is
+ * outside [0, k] or a forced next token is >= V. */
 int hs_round_host(hs_model *m, int k, const int32_t *forced_n_host, const int32_t *forced_next_host,
                   int32_t *n_acc_host, int32_t *emitted_host);
 
@@ -194,6 +210,12 @@ int hs_profile(hs_model *m, int enable);
 int hs_profile_read(hs_model *m, double *ms, int64_t *launches, double *bytes);
 /* Device status word: 0, or the first hs_status a kernel recorded.  Synchronises. */
 int hs_device_status(hs_model *m);
+/* Puts the status word back to 0 (async, on the model's stream). */
+int hs_clear_status(hs_model *m);
+/* Self-test of the bounded device-side wait: enqueues a one-warp kernel that waits `polls` (1..2^20) times on an
+ * mbarrier nothing will ever complete, gives up and records HS_ERR_TIMEOUT, which hs_device_status then returns.
+ * The kernel ends by itself; the handle stays usable (hs_clear_status).  Async. */
+int hs_selftest_wait_timeout(hs_model *m, int polls);
 const char *hs_last_error(const hs_model *m);
 
 /* Greedy argmax for callers that cannot allocate device memory.  (The paper has no counterpart: this is
@@ -208,7 +230,10 @@ const char *hs_last_error(const hs_model *m);
  * inside the library; every GPU that loads libhs.so holds those 33 KB until the process ends.
  * Limits and rules:
  *  - rows <= 64, otherwise HS_ERR_SIZE and nothing is launched; V >= 1.  Bad pointers/sizes:
- *    HS_ERR_INVALID_ARG.  A failing CUDA call: HS_ERR_CUDA.
+ *    HS_ERR_INVALID_ARG - that includes alignment: logits_dev must be 16-byte aligned when V is a multiple of 4
+ *    (rows are then read 128 bits at a time; a view that starts inside a larger tensor may not be), 4-byte
+ *    aligned otherwise, token_dev and margin_dev 4-byte aligned.  A failing CUDA call: HS_ERR_CUDA.
+ *  - A row whose values are all -inf or NaN gets token 0 and margin 0.
  *  - The call allocates and frees nothing.  It is asynchronous on `stream` (a cudaStream_t).
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
  *    that device current; make that first call outside any stream capture.

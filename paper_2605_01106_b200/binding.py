@@ -19,7 +19,8 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_set_attn_geometry", "hs_profile", "hs_profile_read", "hs_device_status", "hs_last_error", "hs_destroy", "hs_argmax_static"]
+           "hs_set_attn_geometry", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
+           "hs_selftest_wait_timeout", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
 class HsError(RuntimeError):
@@ -55,7 +56,7 @@ def load_library(path: str | None = None):
     L.hs_query_sizes.argtypes = [cfgp, szp]
     L.hs_weight_offset.restype = i64
     L.hs_weight_offset.argtypes = [cfgp, ctypes.c_int, ctypes.c_int]
-    L.hs_init_model.argtypes = [cfgp, bufp, vp, ctypes.POINTER(vp)]
+    L.hs_init_model.argtypes = [cfgp, bufp, szp, vp, ctypes.POINTER(vp)]
     L.hs_reset.argtypes = [vp]
     L.hs_prefill.argtypes = [vp, vp, vp, ctypes.c_int]
     L.hs_draft.argtypes = [vp, ctypes.c_int]
@@ -75,6 +76,8 @@ def load_library(path: str | None = None):
     L.hs_profile.argtypes = [vp, ctypes.c_int]
     L.hs_profile_read.argtypes = [vp, vp, vp, vp]
     L.hs_device_status.argtypes = [vp]
+    L.hs_clear_status.argtypes = [vp]
+    L.hs_selftest_wait_timeout.argtypes = [vp, ctypes.c_int]
     L.hs_last_error.restype = ctypes.c_char_p
     L.hs_last_error.argtypes = [vp]
     L.hs_destroy.argtypes = [vp]
@@ -93,11 +96,20 @@ def argmax_static(logits_dev, tokens_dev, margins_dev=None, stream=None):
     Runs on `stream` (torch stream) or torch's current stream; raises HsError on a non-zero status."""
     import torch
     rows, V = logits_dev.shape
-    st = stream or torch.cuda.current_stream(logits_dev.device)
+    dev = logits_dev.device
+    # the C entry point sees raw pointers only: what they point at is checked here, before anything is launched
+    if logits_dev.dtype != torch.float32 or not logits_dev.is_contiguous() or not logits_dev.is_cuda:
+        raise HsError(-1, "hs_argmax_static: logits must be a contiguous float32 CUDA tensor")
+    if tokens_dev.dtype != torch.int32 or not tokens_dev.is_contiguous() or tokens_dev.device != dev or tokens_dev.numel() != rows:
+        raise HsError(-1, "hs_argmax_static: tokens must be a contiguous int32 tensor of `rows` elements on the logits' device")
+    if margins_dev is not None and (margins_dev.dtype != torch.float32 or not margins_dev.is_contiguous()
+                                    or margins_dev.device != dev or margins_dev.numel() != rows):
+        raise HsError(-1, "hs_argmax_static: margins must be a contiguous float32 tensor of `rows` elements on the logits' device")
+    st = stream or torch.cuda.current_stream(dev)
     rc = lib().hs_argmax_static(logits_dev.data_ptr(), int(V), int(rows), tokens_dev.data_ptr(),
                                 margins_dev.data_ptr() if margins_dev is not None else None, vp(st.cuda_stream))
     if rc != 0:
-        raise HsError(rc, "hs_argmax_static: %s" % {-1: "invalid argument", -2: "more than 64 rows", -5: "CUDA error"}.get(rc, "error"))
+        raise HsError(rc, "hs_argmax_static: %s" % {-1: "invalid argument (null, misaligned or empty)", -2: "more than 64 rows", -5: "CUDA error"}.get(rc, "error"))
 
 
 def make_config(shape, max_batch=1, max_k=8, kv_capacity=1024, flags=0) -> HsConfig:
@@ -131,6 +143,9 @@ class Engine:
     All methods mirror the C entry points; device-side results stay on the device unless a method
     says it returns host data."""
 
+    GUARD = 4096          # bytes of guard pattern kept behind every buffer handed to the library
+    GUARD_BYTE = 0xA5
+
     def __init__(self, shape, weights: np.ndarray, max_batch=1, max_k=8, kv_capacity=1024, flags=0,
                  device="cuda:0", stream=None):
         import torch
@@ -144,14 +159,25 @@ class Engine:
         torch.cuda.set_device(self.device)
         # a stream of its own: the legacy default stream cannot be captured into a CUDA graph
         self.stream = stream or torch.cuda.Stream(self.device)
-        alloc = lambda n, zero: (torch.zeros if zero else torch.empty)(max(int(n), 256), dtype=torch.uint8, device=self.device)
-        self.t_weights = torch.from_numpy(weights).to(self.device)
-        self.t_snap, self.t_dstate, self.t_conv = alloc(self.sizes.snap, True), alloc(self.sizes.dstate, True), alloc(self.sizes.conv, True)
-        self.t_kv, self.t_work = alloc(self.sizes.kv, True), alloc(self.sizes.work, True)
-        self.bufs = HsBuffers(*[t.data_ptr() for t in (self.t_weights, self.t_snap, self.t_dstate, self.t_conv, self.t_kv, self.t_work)])
+
+        def alloc(n):
+            # the library is told about n bytes; a guard pattern sits right behind them (see check_guards)
+            n = max(int(n), 256)
+            t = torch.zeros(n + self.GUARD, dtype=torch.uint8, device=self.device)
+            t[n:] = self.GUARD_BYTE
+            return t
+
+        self.t_weights = alloc(self.sizes.weights)
+        self.t_weights[:weights.nbytes].copy_(torch.from_numpy(weights))
+        self.t_snap, self.t_dstate, self.t_conv = alloc(self.sizes.snap), alloc(self.sizes.dstate), alloc(self.sizes.conv)
+        self.t_kv, self.t_work = alloc(self.sizes.kv), alloc(self.sizes.work)
+        self._guarded = (self.t_weights, self.t_snap, self.t_dstate, self.t_conv, self.t_kv, self.t_work)
+        self.bufs = HsBuffers(*[t.data_ptr() for t in self._guarded])
+        have = HsSizes(*[t.numel() - self.GUARD for t in self._guarded])
         torch.cuda.synchronize(self.device)
         self.h = vp()
-        rc = lib().hs_init_model(ctypes.byref(self.cfg), ctypes.byref(self.bufs), vp(self.stream.cuda_stream), ctypes.byref(self.h))
+        rc = lib().hs_init_model(ctypes.byref(self.cfg), ctypes.byref(self.bufs), ctypes.byref(have),
+                                 vp(self.stream.cuda_stream), ctypes.byref(self.h))
         if rc != 0:
             raise HsError(rc, "hs_init_model failed")
         self.max_k, self.max_batch = max_k, max_batch
@@ -300,3 +326,14 @@ class Engine:
 
     def device_status(self):
         return lib().hs_device_status(self.h)
+
+    def clear_status(self):
+        self._ck(lib().hs_clear_status(self.h))
+
+    def selftest_wait_timeout(self, polls=1000):
+        self._ck(lib().hs_selftest_wait_timeout(self.h, int(polls)))
+
+    def check_guards(self):
+        """True if the guard bytes behind every buffer the library was given are untouched (synchronises)."""
+        self.torch.cuda.synchronize(self.device)
+        return all(bool((t[t.numel() - self.GUARD:] == self.GUARD_BYTE).all().item()) for t in self._guarded)

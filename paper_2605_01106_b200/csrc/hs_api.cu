@@ -209,7 +209,9 @@ AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
     return g;
 }
 
-int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
+// first = true: this pass opens an API call (its predecessor in the stream may be the accept kernel of the last
+// round): its first kernel goes out in plain stream order, see hs_device.cuh.
+int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool first) {
     const hs_config &c = m->c;
     const AttnGeom at_geom = draft ? AttnGeom{m->att_chunk, 1} : attn_geom(m, T, b0, nb);
     cudaStream_t s = m->stream;
@@ -220,7 +222,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
     int cur = 0, hparts = 1;
     const int64_t hps = (int64_t)m->B * m->Tm * d;
     int32_t *st_w = m->ctrl.status;
-    PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->hbuf[0], s), "embed");
+    PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, c.V, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->hbuf[0], st_w, first, s), "embed");
     ++m->launches;
     for (int l = 0; l < c.L; ++l) {
         const HsLayer &ly = m->layers[l];
@@ -232,8 +234,6 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
         ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->hbuf[cur]; ga.ldx0 = d; ga.xparts = hparts; ga.xpstride = hps;
         ga.norm_w = ly.norm1; ga.eps = c.eps;
         ga.O = inr; ga.out = m->zx; ga.ldo = m->in_rows_max; ga.nrows = rows; ga.epi = EPI_STORE;
-        // the mixer that follows reads its recurrent state before its own wait: keep it from starting
-        // until this kernel has waited, i.e. until everything older is complete
         ga.early_trigger = 1;
         ga.pf_ptr = ly.type == HS_LAYER_ATT ? ly.W_o : ly.W_out;
         ga.pf_bytes = 2 * (int64_t)d * (ly.type == HS_LAYER_ATT ? c.qh * c.hd : m->gw);
@@ -358,13 +358,13 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb) {
 }
 
 int enqueue_draft(hs_model *m, int k, int b0, int nb) {
-    for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb); if (rc) return rc; }
+    for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb, st == 0); if (rc) return rc; }
     return HS_OK;
 }
 
 int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const int32_t *fx) {
     AcceptArgs a{};
-    a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd;
+    a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd; a.V = m->c.V;
     a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist;
     PROF(HS_PROF_ACCEPT, 0, launch_accept(a, m->stream), "accept");
     ++m->launches;
@@ -427,11 +427,25 @@ int64_t hs_weight_offset(const hs_config *cfg, int layer, int tensor) {
     return blob_offset(*cfg, layer, tensor);
 }
 
-int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs_model **out) {
-    if (!cfg || !bufs || !out || !valid_config(*cfg)) return HS_ERR_INVALID_ARG;
+static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs, void *stream);
+
+int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, const hs_sizes *have, void *stream, hs_model **out) {
+    if (out) *out = nullptr;
+    if (!cfg || !bufs || !have || !out || !valid_config(*cfg)) return HS_ERR_INVALID_ARG;
     const void *ptrs[6] = {bufs->weights, bufs->snap, bufs->dstate, bufs->conv, bufs->kv, bufs->work};
     for (int i = 0; i < 6; ++i) if (!ptrs[i] || ((uintptr_t)ptrs[i] & (ALIGN - 1))) return HS_ERR_INVALID_ARG;
+    hs_sizes need;
+    if (hs_query_sizes(cfg, &need) != HS_OK) return HS_ERR_INVALID_ARG;
+    if (have->weights < need.weights || have->snap < need.snap || have->dstate < need.dstate || have->conv < need.conv ||
+        have->kv < need.kv || have->work < need.work) return HS_ERR_SIZE;
     hs_model *m = new hs_model();
+    const int rc = init_model(m, cfg, bufs, stream);
+    if (rc != HS_OK) { delete m; return rc; }      // nothing is left behind by a failed call
+    *out = m;
+    return HS_OK;
+}
+
+static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs, void *stream) {
     m->c = *cfg; m->bufs = *bufs; m->stream = (cudaStream_t)stream;
     const hs_config &c = m->c;
     Derived v = derive(c);
@@ -477,7 +491,6 @@ int hs_init_model(const hs_config *cfg, const hs_buffers *bufs, void *stream, hs
     m->Kc = (__nv_bfloat16 *)bufs->kv;
     m->Vc = m->Kc + (size_t)v.n_al * v.B * c.kvh * c.kv_capacity * c.hd;
     m->snap = (float *)bufs->snap; m->dstate = (float *)bufs->dstate;
-    *out = m;
     CK(configure_gemv(), "configure gemv");
     CK(configure_attn(), "configure attention");
     if (configure_gemm_tc() != cudaSuccess) { g_hs_gemm_tc = false; cudaGetLastError(); }   // falls back to several 16-row launches
@@ -520,7 +533,11 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
     for (int b = 0; b < batch; ++b) {
         if (lens_host[b] < 1) return fail(m, HS_ERR_INVALID_ARG, "empty prompt");
         if (m->kv_upper[b] + lens_host[b] > m->c.kv_capacity) return fail(m, HS_ERR_CAPACITY, "prompt exceeds kv_capacity");
+        for (int p = 0; p < lens_host[b]; ++p)
+            if (tokens_host[off + p] < 0 || tokens_host[off + p] >= m->c.V) return fail(m, HS_ERR_INVALID_ARG, "prompt token id outside [0, V)");
+        off += lens_host[b];
     }
+    off = 0;
     for (int b = 0; b < batch; ++b) {
         const int len = lens_host[b];
         for (int p = 0; p < len; p += m->Tm) {
@@ -530,7 +547,7 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
             CK(cudaMemsetAsync(m->ctrl.stage_n + b, 0, 4, m->stream), "prefill stage");
             int32_t n = T - 1;
             CK(cudaMemcpyAsync(m->ctrl.stage_n + b, &n, 4, cudaMemcpyHostToDevice, m->stream), "prefill n");
-            int rc = model_pass(m, false, T, 0, b, 1);
+            int rc = model_pass(m, false, T, 0, b, 1, true);
             if (rc) return rc;
             rc = enqueue_accept(m, T - 1, b, 1, m->ctrl.stage_n, nullptr);
             if (rc) return rc;
@@ -546,6 +563,7 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
 int hs_draft(hs_model *m, int k) {
     if (!m || k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
     if (m->batch < 1) return fail(m, HS_ERR_ORDER, "no active sequences: prefill or set_context first");
+    if (m->phase == 2) return fail(m, HS_ERR_ORDER, "draft after verify: the snapshots hold the verified positions until accept_rollback");
     if (k > 0) {
         const int nb = m->batch;
         int rc = run_maybe_graph(m, (1ull << 40) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
@@ -558,6 +576,7 @@ int hs_draft(hs_model *m, int k) {
 int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (!m || k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
     if (m->batch < 1) return fail(m, HS_ERR_ORDER, "no active sequences: prefill or set_context first");
+    if (m->phase == 2) return fail(m, HS_ERR_ORDER, "verify after verify: the snapshots hold the verified positions until accept_rollback");
     if (!cand_dev && k > 0 && !(m->phase == 1 && m->last_k == k)) return fail(m, HS_ERR_ORDER, "verify(k) needs a preceding draft(k) or explicit candidates");
     const int nb = m->batch, T = k + 1;
     int rc = check_capacity(m, T, 0, nb);
@@ -565,7 +584,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
-    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb); });
+    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
     return HS_OK;
@@ -596,6 +615,14 @@ int hs_round_host(hs_model *m, int k, const int32_t *forced_n_host, const int32_
     if (!m) return HS_ERR_INVALID_ARG;
     const int nb = m->batch;
     if (nb < 1) return fail(m, HS_ERR_ORDER, "no active sequences");
+    if (k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
+    if (m->phase == 2) return fail(m, HS_ERR_ORDER, "round after verify: call accept_rollback first");
+    if (forced_n_host)
+        for (int b = 0; b < nb; ++b)
+            if (forced_n_host[b] < 0 || forced_n_host[b] > k) return fail(m, HS_ERR_INVALID_ARG, "forced accept length outside [0, k]");
+    if (forced_next_host)
+        for (int b = 0; b < nb; ++b)
+            if (forced_next_host[b] >= m->c.V) return fail(m, HS_ERR_INVALID_ARG, "forced next token id >= V");
     if (forced_n_host) CK(cudaMemcpyAsync(m->ctrl.stage_n, forced_n_host, 4 * nb, cudaMemcpyHostToDevice, m->stream), "forced_n upload");
     if (forced_next_host) CK(cudaMemcpyAsync(m->ctrl.stage_next, forced_next_host, 4 * nb, cudaMemcpyHostToDevice, m->stream), "forced_next upload");
     int rc = hs_draft(m, k);
@@ -748,6 +775,19 @@ int hs_device_status(hs_model *m) {
     int32_t st = 0;
     CK(cudaMemcpy(&st, m->ctrl.status, 4, cudaMemcpyDeviceToHost), "status read");
     if (st != 0) { m->err = "a kernel recorded an error in the device status word"; return st; }
+    return HS_OK;
+}
+
+int hs_selftest_wait_timeout(hs_model *m, int polls) {
+    if (!m || polls < 1 || polls > (1 << 20)) return HS_ERR_INVALID_ARG;
+    CK(launch_wait_probe(m->ctrl.status, polls, m->stream), "wait probe");
+    ++m->launches;
+    return HS_OK;
+}
+
+int hs_clear_status(hs_model *m) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    CK(cudaMemsetAsync(m->ctrl.status, 0, 4, m->stream), "status clear");
     return HS_OK;
 }
 

@@ -60,11 +60,17 @@ __device__ __forceinline__ float xreduce(float (&v)[NV], int lane) {
 
 
 // ---- programmatic dependent launch ---------------------------------------------------------------
-// Every kernel of a step is launched with the programmatic-stream-serialization attribute: it may
-// begin while its predecessor is still running.  Code before pdl_wait() may therefore touch only
-// memory that no kernel of the step writes (weights) or that was written at least two kernels
-// earlier; pdl_wait() returns once the predecessor has completed and its writes are visible.
-// pdl_trigger() lets the successor start its own prologue; it is always issued after pdl_wait().
+// Every kernel of a pass except the first is launched with the programmatic-stream-serialization
+// attribute: it may begin while its predecessors are still running.  All kernels call pdl_trigger()
+// at their very start, before their own pdl_wait(), so several kernels of the chain can sit in their
+// prologues at once.  Code before pdl_wait() may therefore read only what NO kernel of the same pass
+// writes: weights and parameters, the RoPE table, and what earlier passes left behind - the control
+// words kv_len / slot (written by the accept kernel) and cached KV rows below kv_len.  That is safe in
+// every mode because the first kernel of a pass is launched in plain stream order (a captured graph's
+// first node likewise starts only when everything enqueued before the graph is complete): nothing of a
+// pass starts before all earlier work has finished.  Prologues write nothing to global memory.
+// pdl_wait() returns once the preceding kernel has completed and its writes are visible; every grid
+// waits before it completes, so completion is transitive along the chain.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -85,11 +91,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 }
 // Bounded wait: gives up after ~2^22 polls (seconds) and reports false, so a copy that never lands
 // turns into an error status instead of a hang.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (int it = 0; it < (1 << 22); ++it)
+__device__ __forceinline__ bool mbar_wait_n(uint64_t *bar, uint32_t parity, int polls) {
+    for (int it = 0; it < polls; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) { return mbar_wait_n(bar, parity, 1 << 22); }
 // 1-D bulk copy; src, dst 16-byte aligned, bytes a multiple of 16
 __device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src, uint32_t bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -133,7 +133,7 @@ struct GemvArgs {
     const void *pf_ptr; int64_t pf_bytes;   // optional: weights of the next projection, prefetched into L2
     __nv_bfloat16 *xb; int64_t xb_rows;     // scratch for the packed activation operand of the many-row kernel: [2][xb_rows][K0+K1]
     int early_trigger;        // 1: let the next kernel start before this one has waited for its predecessor
-                              // (allowed only if that kernel touches nothing but weights before its own wait)
+                              // (what a prologue may read before its own wait is stated in hs_device.cuh)
 };
 // *oparts receives the number of parts written to `out` (1 unless EPI_RESID split the reduction).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
@@ -145,8 +145,9 @@ int gemm_tc_rows(int nrows);
 cudaError_t launch_gemm_tc(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
 cudaError_t configure_attn();
 
-cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
-                         int b0, int nb, float *h, cudaStream_t s);
+// serial = true: launched in plain stream order (without the programmatic attribute); see model_pass
+cudaError_t launch_embed(const __nv_bfloat16 *E, int d, int V, const int32_t *cand, int Tm, int col0, int T,
+                         int b0, int nb, float *h, int32_t *status, bool serial, cudaStream_t s);
 
 struct SsmArgs {
     int H, P, N, di, convd, in_ld;      // in_ld = row stride of zx
@@ -201,9 +202,10 @@ cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int
                           int32_t *tok_out, int tok_col0, float *margin_out, void *part, int32_t *counters, cudaStream_t s);
 
 struct AcceptArgs {
-    int k, Tm, b0, nb, n_rl, B, convd;
+    int k, Tm, b0, nb, n_rl, B, convd, V;
     HsCtrl ctrl;
     const int32_t *forced_n, *forced_next;
     float *cw; const float *hist;       // [n_rl][B][3][convd], [n_rl][B][Tm][convd]
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s);
+cudaError_t launch_wait_probe(int32_t *status, int polls, cudaStream_t s);

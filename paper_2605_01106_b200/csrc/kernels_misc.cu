@@ -2,19 +2,25 @@
 // accept / rollback step (paper Sec. 3.3, greedy rule).
 #include "hs_internal.h"
 #include "hs_device.cuh"
+#include <mutex>
 
 bool g_hs_pdl = true;
 
 namespace {
 using namespace hsd;
 
-// h[row(b,i)][:] = E[cand[b][col0 + i]]
-__global__ void embed_kernel(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
-                             int b0, float *h) {
+// h[row(b,i)][:] = E[cand[b][col0 + i]].  A token id outside [0, V) (a caller's candidate buffer, a forced
+// next token) is never used as an address: the row of token 0 is gathered instead and the status word is set.
+__global__ void embed_kernel(const __nv_bfloat16 *E, int d, int V, const int32_t *cand, int Tm, int col0, int T,
+                             int b0, float *h, int32_t *status) {
     const int i = blockIdx.x, lb = blockIdx.y, b = b0 + lb;
     pdl_trigger();
     pdl_wait();
-    const int tok = __ldcg(cand + b * Tm + col0 + i);
+    int tok = __ldcg(cand + b * Tm + col0 + i);
+    if (tok < 0 || tok >= V) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, (int)HS_ERR_DEVICE);
+        tok = 0;
+    }
     const uint4 *src = reinterpret_cast<const uint4 *>(E + (size_t)tok * d);
     float *dst = h + (size_t)(lb * T + i) * d;
     for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
@@ -109,8 +115,11 @@ __global__ void __launch_bounds__(256) argmax_kernel(const ArgmaxArgs a) {
     t = top2_warp(t);
     if (lane == 0) {
         a.counters[srow] = 0;
-        a.tok_out[b * a.Tm + a.tok_col0 + i] = t.i1;
-        if (a.margin_out) a.margin_out[b * a.Tm + i] = t.v1 - t.v2;
+        // a row without any value above -inf (all -inf or NaN) has no maximum: id 0, like a scan that starts at
+        // element 0 and never finds anything larger; the id is always a valid row of the embedding table
+        const bool none = t.i1 == 0x7fffffff;
+        a.tok_out[b * a.Tm + a.tok_col0 + i] = none ? 0 : t.i1;
+        if (a.margin_out) a.margin_out[b * a.Tm + i] = none ? 0.f : t.v1 - t.v2;
     }
 }
 
@@ -129,6 +138,10 @@ __global__ void accept_kernel(AcceptArgs a) {
     else { n = 0; while (n < k && __ldcg(cand + n + 1) == __ldcg(g + n)) ++n; }
     int next = __ldcg(g + n);
     if (a.forced_next && __ldcg(a.forced_next + b) >= 0) next = __ldcg(a.forced_next + b);
+    if (next < 0 || next >= a.V) {          // only a caller-supplied id can be out of range: never let it reach the gather
+        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) atomicCAS(a.ctrl.status, 0, (int)HS_ERR_DEVICE);
+        next = 0;
+    }
     // conv windows: sequence of raw inputs = [w0 w1 w2 | hist_0 .. hist_k]; new window = entries n+1..n+3
     if (rl < a.n_rl) {
         float *cw = a.cw + ((size_t)rl * a.B + b) * 3 * a.convd;
@@ -156,11 +169,35 @@ __global__ void accept_kernel(AcceptArgs a) {
     }
 }
 
+// Self-test of the bounded wait every copy-fed kernel uses: one warp arms an mbarrier for bytes that no copy
+// will ever deliver, polls it `polls` times, gives up, records HS_ERR_TIMEOUT and returns.  Nothing is in flight
+// when it exits, so the context stays usable.
+__global__ void wait_probe_kernel(int32_t *status, int polls) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_expect_tx(&bar, 16);
+    __syncwarp();
+    const bool ok = __all_sync(0xffffffffu, mbar_wait_n(&bar, 0, polls));
+    if (!ok && threadIdx.x == 0) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);
+}
+
 }  // namespace
 
-cudaError_t launch_embed(const __nv_bfloat16 *E, int d, const int32_t *cand, int Tm, int col0, int T,
-                         int b0, int nb, float *h, cudaStream_t s) {
-    return launch_pdl(embed_kernel, dim3(T, nb), dim3(128), 0, s, E, d, cand, Tm, col0, T, b0, h);
+cudaError_t launch_wait_probe(int32_t *status, int polls, cudaStream_t s) {
+    wait_probe_kernel<<<1, 32, 0, s>>>(status, polls);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_embed(const __nv_bfloat16 *E, int d, int V, const int32_t *cand, int Tm, int col0, int T,
+                         int b0, int nb, float *h, int32_t *status, bool serial, cudaStream_t s) {
+    if (serial) {
+        // first kernel of a pass: ordinary stream order, so that nothing of this pass (whose kernels read control
+        // words in their prologues) starts before everything enqueued earlier - the accept kernel above all - is complete
+        embed_kernel<<<dim3(T, nb), dim3(128), 0, s>>>(E, d, V, cand, Tm, col0, T, b0, h, status);
+        return cudaGetLastError();
+    }
+    return launch_pdl(embed_kernel, dim3(T, nb), dim3(128), 0, s, E, d, V, cand, Tm, col0, T, b0, h, status);
 }
 
 cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int Tm,
@@ -194,21 +231,30 @@ static __device__ __align__(256) unsigned char hs_static_scratch[HS_STATIC_BYTES
 namespace {
 constexpr int HS_STATIC_MAX_DEVICES = 64;
 void *g_static_ptr[HS_STATIC_MAX_DEVICES];     // device address of hs_static_scratch, per device; null = not looked up yet
+std::mutex g_static_mutex;                     // two host threads may make their first call at the same time
 }
 
 extern "C" int hs_argmax_static(const float *logits_dev, int V, int rows, int32_t *token_dev, float *margin_dev, void *stream) {
     if (!logits_dev || !token_dev || V < 1 || rows < 1) return HS_ERR_INVALID_ARG;
     if (rows > HS_STATIC_ROWS) return HS_ERR_SIZE;             // more rows than the built-in scratch holds
+    // the kernel reads rows of a width that is a multiple of four with 128-bit loads: such rows must start on a
+    // 16-byte boundary (a view that begins inside a larger tensor may not); the outputs are plain 32-bit words
+    if (((uintptr_t)logits_dev & ((V & 3) == 0 ? 15u : 3u)) || ((uintptr_t)token_dev & 3u) || ((uintptr_t)margin_dev & 3u))
+        return HS_ERR_INVALID_ARG;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= HS_STATIC_MAX_DEVICES) return HS_ERR_CUDA;
-    if (!g_static_ptr[dev]) {
-        // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
-        // once per device, with that device current.
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, hs_static_scratch) != cudaSuccess || !p) return HS_ERR_CUDA;
-        g_static_ptr[dev] = p;
+    unsigned char *base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+            // once per device, with that device current.
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, hs_static_scratch) != cudaSuccess || !p) return HS_ERR_CUDA;
+            g_static_ptr[dev] = p;
+        }
+        base = static_cast<unsigned char *>(g_static_ptr[dev]);
     }
-    unsigned char *base = static_cast<unsigned char *>(g_static_ptr[dev]);
     int32_t *counters = reinterpret_cast<int32_t *>(base + HS_STATIC_PART_BYTES);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the tickets must start at zero whatever an earlier (possibly failed) call left behind

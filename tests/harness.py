@@ -1,6 +1,6 @@
 """Round-by-round comparison of the CUDA library with the CPU oracle on the same seeded inputs.
 
-Tolerances (from the benchmark spec): token ids, accept lengths and KV/state indices bit-exact wherever the
+Tolerances (those the workload definition states): token ids, accept lengths and KV/state indices bit-exact wherever the
 oracle's top-2 logit margin exceeds 1e-2 (narrower positions are listed, and the GPU is re-synchronised to
 the oracle there); logits within 2e-2 absolute; recurrent states within 1e-3 of the state's magnitude.
 """
@@ -66,9 +66,30 @@ def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
                 # arithmetic difference (about 1e-4 relative: fp32 activations enter the tensor-core projections
                 # as bf16 head + remainder) of a rounding boundary
                 assert (got == want).mean() > 0.75, ("kv exact fraction", l, b, kind, (got == want).mean())
+    # nothing was written behind any of the buffers the library was given
+    assert eng.check_guards(), "guard bytes behind a library buffer were overwritten"
     if rep is not None:
         rep.max_state_err = max(rep.max_state_err, worst)
     return worst
+
+
+def run_rounds_async(eng, seqs, ks):
+    """Rounds with the library's own acceptance and NO host read between them: every call is only enqueued, so
+    consecutive passes follow each other on the device as closely as the launch mode allows.  ks: draft length
+    of each round (0 = plain autoregressive step).  The oracle sequences take the same rounds; the caller compares
+    afterwards (compare_states with kv_rows=None covers kv_len, pending, recurrent state and every KV row, i.e.
+    every consumed token)."""
+    for k in ks:
+        eng.draft(k)
+        eng.verify(k)
+        eng.accept_rollback(readback=False)
+    emitted = []
+    for o in seqs:
+        toks = []
+        for k in ks:
+            toks += list(o.round(k)["emitted"])
+        emitted.append(toks)
+    return emitted
 
 
 def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_every=1, check_logits=True,

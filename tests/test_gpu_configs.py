@@ -88,7 +88,9 @@ def test_cfg4_sequential_full_size(env):
 
 
 def test_cfg3_3b_batch1(env):
-    s, eng, model, seqs = make(env, "cfg3_3b", 1, 4, 2100, {0}, [2048], small_init="unit")
+    # perturbed small parameters (norm weights, D, conv bias): a kernel that dropped one of them at this shape
+    # (N = 256, 80 heads, 20 query heads) would be noticed
+    s, eng, model, seqs = make(env, "cfg3_3b", 1, 4, 2100, {0}, [2048])
     rep = env["harness"].run_rounds(eng, seqs, s, 2, 1, forced=[[1]])
     rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=[[2]], rep=rep)
     print(rep)
@@ -96,9 +98,11 @@ def test_cfg3_3b_batch1(env):
 
 
 def test_cfg3_3b_batch8_two_checked(env):
-    s, eng, model, seqs = make(env, "cfg3_3b", 8, 4, 2100, {0, 5}, [2048] * 8, small_init="unit")
+    s, eng, model, seqs = make(env, "cfg3_3b", 8, 4, 2100, {0, 5}, [2048] * 8)
     forced = [hi.forced_accept(4, 1, seq=b) for b in range(8)]
     rep = env["harness"].run_rounds(eng, seqs, s, 4, 1, forced=forced)
+    forced = [hi.forced_accept(2, 1, seq=20 + b) for b in range(8)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 1, forced=forced, rep=rep)
     print(rep)
     assert eng.device_status() == 0
 

@@ -129,3 +129,73 @@ def test_call_order_and_capacity_errors(env):
             eng.round(2)
     assert e.value.code == -3
     assert eng.device_status() == 0                # the host refused before any kernel overran the cache
+
+
+def test_order_and_argument_errors_leave_the_state_alone(env):
+    # a second verify (or a draft) between verify and accept_rollback would start from snapshots that already hold
+    # the verified positions: refused; a forced accept length beyond k and token ids outside the vocabulary are
+    # refused on the host before anything is enqueued
+    s, eng, model, seqs = setup(env, "cfg1_tiny", [16], max_k=2, cap=128)
+    hs = env["hs"]
+    L = hs.lib()
+    eng.draft(2); eng.verify(2)
+    for call in (lambda: eng.verify(2), lambda: eng.draft(2), lambda: eng.round_host(2)):
+        with pytest.raises(hs.HsError) as e:
+            call()
+        assert e.value.code == -4
+    eng.accept_rollback(readback=True)
+    for o in seqs:
+        o.round(2)
+    with pytest.raises(hs.HsError) as e:
+        eng.round_host(2, forced_n=[3])
+    assert e.value.code == -1
+    with pytest.raises(hs.HsError) as e:
+        eng.round_host(2, forced_n=[1], forced_next=[s.V])
+    assert e.value.code == -1
+    bad = np.array([5, s.V, 7], np.int32); lens = np.array([3], np.int32)
+    assert L.hs_prefill(eng.h, bad.ctypes.data, lens.ctypes.data, 1) == -1
+    bad[1] = -2
+    assert L.hs_prefill(eng.h, bad.ctypes.data, lens.ctypes.data, 1) == -1
+    # nothing of the refused calls ran: the next round still agrees with the oracle
+    env["harness"].run_rounds(eng, seqs, s, 2, 2)
+    assert eng.device_status() == 0
+
+
+def test_out_of_range_candidate_is_not_used_as_an_address(env):
+    # candidates supplied on the device cannot be checked by the host: the gather clamps them and reports
+    s, eng, model, seqs = setup(env, "cfg1_tiny", [16], max_k=2, cap=128)
+    torch, hs = env["torch"], env["hs"]
+    cand = torch.tensor([[3, 2 ** 30, -5]], dtype=torch.int32, device=eng.device)
+    eng.verify(2, cand)
+    eng.accept_rollback(readback=True)
+    assert eng.device_status() == -7
+    eng.clear_status()
+    assert eng.device_status() == 0 and eng.check_guards()
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("name", ["cfg1_tiny", "test_seq"])
+def test_rounds_back_to_back_without_host_reads(env, name, flags):
+    # 24 rounds, k = 0 (verify directly after accept) mixed with k = 2 and 4, the library's own acceptance, and no
+    # host read or synchronisation between rounds: the control words (kv_len, snapshot slot) written by the accept
+    # kernel of one round are read by the first mixer / attention kernels of the next as early as the launch mode
+    # lets them start.  Afterwards every consumed token (all KV rows), the recurrent state, the conv window,
+    # kv_len and the pending token must be the oracle's.
+    s, eng, model, seqs = setup(env, name, [hi.CONFIGS[name].prompt_len], max_k=4, cap=512, flags=flags)
+    ks = [2, 0, 0, 2, 4, 0, 2, 2, 0, 4, 0, 0] * 2
+    env["harness"].run_rounds_async(eng, seqs, ks)
+    env["harness"].compare_states(eng, seqs, s, kv_rows=None)
+    assert eng.get_context(0)[0] >= hi.CONFIGS[name].prompt_len + len(ks)      # at least one token per round
+    assert eng.device_status() == 0
+
+
+def test_bounded_wait_runs_out_and_reports(env):
+    # every wait on a copy barrier gives up after a fixed number of polls; here nothing ever completes the barrier:
+    # the kernel must end by itself, the status word must say HS_ERR_TIMEOUT, and the handle must stay usable
+    s, eng, model, seqs = setup(env, "cfg1_tiny", [16], max_k=2, cap=128)
+    eng.selftest_wait_timeout(2000)
+    assert eng.device_status() == -6
+    eng.clear_status()
+    assert eng.device_status() == 0
+    env["harness"].run_rounds(eng, seqs, s, 2, 2)
+    assert eng.device_status() == 0

@@ -69,3 +69,40 @@ def test_invalid_configs_are_rejected(hs):
     assert L.hs_query_sizes(None, ctypes.byref(sz)) == -1
     assert L.hs_draft(None, 1) == -1 and L.hs_verify(None, 1, None) == -1
     assert L.hs_accept_rollback(None, None, None, None, None) == -1
+
+
+def test_init_refuses_short_buffers_before_any_device_work(hs):
+    # hs_init_model is told how many bytes each caller buffer really has; a short one is HS_ERR_SIZE, decided on
+    # the host before any CUDA call (the pointers below are never dereferenced), and no handle is left behind
+    s = hi.CONFIGS["cfg1_tiny"]
+    cfg = hs.make_config(s, max_batch=1, max_k=2, kv_capacity=64)
+    need = hs.query_sizes(cfg)
+    L = hs.load_library()
+    fake = hs.HsBuffers(*[0x10000 * (i + 1) for i in range(6)])
+    for field in ("weights", "snap", "dstate", "conv", "kv", "work"):
+        have = hs.HsSizes(*[getattr(need, f) for f in ("weights", "snap", "dstate", "conv", "kv", "work")])
+        setattr(have, field, getattr(need, field) - 1)
+        h = hs.vp(0xdead)
+        assert L.hs_init_model(ctypes.byref(cfg), ctypes.byref(fake), ctypes.byref(have), None, ctypes.byref(h)) == -2, field
+        assert not h.value
+    # misaligned or null buffers and a missing size record are invalid arguments
+    have = hs.HsSizes(*[getattr(need, f) for f in ("weights", "snap", "dstate", "conv", "kv", "work")])
+    odd = hs.HsBuffers(0x10000, 0x20000, 0x30010, 0x40000, 0x50000, 0x60000)
+    h = hs.vp()
+    assert L.hs_init_model(ctypes.byref(cfg), ctypes.byref(odd), ctypes.byref(have), None, ctypes.byref(h)) == -1
+    assert L.hs_init_model(ctypes.byref(cfg), ctypes.byref(fake), None, None, ctypes.byref(h)) == -1
+    assert L.hs_round_host(None, 1, None, None, None, None) == -1
+    assert L.hs_selftest_wait_timeout(None, 10) == -1 and L.hs_clear_status(None) == -1
+
+
+def test_static_argmax_argument_checks_need_no_device(hs):
+    # pointer, size and alignment checks of the allocation-free argmax come before any CUDA call
+    L = hs.load_library()
+    assert L.hs_argmax_static(None, 8, 1, 0x1000, None, None) == -1
+    assert L.hs_argmax_static(0x1000, 8, 1, None, None, None) == -1
+    assert L.hs_argmax_static(0x1000, 0, 1, 0x2000, None, None) == -1
+    assert L.hs_argmax_static(0x1000, 8, 65, 0x2000, None, None) == -2
+    assert L.hs_argmax_static(0x1004, 8, 1, 0x2000, None, None) == -1        # V % 4 == 0: rows are read 128 bits at a time
+    assert L.hs_argmax_static(0x1000, 8, 1, 0x2002, None, None) == -1
+    assert L.hs_argmax_static(0x1000, 8, 1, 0x2000, 0x3001, None) == -1
+    assert L.hs_argmax_static(0x1002, 7, 1, 0x2000, None, None) == -1        # floats are 4-byte aligned at least

@@ -57,3 +57,70 @@ def test_static_argmax_matches_verify_twice_and_rejects_oversize():
         hs.argmax_static(big, torch.zeros(65, dtype=torch.int32, device=dev))
     assert e.value.code == -2
     assert eng.device_status() == 0
+
+
+def test_static_argmax_ties_odd_widths_and_misaligned_views():
+    """The device-side tie rule (lowest id wins, margin 0 when the maximum is not unique), row widths that are not
+    a multiple of four or smaller than the number of blocks that share a row, rows without any finite value, and
+    the refusal of a logits view that does not start on a 16-byte boundary - all through the C entry point."""
+    import torch
+    from paper_2605_01106_b200 import build, binding as hs
+    build.build()
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device="cpu").manual_seed(5)
+
+    def run(lg):
+        rows = lg.shape[0]
+        tok = torch.full((rows,), -7, dtype=torch.int32, device=dev)
+        mar = torch.full((rows,), -1.0, dtype=torch.float32, device=dev)
+        hs.argmax_static(lg, tok, mar)
+        torch.cuda.synchronize(dev)
+        return tok.cpu().numpy(), mar.cpu().numpy()
+
+    # ties: the maximum duplicated inside one block's slice, across slices (ids 5, 1000 and 4000 of 4096 lie in
+    # different 128-wide slices), at the very last id, and a constant row
+    V = 4096
+    lg = torch.randn(6, V, generator=g).clamp_(-3, 3)
+    lg[0, [5, 6]] = 9.0
+    lg[1, [4000, 1000, 5]] = 9.0
+    lg[2, [V - 1, 77]] = 9.0
+    lg[3, :] = 0.25
+    lg[4, 2049] = 9.0                                     # unique maximum: margin is top1 - top2
+    lg[5, [0, V - 1]] = 9.0
+    tok, mar = run(lg.to(dev))
+    assert list(tok) == [5, 5, 77, 0, 2049, 0], tok
+    assert list(mar[[0, 1, 2, 3, 5]]) == [0.0] * 5
+    assert mar[4] == 9.0 - float(lg[4][lg[4] < 9.0].max())
+    # widths that are not a multiple of four (scalar path) and narrower than the 32 blocks of a row
+    for V in (7, 30, 33, 1001):
+        lg = torch.randn(5, V, generator=g)
+        lg[1, V - 1] = 50.0
+        lg[2, [V // 2, V - 2]] = 50.0
+        tok, mar = run(lg.to(dev))
+        ref = lg.numpy()
+        assert np.array_equal(tok, ref.argmax(axis=1).astype(np.int32)), (V, tok)
+        top2 = np.sort(ref, axis=1)[:, -2:]
+        assert np.array_equal(mar, top2[:, 1] - top2[:, 0]), V
+    # a row with no finite value: id 0 (always a valid token), margin 0
+    lg = torch.full((2, 64), float("-inf"))
+    lg[1, :] = float("nan")
+    tok, mar = run(lg.to(dev))
+    assert list(tok) == [0, 0] and list(mar) == [0.0, 0.0]
+    # a view that starts one float into a larger tensor is only 4-byte aligned: with V % 4 == 0 it is refused on the
+    # host (the kernel would read it 128 bits at a time), with an odd V it is served by the scalar path
+    big = torch.randn(4 * 64 + 1, generator=g).to(dev)
+    view = big[1:].view(4, 64)
+    assert view.data_ptr() % 16 == 4
+    tok = torch.zeros(4, dtype=torch.int32, device=dev)
+    with pytest.raises(hs.HsError) as e:
+        hs.argmax_static(view, tok)
+    assert e.value.code == -1
+    view7 = big[1:1 + 4 * 7].view(4, 7)
+    hs.argmax_static(view7, tok)
+    torch.cuda.synchronize(dev)
+    assert np.array_equal(tok.cpu().numpy(), view7.cpu().numpy().argmax(axis=1).astype(np.int32))
+    # the binding refuses tensors the C entry point could not interpret
+    for bad in (lambda: hs.argmax_static(view.half(), tok), lambda: hs.argmax_static(big[: 4 * 64].view(4, 64).t(), tok),
+                lambda: hs.argmax_static(big[: 4 * 64].view(4, 64), tok[:3])):
+        with pytest.raises(hs.HsError):
+            bad()
