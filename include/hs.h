@@ -199,6 +199,18 @@ int64_t hs_launch_count(const hs_model *m);
  * for small batch * capacity): otherwise HS_ERR_INVALID_ARG and nothing changes.  Results do not depend on
  * the setting beyond fp32 summation order. */
 int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);
+/* Tuning / measurement hook: switch a kernel choice on (value != 0) or off.  The choices are process-wide (they
+ * apply to every handle); the handle's captured graphs are dropped so that the next step is captured afresh.
+ * Results are the same within fp32 summation order.  Synchronises the stream.
+ *   HS_OPT_CLUSTER_REDUCE  residual projections with 4..16 activation rows add the partial sums of their K split
+ *                          inside a thread-block cluster (default on; off: the consumers add the parts)
+ *   HS_OPT_GEMM_MMA        4..16 activation rows on the warp-level tensor path (default on; off: CUDA cores)
+ *   HS_OPT_GEMM_TC         more than 16 activation rows on tcgen05 (default on; off: several 16-row launches)
+ *   HS_OPT_PDL             programmatic dependent launch between the kernels of a pass (default on)
+ *   HS_OPT_ATTN_SMALL      verify attention with at most 16 query rows per KV head over caches of up to 1024 keys
+ *                          (2048 in a sequential hybrid) in its latency-lean form (default on; off: the general form) */
+enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4 };
+int hs_set_option(hs_model *m, int option, int value);
 /* Measurement hook.  hs_profile(m, 1) brackets every following kernel launch with two CUDA events on
  * the launching stream (graph replay is bypassed while it is on); hs_profile_read synchronises and
  * returns, per category, the summed device time in ms, the number of launches and the algorithmic

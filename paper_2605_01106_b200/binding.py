@@ -19,7 +19,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_set_attn_geometry", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
+           "hs_set_attn_geometry", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
            "hs_selftest_wait_timeout", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
@@ -73,6 +73,7 @@ def load_library(path: str | None = None):
     L.hs_launch_count.restype = i64
     L.hs_launch_count.argtypes = [vp]
     L.hs_set_attn_geometry.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    L.hs_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     L.hs_profile.argtypes = [vp, ctypes.c_int]
     L.hs_profile_read.argtypes = [vp, vp, vp, vp]
     L.hs_device_status.argtypes = [vp]
@@ -310,6 +311,12 @@ class Engine:
     def set_attn_geometry(self, chunk, tiles=1):
         """Fix the KV split of verify-mode attention (chunk keys x tiles per CTA); chunk = 0: automatic."""
         self._ck(lib().hs_set_attn_geometry(self.h, int(chunk), int(tiles)))
+
+    OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL = range(5)
+
+    def set_option(self, option, value):
+        """Switch a kernel choice (process-wide) on or off; see hs_set_option."""
+        self._ck(lib().hs_set_option(self.h, int(option), int(value)))
 
     def profile(self, enable):
         self._ck(lib().hs_profile(self.h, int(enable)))

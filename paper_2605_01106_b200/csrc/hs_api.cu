@@ -6,6 +6,8 @@
 #include <cstring>
 #include <algorithm>
 
+bool g_hs_attn_small = true;   // short caches and few query rows use the latency-lean attention form
+
 namespace {
 
 constexpr int64_t ALIGN = 256;
@@ -189,17 +191,25 @@ double gemv_bytes(const GemvArgs &a) {
 // tiles over several clusters.  Tiles per CTA: one, unless the launch would have far more CTAs than the GPU
 // runs at once (long caches at large batch) - then a CTA walks up to sixteen 64-key tiles, so that staging
 // the queries and combining the partials is paid once per 1024 keys.
+// Few query rows (G * T <= 16) over caches that fit one cluster: the latency-lean attention form, keys per CTA in
+// steps of 32 up to 128 (parallel blocks: the mixer CTAs of the fused launch get the same shared memory) or 256.
 struct AttnGeom {
-    int chunk, tiles;
-    int code() const { return (chunk / 16 - 1) * 32 + tiles - 1; }   // < 256, part of the graph key
+    int chunk, tiles, small;
+    int code() const { return small * 512 + (chunk / 16 - 1) * 32 + tiles - 1; }   // < 1024, part of the graph key
 };
 AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
-    if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles};
+    if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles, 0};
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
+    {
+        const int limit = m->c.arch == HS_ARCH_PARALLEL ? 128 : 256;
+        int ck = 32;
+        while (ck < limit && 8 * ck < maxlen + T) ck += 32;
+        if (g_hs_attn_small && (m->c.qh / m->c.kvh) * T <= 16 && 8 * ck >= maxlen + T) return AttnGeom{ck, 1, 1};
+    }
     int want = 32;
     while (want < 128 && 8 * want < maxlen + T) want += 32;
-    AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1};
+    AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1, 0};
     const int64_t ctas64 = (int64_t)nb * m->c.kvh * ((maxlen + T + 63) / 64);
     const int64_t fill = 148 * 8;             // CTAs that keep every SM busy for several rounds
     if (g.chunk == 128 && ctas64 >= 4 * fill) {
@@ -213,7 +223,7 @@ AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
 // round): its first kernel goes out in plain stream order, see hs_device.cuh.
 int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool first) {
     const hs_config &c = m->c;
-    const AttnGeom at_geom = draft ? AttnGeom{m->att_chunk, 1} : attn_geom(m, T, b0, nb);
+    const AttnGeom at_geom = draft ? AttnGeom{m->att_chunk, 1, 0} : attn_geom(m, T, b0, nb);
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
@@ -289,7 +299,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
             aa.Kc = m->Kc + ly.al * per_layer; aa.Vc = m->Vc + ly.al * per_layer; aa.cap = c.kv_capacity;
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
-            aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles;
+            aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles; aa.small = at_geom.small;
             aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
             bool fused = false;
             if (ssm_deferred) {
@@ -566,7 +576,7 @@ int hs_draft(hs_model *m, int k) {
     if (m->phase == 2) return fail(m, HS_ERR_ORDER, "draft after verify: the snapshots hold the verified positions until accept_rollback");
     if (k > 0) {
         const int nb = m->batch;
-        int rc = run_maybe_graph(m, (1ull << 40) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
+        int rc = run_maybe_graph(m, (1ull << 60) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
         if (rc) return rc;
     }
     m->phase = 1; m->last_k = k;
@@ -584,7 +594,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
-    rc = run_maybe_graph(m, (2ull << 40) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
+    rc = run_maybe_graph(m, (2ull << 60) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
     return HS_OK;
@@ -744,6 +754,19 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
     if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
         return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk a multiple of 16 up to 128, tiles 1..32, chunk * tiles >= workspace chunk");
     m->att_force_chunk = chunk; m->att_force_tiles = tiles;
+    return HS_OK;
+}
+
+int hs_set_option(hs_model *m, int option, int value) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    bool *flag = option == HS_OPT_CLUSTER_REDUCE ? &g_hs_cluster_reduce : option == HS_OPT_GEMM_MMA ? &g_hs_gemm_mma
+               : option == HS_OPT_GEMM_TC ? &g_hs_gemm_tc : option == HS_OPT_PDL ? &g_hs_pdl
+               : option == HS_OPT_ATTN_SMALL ? &g_hs_attn_small : nullptr;
+    if (!flag) return fail(m, HS_ERR_INVALID_ARG, "unknown option");
+    CK(cudaStreamSynchronize(m->stream), "option sync");
+    *flag = value != 0;
+    for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);     // captured with the old choice
+    m->graphs.clear(); m->graph_launches.clear();
     return HS_OK;
 }
 

@@ -90,6 +90,7 @@ struct hs_model {
 // Every kernel of a step is launched with programmatic stream serialization: it may start while its
 // predecessor still runs and synchronises with griddepcontrol.wait (see hs_device.cuh).
 extern bool g_hs_pdl;
+extern bool g_hs_cluster_reduce; // residual projections of 4..16 rows reduce their K split inside a thread-block cluster
 extern bool g_hs_gemm_mma;     // projections with 2..16 activation rows on the tensor cores (default) or the CUDA cores
 // cluster_x > 1 launches thread-block clusters of that many CTAs along x (grid.x must be a multiple).
 template <class... KArgs, class... Args>
@@ -189,6 +190,7 @@ struct AttnArgs {
     float *o;                           // [rows][qh*hd]
     float *part_acc, *part_ml; int32_t *counters; int32_t *status;
     int chunk, tiles, nch;              // keys per tile, tiles per CTA, CTAs (key ranges) that cover the cache capacity
+    int small;                          // 1: the latency-lean form (G*T <= 16 rows, every cache within one cluster of 8 CTAs x chunk keys)
     int T, b0, nb;
 };
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);

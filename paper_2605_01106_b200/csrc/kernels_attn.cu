@@ -38,7 +38,7 @@ constexpr int AT_CL = 8;               // CTAs (chunks) per thread-block cluster
 
 struct AttnLayout {
     int kstr, keys, mrows, pstr, sstr;
-    size_t k_off, v_off, q_off, s_off, p_off, ml_off, corr_off, new_off, rope_off, red_off, total;
+    size_t k_off, v_off, q_off, s_off, p_off, ml_off, corr_off, new_off, rope_off, red_off, rx_off, total;
 };
 // shared-memory carve-up for head dim hd, chunk ck, gt query rows
 __host__ __device__ inline AttnLayout attn_layout(int hd, int ck, int gt) {
@@ -59,6 +59,8 @@ __host__ __device__ inline AttnLayout attn_layout(int hd, int ck, int gt) {
     L.new_off = o; o += (size_t)2 * HS_MAX_T * L.kstr * 2;    // the new K | V rows as they are cached
     L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
     L.red_off = o; o += (size_t)(AT_CL * HS_MAX_GT * 3 + HS_MAX_GT * 2) * 4;
+    // what the peers of the cluster send: per source rank [gt][hd / AT_CL] partial outputs, then [gt][2] (max, sum)
+    L.rx_off = o; o += (size_t)AT_CL * gt * (hd / AT_CL + 2) * 4;
     L.total = (o + 127) / 128 * 128;
     return L;
 }
@@ -161,6 +163,23 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     // ---- queries: RoPE at position len + i, pre-multiplied by 1/sqrt(hd), split into bf16 head + remainder
     const int rowbase = lb * T;
     const float scale = rsqrtf((float)HD);
+    // the CTA of the last key range also needs the raw k and v of the new positions: requested now, together with
+    // the queries, so that both arrive after one trip to L2
+    constexpr int NKV = (HS_MAX_T * (HD / 2) + AT_THREADS - 1) / AT_THREADS;
+    float kraw[NKV][4];
+    if (last) {
+#pragma unroll
+        for (int it = 0; it < NKV; ++it) {
+            const int idx = tid + it * AT_THREADS;
+            kraw[it][0] = kraw[it][1] = kraw[it][2] = kraw[it][3] = 0.f;
+            if (idx < T * (HD / 2)) {
+                const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+                const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
+                kraw[it][0] = __ldcg(row + a.k_off + kh * HD + e); kraw[it][1] = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
+                kraw[it][2] = __ldcg(row + a.v_off + kh * HD + e); kraw[it][3] = __ldcg(row + a.v_off + kh * HD + e + HD / 2);
+            }
+        }
+    }
     {
         // thread = (rotation pair e, one of NH interleaved sets of query rows); four rows per round, whose loads
         // are all issued before the first use
@@ -196,16 +215,17 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     if (last) {
         // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached: appended to the cache and kept
         // aside; they join the last tile behind its cached keys
-#pragma unroll 1
-        for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
+#pragma unroll
+        for (int it = 0; it < NKV; ++it) {
+            const int idx = tid + it * AT_THREADS;
+            if (idx >= T * (HD / 2)) break;
             const int i = idx / (HD / 2), e = idx - i * (HD / 2);
-            const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
             const float2 cs = rope_s[idx];
-            const float x0 = __ldcg(row + a.k_off + kh * HD + e), x1 = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
+            const float x0 = kraw[it][0], x1 = kraw[it][1];
             const __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * cs.x - x1 * cs.y);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
-            const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(kraw[it][2]);
+            const __nv_bfloat16 v1 = __float2bfloat16_rn(kraw[it][3]);
             Kn_s[i * KSTR + e] = k0; Kn_s[i * KSTR + e + HD / 2] = k1;
             Vn_s[i * KSTR + e] = v0; Vn_s[i * KSTR + e + HD / 2] = v1;
             Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
@@ -288,17 +308,20 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         fetch(K_s, Kb, t + 1);              // the K buffer is free: next tile's keys arrive during softmax and P V
         // ---- softmax of the tile folded into the running (max, sum): eight lanes per query row, sixteen rows
         //      per pass; probabilities as bf16 head + remainder
-        constexpr int LPR = MT == 1 ? 8 : 4;          // lanes per query row: one pass covers 16 (MT = 1) or 32 rows
+        // lanes per query row: as many as the block has for GT rows (a power of two up to 32), so that a few rows
+        // (small k) are not left to a fraction of one warp
+        const int LPR = GT * 32 <= AT_THREADS ? 32 : GT * 16 <= AT_THREADS ? 16 : GT * 8 <= AT_THREADS ? 8 : 4;
+        const int lsh = LPR == 32 ? 5 : LPR == 16 ? 4 : LPR == 8 ? 3 : 2;
 #pragma unroll 1
         for (int q0 = 0; q0 < GT; q0 += AT_THREADS / LPR) {
-            const int qi = q0 + tid / LPR, sub = tid % LPR;
+            const int qi = q0 + (tid >> lsh), sub = tid & (LPR - 1);
             const bool rv = qi < GT;
             const float m_old = rv ? ml_s[2 * qi] : -INFINITY, l_old = rv ? ml_s[2 * qi + 1] : 0.f;
             float mx = m_old;
             if (rv)
 #pragma unroll 4
                 for (int j = sub; j < nkp; j += LPR) mx = fmaxf(mx, s_s[qi * SSTR + j]);
-#pragma unroll
+#pragma unroll 1
             for (int o = LPR / 2; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             float sum = 0.f;
             if (rv)
@@ -311,7 +334,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
                     Ph_s[qi * PSTR + j] = h; Pl_s[qi * PSTR + j] = l;
                     sum += p;
                 }
-#pragma unroll
+#pragma unroll 1
             for (int o = LPR / 2; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             if (rv && sub == 0) {
                 const float corr = m_old == -INFINITY ? 0.f : __expf(m_old - mx);
@@ -353,22 +376,36 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         fetch(V_s, Vb, t + 1);
     }
     cp_async_wait_all();                    // only empty groups can be left
-    // ---- this CTA's partial into its own shared memory (the query tiles are no longer needed)
-    float *acc_s = reinterpret_cast<float *>(Qh_s);          // [GT][HD] fp32
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int row = mt * 16 + g8 + hh * 8, d = warp * DW + nt * 8 + 2 * t4;
-                if (row < GT) *reinterpret_cast<float2 *>(acc_s + row * HD + d) = make_float2(O[mt][nt][2 * hh], O[mt][nt][2 * hh + 1]);
-            }
-    float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
-    // ---- combine the chunks of this cluster through distributed shared memory: rank r sums output dims
-    //      [r * DS, (r + 1) * DS) over all ranks
+    // ---- combine the key ranges of this cluster.  Rank r finishes the output dimensions [r * DS, (r + 1) * DS):
+    //      every CTA that holds keys stores, straight from its accumulator registers, the slice each peer finishes
+    //      into that peer's shared memory (plus its running max and sum), the cluster meets at ONE barrier, and every
+    //      rank merges what it received - in rank order, so the result does not depend on timing.  Nothing is read
+    //      from a peer after the barrier, so a CTA may exit as soon as it is done.
     constexpr int DS = HD / AT_CL;
-    cluster.sync();
+    float *rx_acc = reinterpret_cast<float *>(smraw + L.rx_off);          // [source rank][GT][DS]
+    float *rx_ml = rx_acc + (size_t)AT_CL * GT * DS;                       // [source rank][GT][2]
+    const int nlive = min(AT_CL, nsplit - cl * AT_CL);                     // ranks of this cluster that hold keys
+    if (crank < nlive) {
+        const uint32_t acc_a = smem_u32(rx_acc) + (uint32_t)crank * GT * DS * 4;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = mt * 16 + g8 + hh * 8, d = warp * DW + nt * 8 + 2 * t4;
+                    if (row < GT)
+                        dsmem_st_v2(dsmem_addr(acc_a + (uint32_t)(row * DS + (d % DS)) * 4, (uint32_t)(d / DS)), O[mt][nt][2 * hh], O[mt][nt][2 * hh + 1]);
+                }
+        const uint32_t ml_a = smem_u32(rx_ml) + (uint32_t)crank * GT * 2 * 4;
+#pragma unroll 1
+        for (int idx = tid; idx < GT * AT_CL; idx += AT_THREADS) {
+            const int dest = idx & (AT_CL - 1), qi = idx >> 3;
+            dsmem_st_v2(dsmem_addr(ml_a + (uint32_t)qi * 8, (uint32_t)dest), ml_s[2 * qi], ml_s[2 * qi + 1]);
+        }
+    }
+    float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
+    cluster_arrive(); cluster_wait();
     const int nclus = (nsplit + AT_CL - 1) / AT_CL;
     const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
     float *Md_s = red_s;                                     // [GT][2] merged (M, den), for the cluster partial
@@ -379,9 +416,12 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
         float2 mlr[AT_CL];
         float4 v[AT_CL];
 #pragma unroll
-        for (int r = 0; r < AT_CL; ++r) {                    // all remote reads are independent: one round trip
-            mlr[r] = *reinterpret_cast<const float2 *>(cluster.map_shared_rank(ml_s, r) + 2 * qi);
-            v[r] = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(acc_s, r) + qi * HD + d);
+        for (int r = 0; r < AT_CL; ++r) {
+            mlr[r] = make_float2(-INFINITY, 0.f); v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r < nlive) {
+                mlr[r] = *reinterpret_cast<const float2 *>(rx_ml + ((size_t)r * GT + qi) * 2);
+                v[r] = *reinterpret_cast<const float4 *>(rx_acc + ((size_t)r * GT + qi) * DS + dd);
+            }
         }
         float M = -INFINITY;
 #pragma unroll
@@ -407,7 +447,6 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     }
     if (nclus > 1) __syncthreads();
     if (nclus > 1 && crank == 0 && tid < 2 * GT) a.part_ml[(pbase + cl) * HS_MAX_GT * 2 + tid] = Md_s[tid];
-    cluster.sync();                                          // peers may still be reading this CTA's shared memory
     if (nclus == 1) return;
     // ---- several clusters: the CTA that arrives last merges the cluster partials in order
     __threadfence();
@@ -471,6 +510,288 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Short caches and few query rows (G*T <= 16, the whole cache within one cluster of eight CTAs): the
+// latency-lean form.  A CTA holds its whole key range (up to 256 cached keys plus the new rows) in shared
+// memory, fetched before the dependency wait.  After the queries are staged there is no block-wide
+// synchronisation any more: every warp takes 16 keys at a time, computes the scores on the tensor cores,
+// keeps the probabilities in registers (the accumulator layout of the score tile is the operand layout of
+// the P V product), runs its own running softmax over its key groups and accumulates its own partial output
+// over the full head dimension.  Each warp then stores, straight from registers, the slice of its partial that
+// each rank of the cluster finishes into that rank's shared memory, the cluster meets at one barrier, and
+// every rank merges the 4 x 8 warp partials of its output dimensions in a fixed order.
+struct AttnSmallLayout { int kstr, keys; size_t k_off, v_off, q_off, rope_off, rx_off, total; };
+__host__ __device__ inline AttnSmallLayout attn_small_layout(int hd, int ck, int gt) {
+    AttnSmallLayout L;
+    L.kstr = hd + 8;
+    L.keys = ck + 16;                      // cached keys + the new rows, rounded to the MMA k step
+    size_t o = 128;
+    L.k_off = o; o += (size_t)L.keys * L.kstr * 2;
+    L.v_off = o; o += (size_t)L.keys * L.kstr * 2;
+    L.q_off = o; o += (size_t)2 * 16 * L.kstr * 2;              // 16 query rows: bf16 head | remainder
+    L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
+    L.rx_off = o; o += (size_t)AT_CL * AT_WARPS * gt * (hd / AT_CL + 2) * 4;   // per source warp: [gt][hd/8] partials, [gt][2] (max, sum)
+    L.total = (o + 127) / 128 * 128;
+    return L;
+}
+constexpr int AT_SMALL_MAXCHUNK = 256;
+
+template <int HD>
+__device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int split, const int kh, const int lb, unsigned char *smraw) {
+    const int CK = a.chunk;                        // cached keys per CTA: a multiple of 16 up to 256
+    const int G = a.qh / a.kvh, T = a.T, GT = G * T;
+    const AttnSmallLayout L = attn_small_layout(HD, CK, GT);
+    const int KSTR = L.kstr;
+    __nv_bfloat16 *K_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.k_off);         // [keys][KSTR]
+    __nv_bfloat16 *V_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.v_off);
+    __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.q_off);        // [16][KSTR] rotated, pre-scaled
+    __nv_bfloat16 *Ql_s = Qh_s + (size_t)16 * KSTR;
+    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);                 // [T][HD/2]
+    constexpr int DS = HD / AT_CL, NSRC = AT_CL * AT_WARPS;
+    float *rx_acc = reinterpret_cast<float *>(smraw + L.rx_off);                     // [source warp][GT][DS]
+    float *rx_ml = rx_acc + (size_t)NSRC * GT * DS;                                  // [source warp][GT][2]
+
+    const int b = a.b0 + lb;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t tinv = (65536u + T - 1) / T;      // x / T == (x * tinv) >> 16 for the small x used here
+    pdl_trigger();
+
+    // ---- before the wait: kv_len, the whole key range of this CTA, the RoPE rows
+    const int len = __ldcg(a.kv_len + b);
+    const int nsplit = max(1, (len + CK - 1) / CK);
+    if (len + T > a.cap || nsplit > AT_CL) {      // never write past the cache; a cache longer than the host's bound is a host error
+        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, len + T > a.cap ? (int)HS_ERR_CAPACITY : (int)HS_ERR_DEVICE);
+        return;
+    }
+    const int crank = split;                      // the grid has exactly one cluster along x
+    const bool live = split < nsplit, last = split == nsplit - 1;
+    const int c0 = split * CK, rc = live ? min(len, c0 + CK) - c0 : 0;
+    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+#pragma unroll 2
+    for (int idx = tid; idx < rc * (HD / 8); idx += AT_THREADS) {
+        const int j = idx / (HD / 8), c = idx - j * (HD / 8);
+        cp_async16(K_s + (size_t)j * KSTR + 8 * c, Kb + (size_t)(c0 + j) * HD + 8 * c);
+    }
+#pragma unroll 2
+    for (int idx = tid; idx < rc * (HD / 8); idx += AT_THREADS) {
+        const int j = idx / (HD / 8), c = idx - j * (HD / 8);
+        cp_async16(V_s + (size_t)j * KSTR + 8 * c, Vb + (size_t)(c0 + j) * HD + 8 * c);
+    }
+    cp_async_commit();
+#pragma unroll 1
+    for (int idx = tid; idx < T * (HD / 2); idx += AT_THREADS) {
+        const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+        rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
+    }
+    // query rows that do not exist are zero (their results are never stored)
+#pragma unroll 1
+    for (int idx = tid; idx < (16 - GT) * (HD / 8); idx += AT_THREADS) {
+        const int r = GT + idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4 *>(Qh_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(Ql_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+    }
+    pdl_wait();
+    __syncthreads();                        // rope_s complete
+
+    // ---- after the wait: one trip to L2 for the queries and (last key range) the raw k, v of the new positions
+    const int rowbase = lb * T;
+    const float scale = rsqrtf((float)HD);
+    constexpr int NKV = (HS_MAX_T * (HD / 2) + AT_THREADS - 1) / AT_THREADS;
+    float kraw[NKV][4];
+    if (last) {
+#pragma unroll
+        for (int it = 0; it < NKV; ++it) {
+            const int idx = tid + it * AT_THREADS;
+            kraw[it][0] = kraw[it][1] = kraw[it][2] = kraw[it][3] = 0.f;
+            if (idx < T * (HD / 2)) {
+                const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+                const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
+                kraw[it][0] = __ldcg(row + a.k_off + kh * HD + e); kraw[it][1] = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
+                kraw[it][2] = __ldcg(row + a.v_off + kh * HD + e); kraw[it][3] = __ldcg(row + a.v_off + kh * HD + e + HD / 2);
+            }
+        }
+    }
+    if (live) {
+        constexpr int HP = HD / 2, NH = AT_THREADS / HP;
+        const int e = tid % HP, part = tid / HP;
+#pragma unroll 1
+        for (int q0 = part; q0 < GT; q0 += 4 * NH) {
+            float x0[4], x1[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                x0[u] = x1[u] = 0.f;
+                if (qi < GT) {
+                    const int gq = (int)((qi * tinv) >> 16);
+                    const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                    x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                if (qi < GT) {
+                    const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
+                    __nv_bfloat16 h, l;
+                    split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                    split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
+                }
+            }
+        }
+    }
+    const int nkeys = rc + (last ? T : 0);
+    const int nkp = (nkeys + 15) & ~15;
+    if (last) {
+        // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached: appended to the cache and placed behind
+        // the cached keys of this range
+#pragma unroll
+        for (int it = 0; it < NKV; ++it) {
+            const int idx = tid + it * AT_THREADS;
+            if (idx >= T * (HD / 2)) break;
+            const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+            const float2 cs = rope_s[idx];
+            const float x0 = kraw[it][0], x1 = kraw[it][1];
+            const __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * cs.x - x1 * cs.y);
+            const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(kraw[it][2]);
+            const __nv_bfloat16 v1 = __float2bfloat16_rn(kraw[it][3]);
+            K_s[(size_t)(rc + i) * KSTR + e] = k0; K_s[(size_t)(rc + i) * KSTR + e + HD / 2] = k1;
+            V_s[(size_t)(rc + i) * KSTR + e] = v0; V_s[(size_t)(rc + i) * KSTR + e + HD / 2] = v1;
+            Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
+            Vb[(size_t)(len + i) * HD + e] = v0; Vb[(size_t)(len + i) * HD + e + HD / 2] = v1;
+        }
+    }
+    // V rows of the padding keys must be finite: their probabilities are zero, and 0 * NaN is not
+#pragma unroll 1
+    for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += AT_THREADS) {
+        const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4 *>(V_s + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+    }
+    cp_async_wait_all();
+    __syncthreads();                        // keys, values, queries in place: the last block-wide barrier
+
+    // ---- per warp: 16 keys at a time, probabilities in registers, running softmax, partial output over all of HD
+    const int g8 = lane >> 2, t4 = lane & 3;
+    constexpr int NT = HD / 8;
+    float O[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { O[nt][0] = O[nt][1] = O[nt][2] = O[nt][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};      // rows g8 and g8 + 8
+    const int ti0 = g8 - (int)((g8 * tinv) >> 16) * T, ti1 = (g8 + 8) - (int)(((g8 + 8) * tinv) >> 16) * T;   // position index of the two rows
+#pragma unroll 1
+    for (int kb = warp * 16; kb < nkp; kb += AT_WARPS * 16) {
+        float S[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) { S[nt][0] = S[nt][1] = S[nt][2] = S[nt][3] = 0.f; }
+#pragma unroll 2
+        for (int ks = 0; ks < HD / 16; ++ks) {
+            uint32_t bk[4], ah[4], al[4];
+            ldsm_x4(bk, K_s + (size_t)(kb + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
+            const size_t qo = (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
+            ldsm_x4(ah, Qh_s + qo);
+            ldsm_x4(al, Ql_s + qo);
+            mma_bf16(S[0], ah, bk[0], bk[1]); mma_bf16(S[1], ah, bk[2], bk[3]);
+            mma_bf16(S[0], al, bk[0], bk[1]); mma_bf16(S[1], al, bk[2], bk[3]);
+        }
+        // masks: keys beyond the range and, among the new rows, later positions
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int key = kb + nt * 8 + 2 * t4 + (e & 1), ti = (e >> 1) ? ti1 : ti0;
+                if (key >= nkeys || (last && key >= rc && key - rc > ti)) S[nt][e] = -INFINITY;
+                mx[e >> 1] = fmaxf(mx[e >> 1], S[nt][e]);
+            }
+        uint32_t ph[4], pl[4];
+        float corr[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+            const float mnew = fmaxf(m_run[r], mx[r]);
+            const float muse = mnew == -INFINITY ? 0.f : mnew;         // a row that has seen no key yet: everything stays zero
+            corr[r] = __expf(m_run[r] - muse);                        // exp(-inf) = 0 on the first group
+            m_run[r] = mnew;
+            float sum = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                const float p0 = __expf(S[nt][2 * r] - muse), p1 = __expf(S[nt][2 * r + 1] - muse);
+                sum += p0 + p1;
+                __nv_bfloat16 h0, l0, h1, l1;
+                split_bf16(p0, h0, l0); split_bf16(p1, h1, l1);
+                // A fragment of P (16 rows x 16 keys): register r + 2 * nt holds row g8 + 8 r, keys 8 nt + 2 t4, + 1
+                ph[r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                pl[r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            }
+            l_run[r] = fmaf(l_run[r], corr[r], sum);
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { O[nt][0] *= corr[0]; O[nt][1] *= corr[0]; O[nt][2] *= corr[1]; O[nt][3] *= corr[1]; }
+#pragma unroll
+        for (int p = 0; p < NT / 2; ++p) {
+            uint32_t bv[4];
+            ldsm_x4_t(bv, V_s + (size_t)(kb + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + p * 16 + (lane >> 4) * 8);
+            mma_bf16(O[2 * p], ph, bv[0], bv[1]); mma_bf16(O[2 * p + 1], ph, bv[2], bv[3]);
+            mma_bf16(O[2 * p], pl, bv[0], bv[1]); mma_bf16(O[2 * p + 1], pl, bv[2], bv[3]);
+        }
+    }
+    // ---- send this warp's partial: the DS dimensions rank r finishes go to rank r, (max, sum) to every rank
+    if (live) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+        }
+        const int src = crank * AT_WARPS + warp;
+        const uint32_t acc_a = smem_u32(rx_acc) + (uint32_t)src * GT * DS * 4, ml_a = smem_u32(rx_ml) + (uint32_t)src * GT * 2 * 4;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int d = nt * 8 + 2 * t4;
+            const uint32_t dest = (uint32_t)(d / DS), off = (uint32_t)(d % DS) * 4;
+            if (g8 < GT) dsmem_st_v2(dsmem_addr(acc_a + (uint32_t)(g8 * DS) * 4 + off, dest), O[nt][0], O[nt][1]);
+            if (g8 + 8 < GT) dsmem_st_v2(dsmem_addr(acc_a + (uint32_t)((g8 + 8) * DS) * 4 + off, dest), O[nt][2], O[nt][3]);
+        }
+        if (t4 == 0) {
+#pragma unroll
+            for (int dest = 0; dest < AT_CL; ++dest) {
+                if (g8 < GT) dsmem_st_v2(dsmem_addr(ml_a + (uint32_t)g8 * 8, (uint32_t)dest), m_run[0], l_run[0]);
+                if (g8 + 8 < GT) dsmem_st_v2(dsmem_addr(ml_a + (uint32_t)(g8 + 8) * 8, (uint32_t)dest), m_run[1], l_run[1]);
+            }
+        }
+    }
+    cluster_arrive(); cluster_wait();
+    // ---- merge the partials of all warps of all live ranks for this rank's output dimensions, in source order
+    const int nsrc = min(AT_CL, nsplit) * AT_WARPS;
+    float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
+    constexpr int DV = DS / 4;
+#pragma unroll 1
+    for (int idx = tid; idx < GT * DV; idx += AT_THREADS) {
+        const int qi = idx / DV, dd = (idx - qi * DV) * 4, d = crank * DS + dd;
+        float M = -INFINITY;
+#pragma unroll 4
+        for (int sidx = 0; sidx < nsrc; ++sidx) M = fmaxf(M, rx_ml[((size_t)sidx * GT + qi) * 2]);
+        float den = 0.f;
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int sidx = 0; sidx < nsrc; ++sidx) {
+            const float2 mlv = *reinterpret_cast<const float2 *>(rx_ml + ((size_t)sidx * GT + qi) * 2);
+            const float4 v = *reinterpret_cast<const float4 *>(rx_acc + ((size_t)sidx * GT + qi) * DS + dd);
+            const float w = mlv.x == -INFINITY ? 0.f : __expf(mlv.x - M);
+            den = fmaf(w, mlv.y, den);
+            sum.x = fmaf(w, v.x, sum.x); sum.y = fmaf(w, v.y, sum.y); sum.z = fmaf(w, v.z, sum.z); sum.w = fmaf(w, v.w, sum.w);
+        }
+        const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
+        const float inv = 1.0f / den;
+        *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
+            make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
+    }
+}
+
 template <int HD, int MT>
 __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
@@ -482,13 +803,21 @@ __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
 // clusters) are attention CTAs, the rest mixer CTAs - and the dependent-launch chain is one kernel shorter.
 struct FusedGeo { int attn_nx, attn_ctas, ssm_nx, ssm_ctas; };
 
+template <int HD>
+__global__ void __launch_bounds__(AT_THREADS) attn_small_kernel(const AttnArgs a) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    attn_small_body<HD>(a, blockIdx.x, blockIdx.y, blockIdx.z, smraw);
+}
+
+// MT = 0 selects the latency-lean attention body (few query rows, cache within one cluster)
 template <int EPL, int HD, int MT, int TMAX>
 __global__ void __launch_bounds__(AT_THREADS) ssm_attn_kernel(const SsmArgs sa, const AttnArgs aa, const FusedGeo g) {
     extern __shared__ __align__(128) unsigned char smraw[];
     const int id = blockIdx.x;
     if (id < g.attn_ctas) {
         const int split = id % g.attn_nx, t = id / g.attn_nx;
-        attn_body<HD, MT>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
+        if (MT == 0) attn_small_body<HD>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
+        else attn_body<HD, MT == 0 ? 1 : MT>(aa, split, t % aa.kvh, t / aa.kvh, smraw);
     } else if (id - g.attn_ctas < g.ssm_ctas) {
         const int j = id - g.attn_ctas, bx = j % g.ssm_nx, t = j / g.ssm_nx;
         ssm_body<EPL, 16, TMAX>(sa, bx, t % sa.H, t / sa.H);
@@ -502,18 +831,32 @@ cudaError_t launch_t(const AttnArgs &a, cudaStream_t s) {
     return launch_pdl_cluster(attn_kernel<HD, MT>, grid, dim3(AT_THREADS), smem, s, AT_CL, a);
 }
 
+template <int HD>
+cudaError_t launch_small_t(const AttnArgs &a, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_small_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_small_layout(HD, AT_SMALL_MAXCHUNK, 16).total);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_small_kernel<HD>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const size_t smem = attn_small_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
+    return launch_pdl_cluster(attn_small_kernel<HD>, dim3(AT_CL, a.kvh, a.nb), dim3(AT_THREADS), smem, s, AT_CL, a);
+}
+
 template <int EPL, int HD, int MT, int TMAX>
 cudaError_t launch_fused_t(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s) {
     FusedGeo g;
-    g.attn_nx = (a.nch + AT_CL - 1) / AT_CL * AT_CL;
+    g.attn_nx = MT == 0 ? AT_CL : (a.nch + AT_CL - 1) / AT_CL * AT_CL;
     g.attn_ctas = g.attn_nx * a.kvh * a.nb;
     g.ssm_nx = sa.P / 16;
     g.ssm_ctas = g.ssm_nx * sa.H * sa.nb;
     const int total = (g.attn_ctas + g.ssm_ctas + AT_CL - 1) / AT_CL * AT_CL;
-    const size_t smem = attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
+    const size_t smem = MT == 0 ? attn_small_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total : attn_layout(HD, a.chunk, (a.qh / a.kvh) * a.T).total;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT, TMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_layout(HD, 128, MT * 16).total);
+        const size_t most = MT == 0 ? attn_small_layout(HD, AT_SMALL_MAXCHUNK, 16).total : attn_layout(HD, 128, MT * 16).total;
+        cudaError_t e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT, TMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(ssm_attn_kernel<EPL, HD, MT, TMAX>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -542,6 +885,10 @@ cudaError_t configure_attn() {
 
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     const int GT = (a.qh / a.kvh) * a.T;
+    if (a.small) {
+        if (GT > 16 || a.chunk < 16 || a.chunk > AT_SMALL_MAXCHUNK || (a.chunk & 15)) return cudaErrorInvalidValue;
+        return a.hd == 128 ? launch_small_t<128>(a, s) : a.hd == 64 ? launch_small_t<64>(a, s) : cudaErrorInvalidValue;
+    }
     if (GT > HS_MAX_GT || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || a.tiles < 1) return cudaErrorInvalidValue;
     const int mt = (GT + 15) / 16;
 #define CASE(hd_, m_) if (a.hd == hd_ && mt == m_) return launch_t<hd_, m_>(a, s)
@@ -554,11 +901,12 @@ cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
 // 16 state rows, 128 threads in both roles) - otherwise nothing is launched and the caller issues the two
 // kernels one after the other.
 cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s, bool *fused) {
-    const int GT = (a.qh / a.kvh) * a.T, mt = (GT + 15) / 16;
+    const int GT = (a.qh / a.kvh) * a.T, mt = a.small ? 0 : (GT + 15) / 16;
     *fused = false;
     if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || sa.P % 16) return cudaSuccess;
+    if (a.small && GT > 16) return cudaErrorInvalidValue;
 #define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return a.T <= 3 ? launch_fused_t<e_, hd_, m_, 3>(sa, a, s) : launch_fused_t<e_, hd_, m_, HS_MAX_T>(sa, a, s); }
-#define CASES(n_, e_) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)
+#define CASES(n_, e_) CASE(n_, e_, 128, 0) CASE(n_, e_, 64, 0) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)
     CASES(64, 2) CASES(128, 4) CASES(256, 8)
 #undef CASES
 #undef CASE

@@ -21,6 +21,8 @@
 // Epilogues: plain store, residual add (with K split), SwiGLU over interleaved gate/up rows.
 #include "hs_internal.h"
 #include "hs_device.cuh"
+#include <cstdio>
+#include <cstdlib>
 
 namespace {
 using namespace hsd;
@@ -42,7 +44,40 @@ struct GemvGeo {
     int rq, rrem;        // row ranges: units / NR and units % NR
     int nch;             // chunks of a full K range
     long long pf_per;    // bytes of the next projection's weights each CTA pulls into L2
+    int cl, off_part;    // cl = 1: the K splits of a row range form a thread-block cluster and reduce their partial sums
+                         // through distributed shared memory (one part out); off_part: [rows of the range][16] floats
 };
+
+// Residual epilogue with the K split reduced inside the cluster.  Every CTA has left the partial sums of its K
+// range in part_s[local output row][activation row]; the S CTAs of the cluster (rank = K split index) share the
+// row range.  Rank q finishes a contiguous share of the rows: partials added in rank order, then the residual -
+// a fixed order, so the result does not depend on timing.  The second barrier keeps every CTA's shared memory
+// alive until its peers have read it.
+template <int THREADS>
+__device__ __forceinline__ void cluster_reduce_resid(const GemvArgs &a, float *part_s, int S, int q, int r0, int nrow, int nrows) {
+    __syncthreads();
+    cluster_arrive(); cluster_wait();
+    const int lo = nrow * q / S, nloc = nrow * (q + 1) / S - lo;
+#pragma unroll 1
+    for (int idx = threadIdx.x; idx < nloc * nrows; idx += THREADS) {
+        const int xr = idx / nloc, row = lo + idx - xr * nloc;            // consecutive threads: consecutive outputs
+        const size_t oi = (size_t)xr * a.ldo + r0 + row;
+        float res[HS_H_PARTS];
+#pragma unroll
+        for (int p = 0; p < HS_H_PARTS; ++p) res[p] = p < a.rparts ? __ldcg(a.resid + (size_t)p * a.rpstride + oi) : 0.f;
+        const uint32_t local = smem_u32(part_s + row * GV_MAXROWS + xr);
+        float v[HS_H_PARTS];
+#pragma unroll
+        for (int p = 0; p < HS_H_PARTS; ++p) v[p] = p < S ? dsmem_ld_f32(dsmem_addr(local, (uint32_t)p)) : 0.f;
+        float sum = v[0];
+#pragma unroll
+        for (int p = 1; p < HS_H_PARTS; ++p) sum += v[p];
+#pragma unroll
+        for (int p = 0; p < HS_H_PARTS; ++p) sum += res[p];
+        a.out[oi] = sum;
+    }
+    cluster_arrive(); cluster_wait();
+}
 
 __device__ __forceinline__ float dot8(const uint4 &w, const float4 &a, const float4 &b, float acc) {
     acc = fmaf(bf_lo(w.x), a.x, acc); acc = fmaf(bf_hi(w.x), a.y, acc);
@@ -304,7 +339,8 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
 }
 
 // EPI / NORMED >= 0 fix the epilogue and the presence of a norm at compile time (shorter program, see above).
-template <int NG, int EPI = -1, int NORMED = -1>
+// CL: residual epilogue with the K split reduced inside a thread-block cluster (cluster_reduce_resid).
+template <int NG, int EPI = -1, int NORMED = -1, bool CL = false>
 __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs a, const GemvGeo g, int32_t *status) {
     constexpr int WR = 8;
     extern __shared__ __align__(128) unsigned char smraw[];
@@ -461,7 +497,7 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
         for (int gq = 0; gq < NG; ++gq) {
             res[gq][0] = res[gq][1] = 0.f;
             const int xr = gq * 8 + g8;
-            if (epi == EPI_RESID && si == 0 && xr < nrows)
+            if (!CL && epi == EPI_RESID && si == 0 && xr < nrows)
 #pragma unroll
                 for (int e = 0; e < 2; ++e)
                     if (2 * t4 + e < rows_in)
@@ -521,18 +557,22 @@ __global__ void __launch_bounds__(GV_THREADS, 2) gemm_mma_kernel(const GemvArgs 
                 for (int e = 0; e < 2; ++e)
                     if (2 * t4 + e < rows_in) {
                         const size_t oi = (size_t)xr * a.ldo + wrow + e;
-                        if (epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = v[e] + res[gq][e];
+                        if (CL) reinterpret_cast<float *>(smraw + g.off_part)[(wrow + e - r0) * GV_MAXROWS + xr] = v[e];
+                        else if (epi == EPI_RESID) a.out[(size_t)si * a.opstride + oi] = v[e] + res[gq][e];
                         else a.out[oi] = v[e];
                     }
             }
         }
     }
+    if (CL) cluster_reduce_resid<GV_THREADS>(a, reinterpret_cast<float *>(smraw + g.off_part), (int)gridDim.x, si, r0, nrow, nrows);
     if (bad) atomicCAS(status, 0, (int)HS_ERR_TIMEOUT);     // a copy never landed
 }
 
 int g_sms = 148;
+int g_max_clusters[HS_H_PARTS + 1] = {0, 0, 0, 0, 0};   // resident clusters by cluster size (0: clusters unavailable)
 }  // namespace
 bool g_hs_gemm_mma = true;
+bool g_hs_cluster_reduce = true;   // residual projections of 4..16 rows reduce their K split inside a thread-block cluster
 namespace {
 constexpr size_t GV_SMEM_MAX = 224 * 1024;
 constexpr size_t GV_SMEM_PAIR = 127 * 1024;   // below this the CTA of the next kernel fits beside it
@@ -541,6 +581,10 @@ template <int NG>
 cudaError_t launch_mma(const GemvArgs &a, const GemvGeo &g, size_t smem, int32_t *status, cudaStream_t s) {
     const dim3 grid(g.S0 + g.S1, g.NR), block(GV_THREADS);
     const int nm = a.norm_w ? 1 : 0;
+    if (g.cl) {
+        if (nm) return launch_pdl_cluster(gemm_mma_kernel<NG, EPI_RESID, 1, true>, grid, block, smem, s, (int)grid.x, a, g, status);
+        return launch_pdl_cluster(gemm_mma_kernel<NG, EPI_RESID, 0, true>, grid, block, smem, s, (int)grid.x, a, g, status);
+    }
 #define MM(ep, n) if (a.epi == ep && nm == n) return launch_pdl(gemm_mma_kernel<NG, ep, n>, grid, block, smem, s, a, g, status)
     MM(EPI_STORE, 1); MM(EPI_STORE, 0); MM(EPI_RESID, 1); MM(EPI_RESID, 0); MM(EPI_SWIGLU, 1); MM(EPI_SWIGLU, 0);
 #undef MM
@@ -585,6 +629,24 @@ cudaError_t configure_gemv() {
     CFGM6(1); CFGM6(2);
 #undef CFGM6
 #undef CFGM
+#define CFGC(n, nm) if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, EPI_RESID, nm, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GV_SMEM_MAX); \
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_mma_kernel<n, EPI_RESID, nm, true>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+    CFGC(1, 0); CFGC(1, 1); CFGC(2, 0); CFGC(2, 1);
+#undef CFGC
+    // how many clusters of 2, 3, 4 CTAs the GPU runs at once with one such CTA per SM: the CTAs of a cluster share a
+    // GPC, so this can be fewer than SMs / size; row ranges are sized so that every cluster is resident at once
+    for (int S = 2; S <= HS_H_PARTS && e == cudaSuccess; ++S) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(S, g_sms / S); cfg.blockDim = dim3(GV_THREADS); cfg.dynamicSmemBytes = GV_SMEM_MAX;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = S; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_mma_kernel<2, EPI_RESID, 1, true>, &cfg) == cudaSuccess && n > 0) g_max_clusters[S] = n;
+        else { g_max_clusters[S] = 0; cudaGetLastError(); }
+        if (getenv("HS_VERBOSE")) fprintf(stderr, "libhs: clusters of %d CTAs resident at once: %d\n", S, g_max_clusters[S]);
+    }
     return e;
 }
 
@@ -639,6 +701,10 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     const int S = g.S0 + g.S1;
     const int units = a.O / g.unit;
     g.NR = g_sms / S;
+    // many activation rows: the consumers of a split residual stream re-add its parts for every row in every CTA,
+    // which costs more than reducing the K split here, inside a cluster
+    g.cl = (g_hs_cluster_reduce && mma && a.epi == EPI_RESID && S > 1 && S <= HS_H_PARTS && g_max_clusters[S] > 0) ? 1 : 0;
+    if (g.cl && g.NR > g_max_clusters[S]) g.NR = g_max_clusters[S];
     if (g.NR < 1) g.NR = 1;
     if (g.NR > units) g.NR = units;
     const int nrow_max = ceil_div(units, g.NR) * g.unit;
@@ -668,9 +734,10 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
     const size_t budget = g.off_ring + tile * GV_WARPS > GV_SMEM_PAIR ? GV_SMEM_MAX : GV_SMEM_PAIR;   // no room for a neighbour anyway: go deep
     while (D < GV_MAXDEPTH && D < tiles_per_warp && g.off_ring + tile * GV_WARPS * (D + 1) <= budget) ++D;
     g.D = D;
-    const size_t smem = g.off_ring + tile * ring_warps * D;
+    size_t smem = g.off_ring + tile * ring_warps * D;
+    if (g.cl) { g.off_part = (int)((smem + 127) / 128 * 128); smem = g.off_part + (size_t)nrow_max * GV_MAXROWS * 4; }
     if (smem > GV_SMEM_MAX) return a.nrows > 1 ? rows_launch((a.nrows + 1) / 2) : cudaErrorInvalidValue;
-    if (oparts) *oparts = a.epi == EPI_RESID ? S : 1;
+    if (oparts) *oparts = (a.epi == EPI_RESID && !g.cl) ? S : 1;
     if (launches) ++*launches;
     if (mma) return NG == 1 ? launch_mma<1>(a, g, smem, status, s) : launch_mma<2>(a, g, smem, status, s);
     if (a.nrows <= 3) {
