@@ -592,12 +592,14 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
         *reinterpret_cast<uint4 *>(Qh_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4 *>(Ql_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
     }
+    const int rowbase = lb * T;
+    const float scale = rsqrtf((float)HD);
+    const int nkeys = rc + (last ? T : 0);
+    const int nkp = (nkeys + 15) & ~15;
     pdl_wait();
     __syncthreads();                        // rope_s complete
 
     // ---- after the wait: one trip to L2 for the queries and (last key range) the raw k, v of the new positions
-    const int rowbase = lb * T;
-    const float scale = rsqrtf((float)HD);
     constexpr int NKV = (HS_MAX_T * (HD / 2) + AT_THREADS - 1) / AT_THREADS;
     float kraw[NKV][4];
     if (last) {
@@ -614,37 +616,33 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
         }
     }
     if (live) {
-        constexpr int HP = HD / 2, NH = AT_THREADS / HP;
+        // thread = (rotation pair e, one of NH interleaved sets of query rows); every load is issued before the first use
+        constexpr int HP = HD / 2, NH = AT_THREADS / HP, U = 16 / NH;
         const int e = tid % HP, part = tid / HP;
-#pragma unroll 1
-        for (int q0 = part; q0 < GT; q0 += 4 * NH) {
-            float x0[4], x1[4];
+        float x0[U], x1[U];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int qi = q0 + u * NH;
-                x0[u] = x1[u] = 0.f;
-                if (qi < GT) {
-                    const int gq = (int)((qi * tinv) >> 16);
-                    const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
-                    x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
-                }
+        for (int u = 0; u < U; ++u) {
+            const int qi = part + u * NH;
+            x0[u] = x1[u] = 0.f;
+            if (qi < GT) {
+                const int gq = (int)((qi * tinv) >> 16);
+                const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
             }
+        }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int qi = q0 + u * NH;
-                if (qi < GT) {
-                    const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
-                    __nv_bfloat16 h, l;
-                    split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
-                    Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
-                    split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
-                    Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
-                }
+        for (int u = 0; u < U; ++u) {
+            const int qi = part + u * NH;
+            if (qi < GT) {
+                const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
+                __nv_bfloat16 h, l;
+                split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
+                Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
+                Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
             }
         }
     }
-    const int nkeys = rc + (last ? T : 0);
-    const int nkp = (nkeys + 15) & ~15;
     if (last) {
         // new K (RoPE) and V rows, rounded to bf16 exactly as they are cached: appended to the cache and placed behind
         // the cached keys of this range
@@ -684,19 +682,27 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
     const int ti0 = g8 - (int)((g8 * tinv) >> 16) * T, ti1 = (g8 + 8) - (int)(((g8 + 8) * tinv) >> 16) * T;   // position index of the two rows
 #pragma unroll 1
     for (int kb = warp * 16; kb < nkp; kb += AT_WARPS * 16) {
-        float S[2][4];
+        // scores: the k steps feed four accumulator sets in turn, so that a chain of dependent MMAs is 4 long, not 16
+        float Sp[4][2][4];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) { S[nt][0] = S[nt][1] = S[nt][2] = S[nt][3] = 0.f; }
-#pragma unroll 2
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) { Sp[c][nt][0] = Sp[c][nt][1] = Sp[c][nt][2] = Sp[c][nt][3] = 0.f; }
+#pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
             uint32_t bk[4], ah[4], al[4];
             ldsm_x4(bk, K_s + (size_t)(kb + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
             const size_t qo = (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
             ldsm_x4(ah, Qh_s + qo);
             ldsm_x4(al, Ql_s + qo);
-            mma_bf16(S[0], ah, bk[0], bk[1]); mma_bf16(S[1], ah, bk[2], bk[3]);
-            mma_bf16(S[0], al, bk[0], bk[1]); mma_bf16(S[1], al, bk[2], bk[3]);
+            mma_bf16(Sp[(2 * ks) & 3][0], ah, bk[0], bk[1]); mma_bf16(Sp[(2 * ks) & 3][1], ah, bk[2], bk[3]);
+            mma_bf16(Sp[(2 * ks + 1) & 3][0], al, bk[0], bk[1]); mma_bf16(Sp[(2 * ks + 1) & 3][1], al, bk[2], bk[3]);
         }
+        float S[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) S[nt][e] = (Sp[0][nt][e] + Sp[1][nt][e]) + (Sp[2][nt][e] + Sp[3][nt][e]);
         // masks: keys beyond the range and, among the new rows, later positions
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
@@ -769,26 +775,46 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
     const int nsrc = min(AT_CL, nsplit) * AT_WARPS;
     float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
     constexpr int DV = DS / 4;
+    // an output = (query row, four dimensions); a group of LPO lanes (a power of two, as many as the block affords)
+    // shares the sources of one output and folds its partial results with shuffles - the order is fixed by the lane
+    // numbers, so the result does not depend on timing
+    const int nout = GT * DV;
+    int lsh = 0;
+    while (lsh < 5 && (nout << (lsh + 1)) <= AT_THREADS) ++lsh;
+    const int LPO = 1 << lsh, sub = tid & (LPO - 1);
 #pragma unroll 1
-    for (int idx = tid; idx < GT * DV; idx += AT_THREADS) {
-        const int qi = idx / DV, dd = (idx - qi * DV) * 4, d = crank * DS + dd;
+    for (int o0 = 0; o0 < nout; o0 += AT_THREADS >> lsh) {
+        const int oi = o0 + (tid >> lsh);
+        const bool valid = oi < nout;
+        const int oc = valid ? oi : 0;
+        const int qi = oc / DV, dd = (oc - qi * DV) * 4, d = crank * DS + dd;
         float M = -INFINITY;
 #pragma unroll 4
-        for (int sidx = 0; sidx < nsrc; ++sidx) M = fmaxf(M, rx_ml[((size_t)sidx * GT + qi) * 2]);
+        for (int sidx = sub; sidx < nsrc; sidx += LPO) M = fmaxf(M, rx_ml[((size_t)sidx * GT + qi) * 2]);
+#pragma unroll 1
+        for (int w = LPO >> 1; w >= 1; w >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, w));
         float den = 0.f;
         float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-        for (int sidx = 0; sidx < nsrc; ++sidx) {
+        for (int sidx = sub; sidx < nsrc; sidx += LPO) {
             const float2 mlv = *reinterpret_cast<const float2 *>(rx_ml + ((size_t)sidx * GT + qi) * 2);
             const float4 v = *reinterpret_cast<const float4 *>(rx_acc + ((size_t)sidx * GT + qi) * DS + dd);
             const float w = mlv.x == -INFINITY ? 0.f : __expf(mlv.x - M);
             den = fmaf(w, mlv.y, den);
             sum.x = fmaf(w, v.x, sum.x); sum.y = fmaf(w, v.y, sum.y); sum.z = fmaf(w, v.z, sum.z); sum.w = fmaf(w, v.w, sum.w);
         }
-        const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
-        const float inv = 1.0f / den;
-        *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
-            make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
+#pragma unroll 1
+        for (int w = LPO >> 1; w >= 1; w >>= 1) {
+            den += __shfl_xor_sync(0xffffffffu, den, w);
+            sum.x += __shfl_xor_sync(0xffffffffu, sum.x, w); sum.y += __shfl_xor_sync(0xffffffffu, sum.y, w);
+            sum.z += __shfl_xor_sync(0xffffffffu, sum.z, w); sum.w += __shfl_xor_sync(0xffffffffu, sum.w, w);
+        }
+        if (valid && sub == 0) {
+            const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
+            const float inv = 1.0f / den;
+            *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
+                make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
+        }
     }
 }
 
