@@ -412,9 +412,12 @@ def run_ours(args):
     # ---- the other workloads (rank 0, single GPU): each from an injected context, one clock record per leg
     by_config = {}
     if world == 1 and args.by_config and args.config == "cfg2_0p5b":
-        plan = [("cfg3_3b", 1, (2, 4)), ("cfg3_3b", 8, (4,)), ("cfg4_seq", 1, (2, 4)), ("cfg5_b64", 64, (4,))]
+        # (workload, batch, draft lengths, extra flags): the batched workloads also with rollback by replay
+        # (HS_FLAG_REPLAY: an update log instead of k + 1 state snapshots per verify pass)
+        plan = [("cfg3_3b", 1, (2, 4), 0), ("cfg3_3b", 8, (4,), 0), ("cfg3_3b", 8, (4,), hs.HS_FLAG_REPLAY),
+                ("cfg4_seq", 1, (2, 4), 0), ("cfg5_b64", 64, (4,), 0), ("cfg5_b64", 64, (4,), hs.HS_FLAG_REPLAY)]
         blobs = {"cfg2_0p5b": blob}
-        for name, nb, kset in plan:
+        for name, nb, kset, xflags in plan:
             sc = hi.CONFIGS[name]
             arch = lambda c: (c.arch, c.L, c.d, c.V, c.H, c.P, c.N, c.qh, c.kvh, c.hd, c.ff, c.gh, c.gdk, c.gdv)
             if name not in blobs:
@@ -427,16 +430,22 @@ def run_ours(args):
             lens_c = hi.context_lengths(nb, 4096, 16384) if name == "cfg5_b64" else np.full(nb, sc.prompt_len, np.int32)
             mk = max(kset)
             cap_c = int(lens_c.max()) + (steps + warm + 4) * (mk + 1) + 64
-            e = hs.Engine(sc, blobs[name], max_batch=nb, max_k=mk, kv_capacity=cap_c, flags=hs.HS_FLAG_GRAPHS, device=str(dev))
+            e = hs.Engine(sc, blobs[name], max_batch=nb, max_k=mk, kv_capacity=cap_c, flags=hs.HS_FLAG_GRAPHS | xflags, device=str(dev))
             restore = inject_random_context(torch, e, sc, nb, lens_c)
-            entry = {"batch": nb, "context": "injected, lengths %d..%d (mean %.0f)" % (lens_c.min(), lens_c.max(), lens_c.mean())}
+            entry = {"batch": nb, "context": "injected, lengths %d..%d (mean %.0f)" % (lens_c.min(), lens_c.max(), lens_c.mean()),
+                     "rollback": "replay log" if xflags & hs.HS_FLAG_REPLAY else "state snapshots"}
+            unit = 4.0 * nb * sum((sc.H * sc.P * sc.N if sc.layer_type(l) == hi.LAYER_PAR else sc.gh * sc.gdv * sc.gdk)
+                                  for l in range(sc.L) if sc.layer_type(l) != hi.LAYER_ATT)        # bytes of all recurrent states
             for kk in kset:
                 smp = ClockSampler(local_rank); smp.start()
                 r = legs.timed(e, nb, kk, restore, float(lens_c.mean()))
                 rep = legs.report(sc, nb, kk, r, peak)
                 rep["clocks"] = smp.stop()
+                # recurrent-state bytes one round really moves in its verify + rollback: snapshots: read 1, write k + 1;
+                # replay: read 1 in verify, read 1 + write 1 in the replay kernel (the algorithmic figure counts 2)
+                rep["state_traffic_bytes_per_round"] = unit * (3 if xflags & hs.HS_FLAG_REPLAY else kk + 2)
                 entry["k%d" % kk] = rep
-            by_config["%s_b%d" % (name, nb)] = entry
+            by_config["%s@b%d%s" % (name, nb, "+replay" if xflags & hs.HS_FLAG_REPLAY else "")] = entry
             e.close()
             del e
             torch.cuda.empty_cache()

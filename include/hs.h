@@ -67,13 +67,19 @@ typedef struct hs_config {
 } hs_config;
 
 enum {
-    HS_FLAG_GRAPHS = 1         /* replay each (mode, k, batch) step as a captured CUDA graph */
+    HS_FLAG_GRAPHS = 1,        /* replay each (mode, k, batch) step as a captured CUDA graph */
+    HS_FLAG_REPLAY = 2         /* rollback by replay: verify keeps no per-position state snapshots but a small log of
+                                  the k+1 state updates (Mamba-2: decay, dt*x, B; DeltaNet: alpha, beta, k, v), and
+                                  hs_accept_rollback applies the accepted n+1 updates to the committed state in place.
+                                  State traffic per verify round: 3 state units (read, read, write) instead of k+2;
+                                  the snapshot buffer shrinks to one state per sequence plus the log.  Same results. */
 };
 
 /* Bytes the caller must provide (each buffer 256-byte aligned). */
 typedef struct hs_sizes {
     int64_t weights;           /* weight blob, format below */
-    int64_t snap;              /* recurrent-state snapshots [rec layer][seq][max_k+1][state] fp32 */
+    int64_t snap;              /* recurrent-state snapshots [rec layer][seq][max_k+1][state] fp32; with HS_FLAG_REPLAY:
+                                  committed states [rec layer][seq][state], then the update log [rec layer][seq][max_k+1][w] */
     int64_t dstate;            /* draft scratch state       [rec layer][seq][state] fp32 */
     int64_t conv;              /* conv windows: committed, per-position history, draft ping-pong, fp32 */
     int64_t kv;                /* K then V: [attn layer][seq][kv head][kv_capacity][hd] bf16 each */

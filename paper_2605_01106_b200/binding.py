@@ -15,6 +15,7 @@ _LIB = None
 i32, i64, f32, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p
 
 HS_FLAG_GRAPHS = 1
+HS_FLAG_REPLAY = 2
 STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",

@@ -95,6 +95,7 @@ bool valid_config(const hs_config &c) {
 
 struct Derived {
     int B, Tm, R, n_rl, n_al, convd, gw, in_rows_max, att_chunk, att_nch;
+    int nslot, log_w;         // state slots per (layer, sequence); floats of one logged update (rollback by replay)
     int64_t state_elems;
 };
 
@@ -112,6 +113,9 @@ Derived derive(const hs_config &c) {
     v.convd = conv_channels(c);
     v.gw = c.arch == HS_ARCH_PARALLEL ? d_inner(c) : c.gh * c.gdv;
     v.state_elems = c.arch == HS_ARCH_PARALLEL ? (int64_t)c.H * c.P * c.N : (int64_t)c.gh * c.gdv * c.gdk;
+    const bool replay = (c.flags & HS_FLAG_REPLAY) != 0;
+    v.nslot = replay ? 1 : v.Tm;
+    v.log_w = !replay ? 0 : c.arch == HS_ARCH_PARALLEL ? c.H + c.H * c.P + c.N : c.gh * (2 + c.gdk + c.gdv);
     // keys per attention CTA: the largest of 128 / 64 / 32 that still gives about two CTAs per SM
     int chunk = 128;
     while (chunk > 32 && (int64_t)c.max_batch * c.kvh * ((c.kv_capacity + chunk - 1) / chunk) < 296) chunk >>= 1;
@@ -262,9 +266,14 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 win_out = m->dcw + (step & 1) * half + lrB * 3 * m->convd;
             }
             const float *st_in; int64_t in_seq, in_slot; float *st_out; int64_t out_seq, out_slot;
-            float *snap_l = m->snap + lrB * m->Tm * se, *dst_l = m->dstate + lrB * se;
-            if (!draft) { st_in = snap_l; in_seq = m->Tm * se; in_slot = se; st_out = snap_l; out_seq = m->Tm * se; out_slot = se; }
-            else if (step == 0) { st_in = snap_l; in_seq = m->Tm * se; in_slot = se; st_out = dst_l; out_seq = se; out_slot = 0; }
+            // snapshots: slot i of (layer, sequence) holds the state after position i and `slot` names the committed one;
+            // rollback by replay: one slot, the committed state, and the verify pass writes the update log instead
+            const int64_t ns = m->nslot;
+            const bool replay = m->log_w != 0;
+            float *snap_l = m->snap + lrB * ns * se, *dst_l = m->dstate + lrB * se;
+            float *log_l = (!draft && replay) ? m->ulog + lrB * m->Tm * m->log_w : nullptr;
+            if (!draft) { st_in = snap_l; in_seq = ns * se; in_slot = replay ? 0 : se; st_out = snap_l; out_seq = ns * se; out_slot = replay ? 0 : se; }
+            else if (step == 0) { st_in = snap_l; in_seq = ns * se; in_slot = replay ? 0 : se; st_out = dst_l; out_seq = se; out_slot = 0; }
             else { st_in = dst_l; in_seq = se; in_slot = 0; st_out = dst_l; out_seq = se; out_slot = 0; }
             if (ly.type == HS_LAYER_PAR) {
                 SsmArgs sa{};
@@ -274,6 +283,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 sa.state_in = st_in; sa.in_seq_stride = in_seq; sa.in_slot_stride = in_slot;
                 sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
                 sa.slot = m->ctrl.slot; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
+                sa.log = log_l; sa.log_w = m->log_w;
                 if (with_attn) { ssm_args = sa; ssm_deferred = true; }      // goes out together with the attention
                 else PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
             } else {
@@ -284,6 +294,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 gd.state_in = st_in; gd.in_seq_stride = in_seq; gd.in_slot_stride = in_slot;
                 gd.state_out = st_out; gd.out_seq_stride = out_seq; gd.out_slot_stride = out_slot;
                 gd.slot = m->ctrl.slot; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
+                gd.log = log_l; gd.log_w = m->log_w;
                 PROF(HS_PROF_MIXER, 0, launch_gdn(gd, s), "gdn");
             }
             if (!ssm_deferred) ++m->launches;
@@ -375,9 +386,18 @@ int enqueue_draft(hs_model *m, int k, int b0, int nb) {
 int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const int32_t *fx) {
     AcceptArgs a{};
     a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd; a.V = m->c.V;
-    a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist;
+    a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist; a.replay = m->log_w != 0;
     PROF(HS_PROF_ACCEPT, 0, launch_accept(a, m->stream), "accept");
     ++m->launches;
+    if (m->log_w && m->n_rl > 0) {
+        // rollback by replay: the accepted updates go into the committed state, every recurrent layer in one launch
+        ReplayArgs r{};
+        r.arch = m->c.arch; r.H = m->c.H; r.P = m->c.P; r.N = m->c.N; r.di = m->di; r.gh = m->c.gh; r.dk = m->c.gdk; r.dv = m->c.gdv;
+        r.state = m->snap; r.log = m->ulog; r.log_w = m->log_w; r.n_acc = m->ctrl.n_acc; r.state_elems = m->state_elems;
+        r.n_rl = m->n_rl; r.B = m->B; r.Tm = m->Tm; r.b0 = b0; r.nb = nb;
+        PROF(HS_PROF_ACCEPT, 0, launch_replay(r, m->stream), "replay");
+        ++m->launches;
+    }
     return HS_OK;
 }
 
@@ -424,7 +444,7 @@ int hs_query_sizes(const hs_config *cfg, hs_sizes *out) {
     const hs_config &c = *cfg;
     Derived v = derive(c);
     out->weights = blob_offset(c, c.L, 0);
-    out->snap = up((int64_t)4 * v.n_rl * v.B * v.Tm * v.state_elems);
+    out->snap = up((int64_t)4 * v.n_rl * v.B * (v.nslot * v.state_elems + (int64_t)v.Tm * v.log_w));
     out->dstate = up((int64_t)4 * v.n_rl * v.B * v.state_elems);
     out->conv = up((int64_t)4 * v.n_rl * v.B * v.convd * (3 + v.Tm + 6));
     out->kv = up((int64_t)2 * 2 * v.n_al * v.B * c.kvh * c.kv_capacity * c.hd);
@@ -462,6 +482,7 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->B = v.B; m->Tm = v.Tm; m->batch = 0; m->di = d_inner(c); m->convd = v.convd; m->gw = v.gw;
     m->n_rl = v.n_rl; m->n_al = v.n_al; m->state_elems = v.state_elems; m->in_rows_max = v.in_rows_max;
     m->att_chunk = v.att_chunk; m->att_nch = v.att_nch; m->att_force_chunk = m->att_force_tiles = 0;
+    m->nslot = v.nslot; m->log_w = v.log_w;
     m->phase = 0; m->last_k = -1; m->last_rows = 0; m->launches = 0; m->prof = false;
     m->kv_upper.assign(v.B, 0);
     const char *wb = (const char *)bufs->weights;
@@ -501,6 +522,7 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->Kc = (__nv_bfloat16 *)bufs->kv;
     m->Vc = m->Kc + (size_t)v.n_al * v.B * c.kvh * c.kv_capacity * c.hd;
     m->snap = (float *)bufs->snap; m->dstate = (float *)bufs->dstate;
+    m->ulog = m->log_w ? m->snap + (size_t)v.n_rl * v.B * v.nslot * v.state_elems : nullptr;
     CK(configure_gemv(), "configure gemv");
     CK(configure_attn(), "configure attention");
     if (configure_gemm_tc() != cudaSuccess) { g_hs_gemm_tc = false; cudaGetLastError(); }   // falls back to several 16-row launches
@@ -666,7 +688,7 @@ static int state_xfer(hs_model *m, int layer, int seq, int kind, void *host, int
             int32_t slot = 0;
             if (to_host) CK(cudaMemcpy(&slot, m->ctrl.slot + seq, 4, cudaMemcpyDeviceToHost), "slot read");
             else CK(cudaMemcpy(m->ctrl.slot + seq, &slot, 4, cudaMemcpyHostToDevice), "slot write");
-            dev = m->snap + (((size_t)ly.rl * m->B + seq) * m->Tm + slot) * m->state_elems;
+            dev = m->snap + (((size_t)ly.rl * m->B + seq) * m->nslot + (m->log_w ? 0 : slot)) * m->state_elems;
         }
         CK(to_host ? cudaMemcpy(host, dev, bytes, dir) : cudaMemcpy(dev, host, bytes, dir), "state copy");
         return HS_OK;

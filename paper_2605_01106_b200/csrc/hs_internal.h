@@ -48,6 +48,9 @@ struct hs_model {
     hs_buffers bufs;
     cudaStream_t stream;
     int B, Tm;                // max_batch, max_k + 1
+    int nslot;                // state slots per (layer, sequence): Tm (snapshots) or 1 (rollback by replay)
+    int log_w;                // floats of one logged update (replay mode), else 0
+    float *ulog;              // [n_rl][B][Tm][log_w] update log (replay mode)
     int batch;                // active sequences
     int di, convd, gw;        // d_inner, conv channels, width of the gated mixer output
     int n_rl, n_al;           // recurrent layers, KV layers
@@ -164,6 +167,8 @@ struct SsmArgs {
     const int32_t *slot;                // [B] committed slot (used when in_slot_stride != 0)
     float *g;                           // [rows][di] gated output y * silu(z)
     int T, Tm, b0, nb;
+    float *log; int log_w;              // verify with rollback by replay: [B][Tm][log_w] update log (decay[H] | dt*x[di] | B[N]);
+                                        // no state is stored.  NULL otherwise
 };
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s);
 
@@ -177,8 +182,22 @@ struct GdnArgs {
     const int32_t *slot;
     float *g;                           // [rows][gh*dv]
     int T, Tm, b0, nb;
+    float *log; int log_w;              // rollback by replay: [B][Tm][log_w] (alpha[gh] | beta[gh] | k[gh*dk] | v[gh*dv]); NULL otherwise
 };
 cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s);
+
+// Rollback by replay: apply the first n_acc[b] + 1 logged updates of every recurrent layer to the committed state in place.
+struct ReplayArgs {
+    int arch;                           // HS_ARCH_*
+    int H, P, N, di;                    // Mamba-2
+    int gh, dk, dv;                     // DeltaNet
+    float *state;                       // [n_rl][B][state]
+    const float *log; int log_w;        // [n_rl][B][Tm][log_w]
+    const int32_t *n_acc;               // [B]
+    int64_t state_elems;
+    int n_rl, B, Tm, b0, nb;
+};
+cudaError_t launch_replay(const ReplayArgs &a, cudaStream_t s);
 
 struct AttnArgs {
     int qh, kvh, hd, in_ld, q_off, k_off, v_off;
@@ -204,7 +223,7 @@ cudaError_t launch_argmax(const float *logits, int V, int T, int b0, int nb, int
                           int32_t *tok_out, int tok_col0, float *margin_out, void *part, int32_t *counters, cudaStream_t s);
 
 struct AcceptArgs {
-    int k, Tm, b0, nb, n_rl, B, convd, V;
+    int k, Tm, b0, nb, n_rl, B, convd, V, replay;   // replay: the committed state stays in slot 0
     HsCtrl ctrl;
     const int32_t *forced_n, *forced_next;
     float *cw; const float *hist;       // [n_rl][B][3][convd], [n_rl][B][Tm][convd]

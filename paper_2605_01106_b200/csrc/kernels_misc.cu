@@ -163,7 +163,7 @@ __global__ void accept_kernel(AcceptArgs a) {
         for (int i = 0; i < k; ++i) d[i] = __ldcg(cand + i + 1);
         for (int i = 0; i <= k; ++i) em[i] = i < n ? d[i] : (i == n ? next : -1);
         a.ctrl.n_acc[b] = n;
-        a.ctrl.slot[b] = n;
+        a.ctrl.slot[b] = a.replay ? 0 : n;
         a.ctrl.kv_len[b] = __ldcg(a.ctrl.kv_len + b) + n + 1;
         a.ctrl.cand[b * Tm] = next;
     }

@@ -110,6 +110,19 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
     }
     __syncthreads();
 
+    // rollback by replay: log the operands of every update (alpha, beta, normalised k, v) instead of storing states
+    if (a.log) {
+        float *lg = a.log + (size_t)b * a.Tm * a.log_w;
+        for (int idx = threadIdx.x; idx < T * (DK + 64); idx += GDN_THREADS) {
+            const int i = idx / (DK + 64), c = idx - i * (DK + 64);
+            if (c < DK) lg[(size_t)i * a.log_w + 2 * a.gh + h * DK + c] = ks[i][c];
+            else if (c - DK < dv) lg[(size_t)i * a.log_w + 2 * a.gh + nk + h * dv + (c - DK)] = vs[i][c - DK];
+        }
+        if (threadIdx.x < T) {
+            lg[(size_t)threadIdx.x * a.log_w + h] = al[threadIdx.x];
+            lg[(size_t)threadIdx.x * a.log_w + a.gh + h] = be[threadIdx.x];
+        }
+    }
     float *sout = a.state_out + (size_t)b * a.out_seq_stride + (size_t)h * dv * DK;
     constexpr int LPV = 32 / RPW;
     for (int i = 0; i < T; ++i) {
@@ -131,7 +144,7 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
         }
         const float o = xreduce<RPW>(part, lane);
         if (rows_ok && (lane & (LPV - 1)) == 0) os[i][warp * RPW + lane / LPV] = o * 0.125f;   // 1/sqrt(64)
-        if (rows_ok) {
+        if (rows_ok && !a.log) {
             float *dst = sout + (size_t)i * a.out_slot_stride;
 #pragma unroll
             for (int r = 0; r < RPW; ++r)
@@ -149,7 +162,112 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Rollback by replay.  The verify pass logged the operands of its k+1 state updates; once the accept kernel has
+// fixed n, the first n + 1 of them are applied to the committed state in place, with the very operations (and
+// operand values) the verify pass used in registers, so the result equals the snapshot it would have stored.
+// One launch covers every recurrent layer: grid z = layer * sequences.
+template <int EPL>
+__global__ void __launch_bounds__(SSM_THREADS) replay_ssm_kernel(const ReplayArgs a) {
+    constexpr int N = 32 * EPL, PR = 16, RPW = PR / (SSM_THREADS / 32);
+    constexpr int VW = EPL < 4 ? EPL : 4, NVEC = EPL / VW;
+    const int p0 = blockIdx.x * PR, h = blockIdx.y, rl = blockIdx.z / a.nb, lb = blockIdx.z - rl * a.nb, b = a.b0 + lb;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_trigger();
+    float *sp = a.state + ((size_t)rl * a.B + b) * a.state_elems + ((size_t)h * a.P + p0 + warp * RPW) * N;
+    const float *lg = a.log + ((size_t)rl * a.B + b) * a.Tm * a.log_w;
+    pdl_wait();
+    const int n = __ldcg(a.n_acc + b);
+    float s[RPW][EPL];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v) {
+            const float *src = sp + r * N + v * (32 * VW) + lane * VW;
+            if (VW == 4) { float4 t = __ldcg(reinterpret_cast<const float4 *>(src)); s[r][v * 4] = t.x; s[r][v * 4 + 1] = t.y; s[r][v * 4 + 2] = t.z; s[r][v * 4 + 3] = t.w; }
+            else { float2 t = __ldcg(reinterpret_cast<const float2 *>(src)); s[r][0] = t.x; s[r][1] = t.y; }
+        }
+#pragma unroll 1
+    for (int i = 0; i <= n; ++i) {
+        const float *li = lg + (size_t)i * a.log_w;
+        const float dec = __ldcg(li + h);
+        float Bv[EPL];
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v)
+#pragma unroll
+            for (int j = 0; j < VW; ++j) Bv[v * VW + j] = __ldcg(li + a.H + a.di + v * (32 * VW) + lane * VW + j);
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const float dtx = __ldcg(li + a.H + h * a.P + p0 + warp * RPW + r);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) s[r][e] = fmaf(dec, s[r][e], dtx * Bv[e]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int v = 0; v < NVEC; ++v) {
+            float *p = sp + r * N + v * (32 * VW) + lane * VW;
+            if (VW == 4) *reinterpret_cast<float4 *>(p) = make_float4(s[r][v * 4], s[r][v * 4 + 1], s[r][v * 4 + 2], s[r][v * 4 + 3]);
+            else *reinterpret_cast<float2 *>(p) = make_float2(s[r][0], s[r][1]);
+        }
+}
+
+__global__ void __launch_bounds__(GDN_THREADS) replay_gdn_kernel(const ReplayArgs a) {
+    constexpr int DK = 64, RPW = 8, LPV = 32 / RPW;
+    const int h = blockIdx.x, rl = blockIdx.y / a.nb, lb = blockIdx.y - rl * a.nb, b = a.b0 + lb, dv = a.dv;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nk = a.gh * DK;
+    pdl_trigger();
+    float *sp = a.state + ((size_t)rl * a.B + b) * a.state_elems + (size_t)h * dv * DK;
+    const float *lg = a.log + ((size_t)rl * a.B + b) * a.Tm * a.log_w;
+    const bool rows_ok = warp * RPW < dv;
+    pdl_wait();
+    const int n = __ldcg(a.n_acc + b);
+    float s[RPW][2];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+        float2 t = rows_ok ? __ldcg(reinterpret_cast<const float2 *>(sp + (warp * RPW + r) * DK + 2 * lane)) : make_float2(0.f, 0.f);
+        s[r][0] = t.x; s[r][1] = t.y;
+    }
+#pragma unroll 1
+    for (int i = 0; i <= n; ++i) {
+        const float *li = lg + (size_t)i * a.log_w;
+        const float alpha = __ldcg(li + h), beta = __ldcg(li + a.gh + h);
+        const float k0 = __ldcg(li + 2 * a.gh + h * DK + 2 * lane), k1 = __ldcg(li + 2 * a.gh + h * DK + 2 * lane + 1);
+        float part[RPW];
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            s[r][0] *= alpha; s[r][1] *= alpha;
+            part[r] = fmaf(s[r][0], k0, s[r][1] * k1);
+        }
+        const float rk = xreduce<RPW>(part, lane);
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) {
+            const float rr = __shfl_sync(0xffffffffu, rk, r * LPV);
+            const float u = beta * ((rows_ok ? __ldcg(li + 2 * a.gh + nk + h * dv + warp * RPW + r) : 0.f) - rr);
+            s[r][0] = fmaf(u, k0, s[r][0]); s[r][1] = fmaf(u, k1, s[r][1]);
+        }
+    }
+    if (rows_ok)
+#pragma unroll
+        for (int r = 0; r < RPW; ++r)
+            *reinterpret_cast<float2 *>(sp + (warp * RPW + r) * DK + 2 * lane) = make_float2(s[r][0], s[r][1]);
+}
+
 }  // namespace
+
+cudaError_t launch_replay(const ReplayArgs &a, cudaStream_t s) {
+    if (a.n_rl < 1) return cudaSuccess;
+    if (a.arch == HS_ARCH_PARALLEL) {
+        const dim3 grid(a.P / 16, a.H, a.nb * a.n_rl);
+        if (a.N == 64) return launch_pdl(replay_ssm_kernel<2>, grid, dim3(SSM_THREADS), 0, s, a);
+        if (a.N == 128) return launch_pdl(replay_ssm_kernel<4>, grid, dim3(SSM_THREADS), 0, s, a);
+        if (a.N == 256) return launch_pdl(replay_ssm_kernel<8>, grid, dim3(SSM_THREADS), 0, s, a);
+        return cudaErrorInvalidValue;
+    }
+    return launch_pdl(replay_gdn_kernel, dim3(a.gh, a.nb * a.n_rl), dim3(GDN_THREADS), 0, s, a);
+}
 
 // a whole head per block once blocks of 16 rows would already fill the GPU several times over
 bool ssm_wide(const SsmArgs &a) { return a.P % 64 == 0 && (int64_t)(a.P / 16) * a.H * a.nb >= 148 * 32; }

@@ -139,6 +139,23 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
     }
     __syncthreads();
 
+    // ---- rollback by replay: instead of a state per position, the verify pass leaves what each update needs - the
+    //      head's decay, this strip's dt * x and (one block per sequence) the shared B - exactly the operands of the
+    //      recurrence below, so that replaying them reproduces its states bit for bit
+    if (a.log) {
+        float *lg = a.log + (size_t)b * a.Tm * a.log_w;
+        for (int idx = threadIdx.x; idx < T * SSM_PR; idx += SSM_THREADS) {
+            const int i = idx / SSM_PR, c = idx - i * SSM_PR;
+            lg[(size_t)i * a.log_w + a.H + h * a.P + p0 + c] = dt_s[i] * xs[i][c];
+        }
+        if (bx == 0 && threadIdx.x < T) lg[(size_t)threadIdx.x * a.log_w + h] = a_s[threadIdx.x];
+        if (owner)
+            for (int idx = threadIdx.x; idx < T * N; idx += SSM_THREADS) {
+                const int i = idx / N, n = idx - i * N;
+                lg[(size_t)i * a.log_w + a.H + a.di + n] = Bs[i][n];
+            }
+    }
+
     // ---- recurrence over the T positions
     float *sout = a.state_out + (size_t)b * a.out_seq_stride + ((size_t)h * a.P + p0 + warp * RPW) * N;
     for (int i = 0; i < T; ++i) {
@@ -170,7 +187,8 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
             const float z = zs[i][warp * RPW + r];
             a.g[(size_t)(rowbase + i) * a.di + col] = (y + Dh * xs[i][warp * RPW + r]) * silu_f(z);
         }
-        // state after position i (verify: snapshot i; draft: the scratch state)
+        // state after position i (verify: snapshot i; draft: the scratch state; rollback by replay: nothing)
+        if (a.log) continue;
         float *dst = sout + (size_t)i * a.out_slot_stride;
 #pragma unroll
         for (int r = 0; r < RPW; ++r)

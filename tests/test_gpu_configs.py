@@ -24,13 +24,13 @@ def env():
 _W = {}
 
 
-def make(env, name, batch, max_k, cap, checked, ctx_lens, small_init="jitter"):
+def make(env, name, batch, max_k, cap, checked, ctx_lens, small_init="jitter", flags=0):
     s = hi.CONFIGS[name]
     if (name, small_init) not in _W:
         _W.clear()                                     # one large blob at a time
         _W[(name, small_init)] = hi.make_weights(s, 0, small_init)
     blob, table = _W[(name, small_init)]
-    eng = env["hs"].Engine(s, blob, max_batch=batch, max_k=max_k, kv_capacity=cap, flags=env["hs"].HS_FLAG_GRAPHS)
+    eng = env["hs"].Engine(s, blob, max_batch=batch, max_k=max_k, kv_capacity=cap, flags=env["hs"].HS_FLAG_GRAPHS | flags)
     model = env["oracle"].Model(s, blob, table, cap)
     seqs = []
     for b in range(batch):
@@ -57,6 +57,15 @@ def test_cfg2_full_size_real_acceptance(env):
     rep = env["harness"].run_rounds(eng, seqs, s, 2, 3)
     print(rep)
     assert eng.device_status() == 0
+
+
+@pytest.mark.parametrize("name,ctx", [("cfg2_0p5b", 512), ("cfg4_seq", 1024)])
+def test_full_size_rollback_by_replay(env, name, ctx):
+    s, eng, model, seqs = make(env, name, 2, 4, ctx + 100, {0, 1}, [ctx, ctx - 37], flags=env["hs"].HS_FLAG_REPLAY)
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 2, forced=[[0, 2], [1, 0]])
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 2, forced=[[4, 1], [2, 3]], rep=rep)
+    print(rep)
+    assert eng.device_status() == 0 and rep.rounds == 4
 
 
 def test_cfg2_attention_geometries(env):

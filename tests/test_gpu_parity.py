@@ -98,6 +98,36 @@ def test_graph_replay_matches(env):
     assert eng.launch_count() > 0 and eng.device_status() == 0
 
 
+@pytest.mark.parametrize("flags", [2, 3])
+@pytest.mark.parametrize("name,k", [("cfg1_tiny", 4), ("cfg1_tiny", 8), ("test_seq", 2), ("test_seq", 4)])
+def test_rollback_by_replay_matches_oracle(env, name, k, flags):
+    # HS_FLAG_REPLAY: verify keeps an update log instead of per-position snapshots and the accepted updates are
+    # replayed into the committed state; every round's state, conv window, KV rows, tokens and accept length must be
+    # the oracle's (whose rollback == recompute property is pinned on the CPU), with and without graph replay
+    s, eng, model, seqs = setup(env, name, [hi.CONFIGS[name].prompt_len], max_k=8, cap=512, flags=flags)
+    rep = env["harness"].run_rounds(eng, seqs, s, k, 8)
+    forced = [hi.forced_accept(k, 8, seq=7)]
+    rep = env["harness"].run_rounds(eng, seqs, s, k, 8, forced=forced, rep=rep)      # every accept length 0..k occurs
+    print(name, k, flags, rep)
+    assert len(rep.n_hist) >= 2 and eng.device_status() == 0
+
+
+def test_rollback_by_replay_ragged_batch_and_async(env):
+    lens = [40, 23, 57]
+    s, eng, model, seqs = setup(env, "cfg1_tiny", lens, max_k=4, cap=512, flags=3)
+    forced = [hi.forced_accept(4, 10, seq=b) for b in range(3)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 10, forced=forced)
+    assert len(rep.n_hist) >= 3
+    env["harness"].run_rounds_async(eng, seqs, [2, 0, 4, 0, 0, 2, 4, 1] * 2)
+    env["harness"].compare_states(eng, seqs, s, kv_rows=None)
+    assert eng.device_status() == 0
+    # the snapshot buffer of this mode is one state per sequence plus the log: smaller than k + 1 snapshots
+    hs = env["hs"]
+    a = hs.query_sizes(hs.make_config(s, 3, 4, 512, flags=0)).snap
+    b = hs.query_sizes(hs.make_config(s, 3, 4, 512, flags=2)).snap
+    assert b < a / 3
+
+
 def test_draft_leaves_cache_and_committed_state_untouched(env):
     s, eng, model, seqs = setup(env, "cfg1_tiny", [32], max_k=4, cap=128)
     hs = env["hs"]
