@@ -332,6 +332,22 @@ def forced_accept(k: int, n_rounds: int, seq: int = 0, seed: int = 2, alpha_num:
     return out
 
 
+DRAFT_SKIP, DRAFT_LINEAR, DRAFT_FULL = 0, 1, 2
+
+
+def draft_plan(s: ModelShape, kind: str = "component") -> np.ndarray:
+    """Per-layer draft plans (data only).  "component": the recurrent pathway of every layer (attention suppressed);
+    "layerskip33": every third layer skipped as a whole (l % 3 == 1), the others kept whole - uniformly selected
+    layers, about 33 %; "full": every layer whole (the draft is the full model: every draft is accepted)."""
+    if kind == "component":
+        return np.full(s.L, DRAFT_LINEAR, np.int32)
+    if kind == "full":
+        return np.full(s.L, DRAFT_FULL, np.int32)
+    if kind == "layerskip33":
+        return np.array([DRAFT_SKIP if l % 3 == 1 else DRAFT_FULL for l in range(s.L)], np.int32)
+    raise ValueError(kind)
+
+
 def expected_tokens_per_round(alpha: float, k: int) -> float:
     return (1.0 - alpha ** (k + 1)) / (1.0 - alpha)
 

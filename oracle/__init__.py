@@ -53,6 +53,7 @@ def lib():
         L.or_model_create.restype = vp
         L.or_model_create.argtypes = [ctypes.POINTER(OrConfig), vp, ctypes.POINTER(OrLayer), c_i64, c_i64, c_i64]
         L.or_model_destroy.argtypes = [vp]
+        L.or_model_set_draft_plan.argtypes = [vp, vp]
         L.or_seq_create.restype = vp
         L.or_seq_create.argtypes = [vp]
         for f in ("or_seq_destroy", "or_seq_reset"):
@@ -224,6 +225,15 @@ class Model:
 
     def new_seq(self) -> "Seq":
         return Seq(self)
+
+    def set_draft_plan(self, plan=None):
+        """Per-layer draft plan (0 skip the layer, 1 recurrent pathway only, 2 whole layer); None: component-aware."""
+        if plan is None:
+            lib().or_model_set_draft_plan(self.h, None)
+        else:
+            p = np.ascontiguousarray(plan, np.int32)
+            assert p.size == self.cfg.L
+            lib().or_model_set_draft_plan(self.h, _p(p))
 
 
 class Seq:

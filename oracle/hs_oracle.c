@@ -168,6 +168,7 @@ typedef struct { double *ssm, *conv, *gdn; } rstate;
 
 struct or_model {
     or_config c; const uint8_t *blob; or_layer *layers;
+    int *plan;                          /* per-layer draft plan (OR_DRAFT_*), NULL = the component-aware draft */
     int64_t embed, lm_head, final_norm;
     int64_t n_ssm, n_conv, n_gdn;       /* doubles per sequence */
     int convd;
@@ -191,7 +192,16 @@ or_model *or_model_create(const or_config *c, const uint8_t *blob, const or_laye
     m->n_conv = (int64_t)c->L * (c->conv_w - 1) * m->convd;
     return m;
 }
-void or_model_destroy(or_model *m) { if (m) { free(m->layers); free(m); } }
+void or_model_destroy(or_model *m) { if (m) { free(m->layers); free(m->plan); free(m); } }
+
+/* Draft strategies (paper Sec. 4.2): which layers the draft model M_S runs.  plan[l] = OR_DRAFT_SKIP: the layer is
+ * the identity (layer skipping, "LayerSkip"); OR_DRAFT_LINEAR: only the SSM / linear-attention pathway (Eq. 4; an
+ * attention layer of a sequential hybrid is then the identity, Eq. 5); OR_DRAFT_FULL: the whole layer, attention
+ * included.  NULL restores the component-aware draft (every layer OR_DRAFT_LINEAR). */
+void or_model_set_draft_plan(or_model *m, const int *plan) {
+    free(m->plan); m->plan = NULL;
+    if (plan) { m->plan = (int *)malloc(sizeof(int) * m->c.L); memcpy(m->plan, plan, sizeof(int) * m->c.L); }
+}
 
 static void rstate_alloc(const or_model *m, rstate *s) {
     s->ssm = m->n_ssm ? (double *)calloc(m->n_ssm, sizeof(double)) : NULL;
@@ -345,7 +355,9 @@ static void gdn_branch(const or_model *m, const or_layer *ly, int l, rstate *st,
 }
 
 /* One token through the stack.  mode 0: full model M_H (Eq. 2 / Eq. 3); mode 1: draft M_S
- * (Eq. 4: attention output zeroed; Eq. 5: attention layers are the identity). */
+ * (Eq. 4: attention output zeroed; Eq. 5: attention layers are the identity; or the model's per-layer draft plan,
+ * Sec. 4.2: layers skipped as a whole, layers kept whole).  A draft layer that runs attention writes its K/V row at
+ * `pos`, beyond the committed length: scratch rows that the verification pass overwrites. */
 static void model_step(const or_model *m, or_seq *s, rstate *st, int token, int pos, int mode, double *logits) {
     const or_config *c = &m->c;
     int d = c->d;
@@ -356,10 +368,13 @@ static void model_step(const or_model *m, or_seq *s, rstate *st, int token, int 
     for (int i = 0; i < d; ++i) h[i] = bf16_val(e[i]);
     for (int l = 0; l < c->L; ++l) {
         const or_layer *ly = &m->layers[l];
+        /* what this layer does in this pass: the full model runs every layer whole; the draft follows its plan */
+        const int what = mode == 0 ? OR_DRAFT_FULL : (m->plan ? m->plan[l] : OR_DRAFT_LINEAR);
+        if (what == OR_DRAFT_SKIP) continue;                         /* h_l = h_{l-1} */
         if (ly->type == 0) {
             or_rmsnorm(h, fvec(m, ly->norm1), d, c->eps, u);
             ssm_branch(m, ly, l, st, u, a);
-            if (mode == 0) {
+            if (what == OR_DRAFT_FULL) {
                 double *b = (double *)malloc(sizeof(double) * d);
                 attn_branch(m, ly, l, s, pos, u, b);
                 for (int i = 0; i < d; ++i) a[i] += b[i];
@@ -373,7 +388,7 @@ static void model_step(const or_model *m, or_seq *s, rstate *st, int token, int 
             for (int i = 0; i < d; ++i) h[i] += a[i];
             mlp_block(m, ly, h);
         } else {
-            if (mode == 1) continue;            /* h_l = h_{l-1} */
+            if (what != OR_DRAFT_FULL) continue;            /* h_l = h_{l-1} */
             or_rmsnorm(h, fvec(m, ly->norm1), d, c->eps, u);
             attn_branch(m, ly, l, s, pos, u, a);
             for (int i = 0; i < d; ++i) h[i] += a[i];

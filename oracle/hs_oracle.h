@@ -46,6 +46,8 @@ typedef struct {
     or_mat Wgate, Wup, Wdown;      /* SwiGLU */
 } or_layer;
 
+enum { OR_DRAFT_SKIP = 0, OR_DRAFT_LINEAR = 1, OR_DRAFT_FULL = 2 };   /* per-layer draft plan, paper Sec. 4.2 */
+
 typedef struct or_model or_model;
 typedef struct or_seq or_seq;
 
@@ -76,6 +78,8 @@ int or_accept_len(const int *d, const int *g, int k);
 or_model *or_model_create(const or_config *c, const uint8_t *blob, const or_layer *layers,
                           int64_t embed, int64_t lm_head, int64_t final_norm);
 void or_model_destroy(or_model *m);
+/* per-layer draft plan (OR_DRAFT_*), length L; NULL: the component-aware draft of Eq. 4 / Eq. 5 */
+void or_model_set_draft_plan(or_model *m, const int *plan);
 or_seq *or_seq_create(or_model *m);
 void or_seq_destroy(or_seq *s);
 void or_seq_reset(or_seq *s);

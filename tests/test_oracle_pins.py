@@ -540,3 +540,52 @@ def test_second_token_gdn_alpha_closed_form(tseq):
     np.testing.assert_allclose(got, want_logits, rtol=1e-9, atol=1e-11)
     # alpha acts visibly: with alpha = 1 (no decay) or with the beta rows used for alpha the state would differ
     assert np.abs(alphas - 1.0).min() > 1e-3 and len(set(np.round(alphas, 6))) == gh
+
+
+# --------------------------------------------------------------------------- draft strategies (Sec. 4.2)
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+def test_draft_plans_reduce_to_known_models(cfg, request):
+    # a per-layer draft plan generalises the component-aware draft: all layers "recurrent pathway only" IS that draft
+    # (Eq. 4 / Eq. 5); all layers whole is the full model; layers skipped as a whole are layers deleted from the stack
+    s, blob, table = request.getfixturevalue(cfg)
+    toks = hi.make_prompt(s.V, 6, seq=9)
+    m, mp = oracle.Model(s, blob, table, 64), oracle.Model(s, blob, table, 64)
+    mp.set_draft_plan(hi.draft_plan(s, "component"))
+    a, b = m.new_seq(), mp.new_seq()
+    for t in toks:
+        np.testing.assert_array_equal(a.step(t, mode=1), b.step(t, mode=1))
+    # whole layers: the draft step at position 0 equals the full model's first step
+    mp.set_draft_plan(hi.draft_plan(s, "full"))
+    np.testing.assert_array_equal(mp.new_seq().step(int(toks[0]), mode=1), m.new_seq().step(int(toks[0]), mode=0))
+    # skipped layers == a stack without them (every kept layer whole), first token
+    plan = hi.draft_plan(s, "layerskip33")
+    assert (plan == hi.DRAFT_SKIP).sum() >= s.L // 3 and (plan == hi.DRAFT_FULL).sum() >= 1
+    mp.set_draft_plan(plan)
+    kept = [l for l in range(s.L) if plan[l] != hi.DRAFT_SKIP]
+    m_kept = oracle.Model(s, blob, table, 64, layer_ids=kept)
+    np.testing.assert_array_equal(mp.new_seq().step(int(toks[0]), mode=1), m_kept.new_seq().step(int(toks[0]), mode=0))
+    mp.set_draft_plan(None)
+    np.testing.assert_array_equal(mp.new_seq().step(int(toks[0]), mode=1), m.new_seq().step(int(toks[0]), mode=1))
+
+
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+@pytest.mark.parametrize("kind", ["layerskip33", "full"])
+def test_any_draft_plan_is_lossless(cfg, kind, request):
+    # whatever the draft proposes, greedy verification emits the full model's own greedy sequence (Sec. 3.3); with the
+    # full model as its own draft every draft is accepted (n = k in every round)
+    s, blob, table = request.getfixturevalue(cfg)
+    m = oracle.Model(s, blob, table, 200)
+    prompt = hi.make_prompt(s.V, s.prompt_len)
+    ref_seq = m.new_seq(); ref_seq.prefill(prompt)
+    ref = ref_seq.greedy(s.gen_tokens)
+    m.set_draft_plan(hi.draft_plan(s, kind))
+    out, ns, q = _decode_spec(m, prompt, 4, s.gen_tokens)
+    np.testing.assert_array_equal(out[: s.gen_tokens], ref)
+    if kind == "full":
+        assert min(ns) == 4
+    # rollback == recompute also holds with drafts that wrote scratch KV rows beyond the committed length
+    q2 = m.new_seq(); q2.prefill(np.concatenate([prompt, out])[: q.len])
+    np.testing.assert_array_equal(q.k()[:, : q.len], q2.k()[:, : q.len])
+    for x, y in ((q.ssm(), q2.ssm()), (q.gdn(), q2.gdn()), (q.conv(), q2.conv())):
+        if x is not None:
+            np.testing.assert_array_equal(x, y)
