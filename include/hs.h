@@ -136,8 +136,9 @@ int hs_reset(hs_model *m);
  * prompts back to back (sequence b starts at sum(lens_host[0..b-1])); lens_host[b] >= 1; every id in [0, V),
  * otherwise HS_ERR_INVALID_ARG before anything is enqueued.  Sets the batch
  * size for the following rounds.  Afterwards kv_len[b] = lens[b] and pending[b] = the greedy choice
- * after the last prompt token (generated token #1).  Runs as repeated verify passes over chunks of
- * max_k+1 tokens with every candidate accepted.  Synchronises the stream before returning. */
+ * after the last prompt token (generated token #1).  Runs as verify passes over chunks of max_k+1 prompt
+ * positions, all sequences of equal chunk length together, with every candidate accepted; nothing waits on the host
+ * between chunks.  Synchronises the stream before returning (tokens_host may be reused afterwards). */
 int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host, int batch);
 
 /* Draft phase (paper Sec. 3.3, "Draft phase": M_S generates k tokens autoregressively; M_S is Eq. 4 for a
@@ -146,6 +147,20 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
  * cand[b][0..k] = [pending, d_1..d_k] stay on the device; the KV cache and the committed state are not touched.
  * 0 <= k <= max_k; k = 0 does nothing.  HS_ERR_ORDER between hs_verify and hs_accept_rollback.  Async. */
 int hs_draft(hs_model *m, int k);
+
+/* Draft strategy (paper Sec. 4.2 and Table 8; Sec. 6.2 recommends layer skipping for sequential hybrids): what
+ * each layer does in draft mode.  plan_host: int32 [L] on the HOST, or NULL for the component-aware draft (every
+ * entry HS_DRAFT_LINEAR).
+ *   HS_DRAFT_SKIP    the layer is the identity (mixer and MLP skipped: "LayerSkip")
+ *   HS_DRAFT_LINEAR  only the SSM / linear-attention pathway runs (Eq. 4); an attention layer of a sequential
+ *                    hybrid is then the identity (Eq. 5)
+ *   HS_DRAFT_FULL    the whole layer, attention included.  Such a draft reads the committed KV cache and appends
+ *                    its own rows behind it (rows kv_len .. kv_len+k-1: scratch, overwritten by the verification
+ *                    pass), so hs_draft then also needs kv_len + k <= kv_capacity (HS_ERR_CAPACITY).
+ * Whatever the plan, greedy verification emits the full model's own tokens (Sec. 3.3); the plan only moves the
+ * acceptance rate and the cost of a draft step.  Synchronises; HS_ERR_ORDER between hs_draft and hs_verify. */
+enum { HS_DRAFT_SKIP = 0, HS_DRAFT_LINEAR = 1, HS_DRAFT_FULL = 2 };
+int hs_set_draft_plan(hs_model *m, const int32_t *plan_host);
 
 /* Verification phase (paper Sec. 3.3, "Verification phase": M_H, Eq. 2 / Eq. 3, processes the prefix and the
  * drafts in a single forward pass; here incrementally from the cached state) over k+1 candidates per sequence

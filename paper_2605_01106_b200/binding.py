@@ -20,7 +20,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_set_attn_geometry", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
+           "hs_set_attn_geometry", "hs_set_draft_plan", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
            "hs_selftest_wait_timeout", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
@@ -74,6 +74,7 @@ def load_library(path: str | None = None):
     L.hs_launch_count.restype = i64
     L.hs_launch_count.argtypes = [vp]
     L.hs_set_attn_geometry.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    L.hs_set_draft_plan.argtypes = [vp, vp]
     L.hs_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     L.hs_profile.argtypes = [vp, ctypes.c_int]
     L.hs_profile_read.argtypes = [vp, vp, vp, vp]
@@ -312,6 +313,13 @@ class Engine:
     def set_attn_geometry(self, chunk, tiles=1):
         """Fix the KV split of verify-mode attention (chunk keys x tiles per CTA); chunk = 0: automatic."""
         self._ck(lib().hs_set_attn_geometry(self.h, int(chunk), int(tiles)))
+
+    def set_draft_plan(self, plan=None):
+        """Per-layer draft plan (0 skip, 1 recurrent pathway only, 2 whole layer), or None for the component-aware draft."""
+        p = None if plan is None else np.ascontiguousarray(plan, np.int32)
+        if p is not None and p.size != self.shape.L:
+            raise HsError(-1, "draft plan needs one entry per layer")
+        self._ck(lib().hs_set_draft_plan(self.h, _ptr(p)))
 
     OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL = range(5)
 

@@ -201,7 +201,9 @@ struct AttnGeom {
     int chunk, tiles, small;
     int code() const { return small * 512 + (chunk / 16 - 1) * 32 + tiles - 1; }   // < 1024, part of the graph key
 };
-AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
+// Tq: query positions per sequence of the launch; T: rows the pass may append beyond the upper bound of kv_len
+// (the same for a verify pass; a draft that keeps attention appends one row per step, k in all)
+AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
     if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles, 0};
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
@@ -209,7 +211,7 @@ AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
         const int limit = m->c.arch == HS_ARCH_PARALLEL ? 128 : 256;
         int ck = 32;
         while (ck < limit && 8 * ck < maxlen + T) ck += 32;
-        if (g_hs_attn_small && (m->c.qh / m->c.kvh) * T <= 16 && 8 * ck >= maxlen + T) return AttnGeom{ck, 1, 1};
+        if (g_hs_attn_small && (m->c.qh / m->c.kvh) * Tq <= 16 && 8 * ck >= maxlen + T) return AttnGeom{ck, 1, 1};
     }
     int want = 32;
     while (want < 128 && 8 * want < maxlen + T) want += 32;
@@ -223,11 +225,16 @@ AttnGeom attn_geom(const hs_model *m, int T, int b0, int nb) {
     return g;
 }
 
+// does the draft run layer l at all?  (a skipped layer and an attention layer that is not kept whole are the identity)
+inline bool draft_runs(const hs_model *m, int l) {
+    return m->plan[l] != HS_DRAFT_SKIP && (m->layers[l].type != HS_LAYER_ATT || m->plan[l] == HS_DRAFT_FULL);
+}
+
 // first = true: this pass opens an API call (its predecessor in the stream may be the accept kernel of the last
 // round): its first kernel goes out in plain stream order, see hs_device.cuh.
 int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool first) {
     const hs_config &c = m->c;
-    const AttnGeom at_geom = draft ? AttnGeom{m->att_chunk, 1, 0} : attn_geom(m, T, b0, nb);
+    const AttnGeom at_geom = draft ? attn_geom(m, 1, m->last_draft_k, b0, nb) : attn_geom(m, T, T, b0, nb);
     cudaStream_t s = m->stream;
     const int rows = nb * T, d = c.d;
     const int64_t se = m->state_elems;
@@ -240,9 +247,11 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
     ++m->launches;
     for (int l = 0; l < c.L; ++l) {
         const HsLayer &ly = m->layers[l];
-        if (draft && ly.type == HS_LAYER_ATT) continue;           // Eq. 5: identity in the draft
-        const bool with_attn = !draft && ly.type != HS_LAYER_GDN;
-        const int inr = draft ? ly.in_rows_draft : ly.in_rows_full;
+        // the full model runs every layer whole; the draft follows its per-layer plan (default: the recurrent pathway of
+        // every layer - Eq. 4 - which makes an attention layer of a sequential hybrid the identity - Eq. 5)
+        if (draft && !draft_runs(m, l)) continue;
+        const bool with_attn = ly.type != HS_LAYER_GDN && (!draft || m->plan[l] == HS_DRAFT_FULL);
+        const int inr = with_attn ? ly.in_rows_full : ly.in_rows_draft;
         // (1) RMSNorm + in-projection (verify: Mamba rows and q|k|v rows in one pass over u)
         GemvArgs ga{};
         ga.W0 = ly.W_in; ga.ldw0 = d; ga.K0 = d; ga.x0 = m->hbuf[cur]; ga.ldx0 = d; ga.xparts = hparts; ga.xpstride = hps;
@@ -311,6 +320,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
             aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles; aa.small = at_geom.small;
+            aa.len_off = draft ? step : 0;
             aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
             bool fused = false;
             if (ssm_deferred) {
@@ -355,8 +365,11 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         gdn.early_trigger = 1;
         {   // next projection in the chain: the following layer's in-projection, or the LM head
             int nl = l + 1;
-            while (nl < c.L && draft && m->layers[nl].type == HS_LAYER_ATT) ++nl;
-            if (nl < c.L) { gdn.pf_ptr = m->layers[nl].W_in; gdn.pf_bytes = 2 * (int64_t)d * (draft ? m->layers[nl].in_rows_draft : m->layers[nl].in_rows_full); }
+            while (nl < c.L && draft && !draft_runs(m, nl)) ++nl;
+            if (nl < c.L) {
+                const bool na = m->layers[nl].type != HS_LAYER_GDN && (!draft || m->plan[nl] == HS_DRAFT_FULL);
+                gdn.pf_ptr = m->layers[nl].W_in; gdn.pf_bytes = 2 * (int64_t)d * (na ? m->layers[nl].in_rows_full : m->layers[nl].in_rows_draft);
+            }
             else { gdn.pf_ptr = m->lm_head; gdn.pf_bytes = 2 * (int64_t)c.V * d; }
         }
         gdn.xb = m->xb; gdn.xb_rows = m->xb_rows;
@@ -379,7 +392,9 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
 }
 
 int enqueue_draft(hs_model *m, int k, int b0, int nb) {
-    for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb, st == 0); if (rc) return rc; }
+    // a draft that keeps attention reads, in a step's attention prologue, the scratch KV row the previous step wrote:
+    // then every step opens in plain stream order
+    for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb, st == 0 || m->plan_attn); if (rc) return rc; }
     return HS_OK;
 }
 
@@ -503,6 +518,7 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
         ly.in_rows_full = in_rows(c, ly.type, false); ly.in_rows_draft = in_rows(c, ly.type, true);
         m->layers.push_back(ly);
     }
+    m->plan.assign(c.L, HS_DRAFT_LINEAR); m->plan_attn = false; m->last_draft_k = 1;
     // carve the work buffer
     char *w = (char *)bufs->work;
     WorkLayout wl = work_layout(c, v);
@@ -569,25 +585,40 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
             if (tokens_host[off + p] < 0 || tokens_host[off + p] >= m->c.V) return fail(m, HS_ERR_INVALID_ARG, "prompt token id outside [0, V)");
         off += lens_host[b];
     }
+    // Chunk c covers prompt positions [c * Tm, (c + 1) * Tm) of every sequence that reaches that far; neighbouring
+    // sequences with the same number of tokens in the chunk go out as one verify pass with every candidate accepted.
+    // Nothing waits on the host between chunks (the token slices and accept lengths are staged by the copies).
+    std::vector<int64_t> start(batch);
+    int maxlen = 0;
     off = 0;
-    for (int b = 0; b < batch; ++b) {
-        const int len = lens_host[b];
-        for (int p = 0; p < len; p += m->Tm) {
-            const int T = std::min(m->Tm, len - p);
-            CK(cudaMemcpyAsync(m->ctrl.cand + b * m->Tm, tokens_host + off + p, sizeof(int32_t) * T,
-                               cudaMemcpyHostToDevice, m->stream), "prefill tokens");
-            CK(cudaMemsetAsync(m->ctrl.stage_n + b, 0, 4, m->stream), "prefill stage");
-            int32_t n = T - 1;
-            CK(cudaMemcpyAsync(m->ctrl.stage_n + b, &n, 4, cudaMemcpyHostToDevice, m->stream), "prefill n");
-            int rc = model_pass(m, false, T, 0, b, 1, true);
-            if (rc) return rc;
-            rc = enqueue_accept(m, T - 1, b, 1, m->ctrl.stage_n, nullptr);
-            if (rc) return rc;
-            CK(cudaStreamSynchronize(m->stream), "prefill sync");   // `n` and the token slice are host temporaries
+    for (int b = 0; b < batch; ++b) { start[b] = off; off += lens_host[b]; maxlen = std::max(maxlen, lens_host[b]); }
+    std::vector<std::vector<int32_t>> acc_lens;           // alive until the final synchronisation
+    for (int p = 0; p < maxlen; p += m->Tm) {
+        acc_lens.emplace_back(batch, 0);
+        std::vector<int32_t> &n = acc_lens.back();
+        std::vector<int> Tb(batch);
+        for (int b = 0; b < batch; ++b) {
+            Tb[b] = std::max(0, std::min(m->Tm, lens_host[b] - p));
+            n[b] = Tb[b] - 1;
+            if (Tb[b] > 0)
+                CK(cudaMemcpyAsync(m->ctrl.cand + b * m->Tm, tokens_host + start[b] + p, sizeof(int32_t) * Tb[b],
+                                   cudaMemcpyHostToDevice, m->stream), "prefill tokens");
         }
-        m->kv_upper[b] += len;
-        off += len;
+        CK(cudaMemcpyAsync(m->ctrl.stage_n, n.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, m->stream), "prefill accept lengths");
+        for (int b0 = 0; b0 < batch;) {
+            int nb = 1;
+            while (b0 + nb < batch && Tb[b0 + nb] == Tb[b0]) ++nb;
+            if (Tb[b0] > 0) {
+                int rc = model_pass(m, false, Tb[b0], 0, b0, nb, true);
+                if (rc) return rc;
+                rc = enqueue_accept(m, Tb[b0] - 1, b0, nb, m->ctrl.stage_n, nullptr);
+                if (rc) return rc;
+                for (int b = b0; b < b0 + nb; ++b) m->kv_upper[b] += Tb[b0];
+            }
+            b0 += nb;
+        }
     }
+    CK(cudaStreamSynchronize(m->stream), "prefill sync");   // host temporaries and the caller's tokens were read by now
     m->batch = batch; m->phase = 0;
     return hs_device_status(m);
 }
@@ -598,7 +629,14 @@ int hs_draft(hs_model *m, int k) {
     if (m->phase == 2) return fail(m, HS_ERR_ORDER, "draft after verify: the snapshots hold the verified positions until accept_rollback");
     if (k > 0) {
         const int nb = m->batch;
-        int rc = run_maybe_graph(m, (1ull << 60) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
+        m->last_draft_k = k;
+        uint64_t geo = 0;
+        if (m->plan_attn) {         // scratch KV rows kv_len .. kv_len + k - 1
+            int rc = check_capacity(m, k, 0, nb);
+            if (rc) return rc;
+            geo = (uint64_t)attn_geom(m, 1, k, 0, nb).code();
+        }
+        int rc = run_maybe_graph(m, (1ull << 60) | (geo << 32) | ((uint64_t)k << 20) | nb, [&] { return enqueue_draft(m, k, 0, nb); });
         if (rc) return rc;
     }
     m->phase = 1; m->last_k = k;
@@ -616,7 +654,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
-    rc = run_maybe_graph(m, (2ull << 60) | ((uint64_t)attn_geom(m, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
+    rc = run_maybe_graph(m, (2ull << 60) | ((uint64_t)attn_geom(m, T, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
     return HS_OK;
@@ -776,6 +814,24 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
     if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
         return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk a multiple of 16 up to 128, tiles 1..32, chunk * tiles >= workspace chunk");
     m->att_force_chunk = chunk; m->att_force_tiles = tiles;
+    return HS_OK;
+}
+
+int hs_set_draft_plan(hs_model *m, const int32_t *plan_host) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    if (m->phase == 1) return fail(m, HS_ERR_ORDER, "the draft plan cannot change between a draft and its verification");
+    std::vector<int> plan(m->c.L, HS_DRAFT_LINEAR);
+    bool attn = false;
+    if (plan_host)
+        for (int l = 0; l < m->c.L; ++l) {
+            if (plan_host[l] < HS_DRAFT_SKIP || plan_host[l] > HS_DRAFT_FULL) return fail(m, HS_ERR_INVALID_ARG, "draft plan entries are HS_DRAFT_SKIP, _LINEAR or _FULL");
+            plan[l] = plan_host[l];
+            if (plan[l] == HS_DRAFT_FULL && m->layers[l].type != HS_LAYER_GDN) attn = true;
+        }
+    CK(cudaStreamSynchronize(m->stream), "plan sync");
+    m->plan = plan; m->plan_attn = attn;
+    for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);     // the draft graphs were captured for the old plan
+    m->graphs.clear(); m->graph_launches.clear();
     return HS_OK;
 }
 

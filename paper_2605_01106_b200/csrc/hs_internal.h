@@ -59,6 +59,8 @@ struct hs_model {
     int att_chunk, att_nch;   // keys per split, max splits
     int att_force_chunk, att_force_tiles;   // 0: automatic
     std::vector<HsLayer> layers;
+    std::vector<int> plan;    // per-layer draft plan (HS_DRAFT_*)
+    bool plan_attn;           // some layer of the draft runs attention (writes scratch KV rows beyond kv_len)
     const __nv_bfloat16 *embed, *lm_head;
     const float *final_norm;
     // carved out of bufs.work
@@ -77,6 +79,7 @@ struct hs_model {
     std::vector<int> kv_upper; // upper bound of kv_len per sequence (exact after a host readback)
     int phase;                 // 0 idle, 1 drafted, 2 verified
     int last_k;                // k of the last draft / verify
+    int last_draft_k;          // draft length of the draft being enqueued (scratch KV rows of a plan that keeps attention)
     int last_rows;             // rows of logits of the last pass
     int64_t launches;
     std::string err;
@@ -209,6 +212,7 @@ struct AttnArgs {
     float *o;                           // [rows][qh*hd]
     float *part_acc, *part_ml; int32_t *counters; int32_t *status;
     int chunk, tiles, nch;              // keys per tile, tiles per CTA, CTAs (key ranges) that cover the cache capacity
+    int len_off;                        // the new rows start at kv_len[b] + len_off (draft step i of a plan that keeps attention: i)
     int small;                          // 1: the latency-lean form (G*T <= 16 rows, every cache within one cluster of 8 CTAs x chunk keys)
     int T, b0, nb;
 };

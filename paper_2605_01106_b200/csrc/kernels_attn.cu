@@ -122,7 +122,7 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
 
     // ---- before the wait: kv_len, the first cached tile, the RoPE rows
-    const int len = __ldcg(a.kv_len + b);
+    const int len = __ldcg(a.kv_len + b) + a.len_off;
     const int SPAN = CK * a.tiles;                // cached keys per CTA
     const int nsplit = max(1, (len + SPAN - 1) / SPAN);
     cg::cluster_group cluster = cg::this_cluster();
@@ -558,7 +558,7 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
     pdl_trigger();
 
     // ---- before the wait: kv_len, the whole key range of this CTA, the RoPE rows
-    const int len = __ldcg(a.kv_len + b);
+    const int len = __ldcg(a.kv_len + b) + a.len_off;
     const int nsplit = max(1, (len + CK - 1) / CK);
     if (len + T > a.cap || nsplit > AT_CL) {      // never write past the cache; a cache longer than the host's bound is a host error
         if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, len + T > a.cap ? (int)HS_ERR_CAPACITY : (int)HS_ERR_DEVICE);

@@ -128,6 +128,38 @@ def test_rollback_by_replay_ragged_batch_and_async(env):
     assert b < a / 3
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("kind", ["layerskip33", "full"])
+@pytest.mark.parametrize("name", ["cfg1_tiny", "test_seq"])
+def test_draft_plans_match_oracle(env, name, kind, flags):
+    # per-layer draft plans (layers skipped whole / kept whole, Sec. 4.2): candidates, accept lengths, tokens and states
+    # against the oracle running the same plan; with every layer kept whole the draft is the full model and every
+    # draft is accepted.  The draft's attention writes scratch KV rows beyond kv_len that verification overwrites.
+    s, eng, model, seqs = setup(env, name, [hi.CONFIGS[name].prompt_len], max_k=4, cap=512, flags=flags)
+    plan = hi.draft_plan(s, kind)
+    eng.set_draft_plan(plan); model.set_draft_plan(plan)
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 6)
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 4, rep=rep)
+    print(name, kind, flags, rep)
+    if kind == "full":
+        assert set(rep.n_hist) == {2, 4}, rep.n_hist
+    with pytest.raises(env["hs"].HsError):
+        eng.set_draft_plan([3] * s.L)
+    eng.set_draft_plan(None); model.set_draft_plan(None)
+    env["harness"].run_rounds(eng, seqs, s, 2, 3, rep=rep)
+    assert eng.device_status() == 0
+
+
+def test_prefill_ragged_batch_matches_oracle(env):
+    # prompts of different lengths go through prefill together, chunk by chunk; shorter ones drop out of later passes
+    lens = [9, 31, 30, 30, 5]
+    s, eng, model, seqs = setup(env, "cfg1_tiny", lens, max_k=4, cap=128)
+    env["harness"].compare_states(eng, seqs, s, kv_rows=None)
+    s, eng, model, seqs = setup(env, "test_seq", [17, 17, 4], max_k=8, cap=128, flags=1)
+    env["harness"].compare_states(eng, seqs, s, kv_rows=None)
+    assert eng.device_status() == 0
+
+
 def test_draft_leaves_cache_and_committed_state_untouched(env):
     s, eng, model, seqs = setup(env, "cfg1_tiny", [32], max_k=4, cap=128)
     hs = env["hs"]
