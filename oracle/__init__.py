@@ -80,6 +80,11 @@ def lib():
         L.or_attention.argtypes = [vp, vp, vp, c_i64, c_int, c_int, c_int, c_int, vp]
         L.or_argmax_margin.argtypes = [vp, c_int, vp]
         L.or_accept_len.argtypes = [vp, vp, c_int]
+        L.or_softmax_t.argtypes = [vp, c_int, c_dbl, vp]
+        L.or_sample_cdf.argtypes = [vp, c_int, c_dbl, vp]
+        L.or_spec_accept.argtypes = [vp, vp, c_int, c_dbl, vp]
+        L.or_residual.argtypes = [vp, vp, c_int, vp]
+        L.or_round_sampled.argtypes = [vp, c_int, c_dbl, vp, vp, c_dbl, vp, c_int, c_int, vp, vp, vp, vp]
         _LIB = L
     return _LIB
 
@@ -161,6 +166,29 @@ def argmax_margin(logits):
 def accept_len(d, g):
     d = np.ascontiguousarray(d, np.int32); g = np.ascontiguousarray(g, np.int32)
     return lib().or_accept_len(_p(d), _p(g), d.size)
+
+
+def softmax_t(logits, tau):
+    lg = _f64(logits); p = np.empty_like(lg)
+    lib().or_softmax_t(_p(lg), lg.size, float(tau), _p(p))
+    return p
+
+
+def sample_cdf(w, u):
+    """(index, margin) of the inverse-CDF draw from unnormalised weights w with uniform u."""
+    w = _f64(w); m = c_dbl()
+    return lib().or_sample_cdf(_p(w), w.size, float(u), ctypes.byref(m)), m.value
+
+
+def spec_accept(pS, pH, x, u):
+    pS, pH = _f64(pS), _f64(pH); m = c_dbl()
+    return bool(lib().or_spec_accept(_p(pS), _p(pH), int(x), float(u), ctypes.byref(m))), m.value
+
+
+def residual(pS, pH):
+    pS, pH = _f64(pS), _f64(pH); r = np.empty_like(pS)
+    lib().or_residual(_p(pS), _p(pH), pS.size, _p(r))
+    return r
 
 
 # ---------------------------------------------------------------------- model
@@ -312,6 +340,19 @@ class Seq:
         rc = lib().or_draft_only(self.h, k, _p(d), _p(lg))
         assert rc == 0, rc
         return (d, lg) if want_logits else d
+
+    def round_sampled(self, k, tau, u_draft, u_acc, u_final, cand_in=None, forced_n=-1, forced_next=-1):
+        """One round at temperature tau > 0 (Eq. 6). Returns dict(cand, n, emitted, margins[2k+1])."""
+        T = k + 1
+        ud, ua = _f64(u_draft), _f64(u_acc)
+        assert ud.size >= k and ua.size >= k
+        ci = np.ascontiguousarray(cand_in, np.int32) if cand_in is not None else None
+        cand, em, mg = np.empty(T, np.int32), np.full(T, -1, np.int32), np.ones(2 * k + 1)
+        n = c_int()
+        rc = lib().or_round_sampled(self.h, k, float(tau), _p(ud), _p(ua), float(u_final), _p(ci), forced_n, forced_next,
+                                    _p(cand), ctypes.byref(n), _p(em), _p(mg))
+        assert rc == 0, rc
+        return dict(cand=cand, n=n.value, emitted=em[:n.value + 1].copy(), margins=mg)
 
     def round(self, k, cand_in=None, forced_n=-1, forced_next=-1, want_logits=False):
         """One speculative round. Returns dict(cand, g, margin, logits, n, emitted)."""

@@ -479,3 +479,107 @@ int or_round(or_seq *s, int k, const int *cand_in, int forced_n, int forced_next
     rstate_free(&run); free(snap); free(cand); free(g); free(lg);
     return 0;
 }
+
+
+/* ------------------------------------------------- speculative sampling at temperature > 0 (paper Sec. 3.3, Eq. 6) */
+/* p_j = exp((l_j - max l) / tau) / Z */
+void or_softmax_t(const double *logits, int V, double tau, double *p) {
+    double mx = logits[0];
+    for (int j = 1; j < V; ++j) if (logits[j] > mx) mx = logits[j];
+    double Z = 0.0;
+    for (int j = 0; j < V; ++j) { p[j] = exp((logits[j] - mx) / tau); Z += p[j]; }
+    for (int j = 0; j < V; ++j) p[j] /= Z;
+}
+
+/* Inverse-CDF draw from unnormalised non-negative weights: the smallest j whose cumulative weight exceeds u * total
+ * (u in [0,1)).  *margin: distance of the threshold to the nearer cumulative boundary of j, relative to the total
+ * (how far u is from choosing a neighbour).  Total 0: returns -1. */
+int or_sample_cdf(const double *w, int V, double u, double *margin) {
+    double tot = 0.0;
+    for (int j = 0; j < V; ++j) tot += w[j];
+    if (!(tot > 0.0)) { if (margin) *margin = 0.0; return -1; }
+    double t = u * tot, c = 0.0;
+    int pick = -1; double lo = 0.0, hi = 0.0;
+    for (int j = 0; j < V; ++j) {
+        double cn = c + w[j];
+        if (w[j] > 0.0 && cn > t) { pick = j; lo = c; hi = cn; break; }
+        c = cn;
+    }
+    if (pick < 0) {                       /* u * total rounded up to the total: the last positive weight */
+        for (int j = V - 1; j >= 0; --j) if (w[j] > 0.0) { pick = j; break; }
+        if (margin) *margin = 0.0;
+        return pick;
+    }
+    if (margin) { double a = t - lo, b = hi - t; *margin = (a < b ? a : b) / tot; }
+    return pick;
+}
+
+/* Eq. 6: draft token x is accepted with probability min(1, P_H(x) / P_S(x)): accepted iff u < that ratio.
+ * *margin = |u - min(1, ratio)| (0 when the ratio is >= 1: then every u accepts and the margin is reported as 1). */
+int or_spec_accept(const double *pS, const double *pH, int x, double u, double *margin) {
+    double ratio = pS[x] > 0.0 ? pH[x] / pS[x] : 1.0;
+    if (ratio >= 1.0) { if (margin) *margin = 1.0; return 1; }
+    if (margin) *margin = fabs(u - ratio);
+    return u < ratio;
+}
+
+/* unnormalised residual distribution max(0, P_H - P_S) a rejected position is resampled from */
+void or_residual(const double *pS, const double *pH, int V, double *r) {
+    for (int j = 0; j < V; ++j) { double d = pH[j] - pS[j]; r[j] = d > 0.0 ? d : 0.0; }
+}
+
+/* One round at temperature tau > 0.  u_draft[k]: uniforms of the k draft draws; u_acc[k]: of the accept tests;
+ * u_final: of the correction draw (from the residual at the first rejection) or the bonus draw (from P_H after the
+ * last draft when all are accepted).  cand_in (k+1 tokens) replaces pending and the drafts (the draft model is still
+ * run over them, for P_S).  margins[2k+1]: draft draws, accept tests (1 where not evaluated), final draw. */
+int or_round_sampled(or_seq *s, int k, double tau, const double *u_draft, const double *u_acc, double u_final,
+                     const int *cand_in, int forced_n, int forced_next,
+                     int *cand_o, int *n_acc, int *emitted, double *margins) {
+    const or_model *m = s->m;
+    int T = k + 1, V = m->c.V;
+    if (k < 0 || !(tau > 0.0) || s->len + T > m->c.kv_capacity) return -1;
+    if (!cand_in && s->pending < 0) return -2;
+    if (forced_n > k) return -3;
+    int *cand = (int *)malloc(sizeof(int) * T);
+    double *lg = (double *)malloc(sizeof(double) * V);
+    double *pS = (double *)malloc(sizeof(double) * (size_t)(k > 0 ? k : 1) * V);
+    double *pH = (double *)malloc(sizeof(double) * (size_t)T * V);
+    double *r = (double *)malloc(sizeof(double) * V);
+    for (int i = 0; i < 2 * k + 1; ++i) margins[i] = 1.0;
+    /* draft phase: M_S draws k tokens from its own distributions, on a scratch copy of the committed state */
+    rstate scratch; rstate_alloc(m, &scratch); rstate_copy(m, &scratch, &s->st);
+    cand[0] = cand_in ? cand_in[0] : s->pending;
+    for (int i = 0; i < k; ++i) {
+        model_step(m, s, &scratch, cand[i], s->len + i, 1, lg);
+        or_softmax_t(lg, V, tau, pS + (size_t)i * V);
+        int tok = or_sample_cdf(pS + (size_t)i * V, V, u_draft[i], &margins[i]);
+        cand[i + 1] = cand_in ? cand_in[i + 1] : tok;
+        if (cand_in) margins[i] = 1.0;
+    }
+    rstate_free(&scratch);
+    /* verification phase: M_H over the T candidates */
+    rstate *snap = (rstate *)malloc(sizeof(rstate) * T);
+    rstate run; rstate_alloc(m, &run); rstate_copy(m, &run, &s->st);
+    for (int i = 0; i < T; ++i) {
+        model_step(m, s, &run, cand[i], s->len + i, 0, lg);
+        or_softmax_t(lg, V, tau, pH + (size_t)i * V);
+        rstate_alloc(m, &snap[i]); rstate_copy(m, &snap[i], &run);
+    }
+    /* Eq. 6: accept draft i+1 with probability min(1, P_H / P_S); stop at the first rejection */
+    int n = 0;
+    while (n < k && or_spec_accept(pS + (size_t)n * V, pH + (size_t)n * V, cand[n + 1], u_acc[n], &margins[k + n])) ++n;
+    if (forced_n >= 0) n = forced_n;
+    int next;
+    if (n < k) { or_residual(pS + (size_t)n * V, pH + (size_t)n * V, V, r); next = or_sample_cdf(r, V, u_final, &margins[2 * k]); }
+    else next = or_sample_cdf(pH + (size_t)k * V, V, u_final, &margins[2 * k]);
+    if (next < 0) { next = 0; for (int j = 1; j < V; ++j) if (pH[(size_t)n * V + j] > pH[(size_t)n * V + next]) next = j; margins[2 * k] = 0.0; }
+    if (forced_next >= 0) next = forced_next;
+    if (emitted) { for (int i = 0; i < n; ++i) emitted[i] = cand[i + 1]; emitted[n] = next; }
+    rstate_copy(m, &s->st, &snap[n]);
+    s->len += n + 1; s->pending = next;
+    if (n_acc) *n_acc = n;
+    if (cand_o) memcpy(cand_o, cand, sizeof(int) * T);
+    for (int i = 0; i < T; ++i) rstate_free(&snap[i]);
+    rstate_free(&run); free(snap); free(cand); free(lg); free(pS); free(pH); free(r);
+    return 0;
+}

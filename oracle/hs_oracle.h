@@ -108,4 +108,13 @@ int or_round(or_seq *s, int k, const int *cand_in, int forced_n, int forced_next
 /* draft phase only, on a scratch copy: d[k] and (optional) logits[k*V]; committed state untouched */
 int or_draft_only(or_seq *s, int k, int *d, double *logits);
 
+/* ---- speculative sampling at temperature > 0 (paper Sec. 3.3, Eq. 6) ---- */
+void or_softmax_t(const double *logits, int V, double tau, double *p);
+int or_sample_cdf(const double *w, int V, double u, double *margin);
+int or_spec_accept(const double *pS, const double *pH, int x, double u, double *margin);
+void or_residual(const double *pS, const double *pH, int V, double *r);
+int or_round_sampled(or_seq *s, int k, double tau, const double *u_draft, const double *u_acc, double u_final,
+                     const int *cand_in, int forced_n, int forced_next,
+                     int *cand_o, int *n_acc, int *emitted, double *margins);
+
 #endif

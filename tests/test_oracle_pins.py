@@ -589,3 +589,89 @@ def test_any_draft_plan_is_lossless(cfg, kind, request):
     for x, y in ((q.ssm(), q2.ssm()), (q.gdn(), q2.gdn()), (q.conv(), q2.conv())):
         if x is not None:
             np.testing.assert_array_equal(x, y)
+
+
+# --------------------------------------------------------------------------- speculative sampling (Eq. 6)
+def test_softmax_temperature_and_inverse_cdf():
+    lg = RNG.standard_normal(9)
+    for tau in (0.3, 0.6, 1.0, 2.5):
+        p = oracle.softmax_t(lg, tau)
+        e = np.exp(lg / tau)
+        np.testing.assert_allclose(p, e / e.sum(), rtol=1e-12)
+    w = np.array([0.0, 0.2, 0.0, 0.5, 0.3])
+    # thresholds inside each positive weight's interval pick it; zero weights are never picked; monotone in u
+    for u, want in ((0.0, 1), (0.19, 1), (0.21, 3), (0.69, 3), (0.71, 4), (0.999999, 4)):
+        j, m = oracle.sample_cdf(w, u)
+        assert j == want
+    j, m = oracle.sample_cdf(w, 0.45)
+    assert j == 3 and abs(m - 0.25) < 1e-12          # 0.45 is 0.25 away from both boundaries (0.2 and 0.7)
+    assert oracle.sample_cdf(np.zeros(4), 0.3)[0] == -1
+    # frequencies over a fine grid of u reproduce the weights (weights need not be normalised)
+    us = (np.arange(20000) + 0.5) / 20000
+    picks = np.array([oracle.sample_cdf(7.0 * w, u)[0] for u in us])
+    np.testing.assert_allclose(np.bincount(picks, minlength=5) / us.size, w, atol=1e-4)
+
+
+def test_speculative_sampling_is_lossless_in_distribution():
+    # Eq. 6: a draft x ~ P_S accepted with probability min(1, P_H(x)/P_S(x)) and otherwise replaced by a draw from
+    # norm(max(0, P_H - P_S)) is distributed exactly as P_H.  Integrate over a stratified grid of the three uniforms.
+    V = 6
+    pS = oracle.softmax_t(RNG.standard_normal(V), 0.7)
+    pH = oracle.softmax_t(RNG.standard_normal(V), 0.7)
+    G = 60
+    us = (np.arange(G) + 0.5) / G
+    r = oracle.residual(pS, pH)
+    np.testing.assert_allclose(r, np.maximum(0.0, pH - pS), rtol=0, atol=0)
+    out = np.zeros(V)
+    for ud in us:
+        x, _ = oracle.sample_cdf(pS, ud)
+        acc_frac = np.mean([oracle.spec_accept(pS, pH, x, ua)[0] for ua in us])
+        np.testing.assert_allclose(acc_frac, min(1.0, pH[x] / pS[x]), atol=1.0 / G)
+        out[x] += acc_frac / G
+        res = np.bincount([oracle.sample_cdf(r, uf)[0] for uf in us], minlength=V) / G
+        out += (1.0 - acc_frac) / G * res
+    np.testing.assert_allclose(out, pH, atol=3.0 / G)
+    # identical distributions: every draft is accepted whatever u
+    assert all(oracle.spec_accept(pH, pH, x, u)[0] for x in range(V) for u in (0.0, 0.5, 0.999999))
+
+
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+def test_sampled_round_reduces_to_greedy_at_low_temperature(cfg, request):
+    # tau -> 0: the draws collapse onto the argmax, so a sampled round emits what the greedy round emits
+    s, blob, table = request.getfixturevalue(cfg)
+    m = oracle.Model(s, blob, table, 160)
+    prompt = hi.make_prompt(s.V, s.prompt_len)
+    a, b = m.new_seq(), m.new_seq()
+    a.prefill(prompt); b.prefill(prompt)
+    for r in range(4):
+        u = hi.uniform01(5, 77 + r, 2 * 4 + 1)
+        ga = a.round(4)
+        gb = b.round_sampled(4, 1e-4, u[:4], u[4:8], u[8])
+        np.testing.assert_array_equal(ga["cand"], gb["cand"])
+        assert ga["n"] == gb["n"]
+        np.testing.assert_array_equal(ga["emitted"], gb["emitted"])
+    np.testing.assert_array_equal(a.ssm() if a.ssm() is not None else a.gdn(), b.ssm() if b.ssm() is not None else b.gdn())
+
+
+def test_sampled_round_state_is_consistent_and_first_token_follows_p_h(tiny):
+    # (i) after sampled rounds the state is the full model over the emitted tokens (rollback == recompute);
+    # (ii) with the full model as its own draft (plan: every layer whole) P_S = P_H: every draft is accepted
+    s, blob, table = tiny
+    m = oracle.Model(s, blob, table, 200)
+    prompt = hi.make_prompt(s.V, 24)
+    q = m.new_seq(); q.prefill(prompt)
+    out, ns = [q.pending], []
+    # (the random-init model's logits are small, so the temperature that makes P_S and P_H differ visibly is small too)
+    for r in range(10):
+        u = hi.uniform01(6, r, 9)
+        res = q.round_sampled(4, 0.01, u[:4], u[4:8], u[8])
+        out += list(res["emitted"]); ns.append(res["n"])
+    assert len(set(ns)) >= 3, ns
+    q2 = m.new_seq(); q2.prefill(np.concatenate([prompt, out])[: q.len])
+    np.testing.assert_array_equal(q.ssm(), q2.ssm())
+    np.testing.assert_array_equal(q.k()[:, : q.len], q2.k()[:, : q.len])
+    m.set_draft_plan(hi.draft_plan(s, "full"))
+    q3 = m.new_seq(); q3.prefill(prompt)
+    for r in range(3):
+        u = hi.uniform01(6, 100 + r, 9)
+        assert q3.round_sampled(4, 0.01, u[:4], u[4:8], u[8])["n"] == 4
