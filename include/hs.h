@@ -162,6 +162,17 @@ int hs_draft(hs_model *m, int k);
 enum { HS_DRAFT_SKIP = 0, HS_DRAFT_LINEAR = 1, HS_DRAFT_FULL = 2 };
 int hs_set_draft_plan(hs_model *m, const int32_t *plan_host);
 
+/* Speculative sampling at temperature > 0 (paper Sec. 3.3, Eq. 6).  temperature = 0 (the default) is greedy decoding.
+ * With temperature > 0: hs_draft draws draft i from softmax(draft logits / temperature) by inverse CDF with the uniform
+ * u_draft_dev[b * max_k + i - 1] and keeps the draft logits; hs_accept_rollback (when no forced accept length is given)
+ * accepts draft i iff u_accept_dev[b * max_k + i - 1] < P_H(x_i) / P_S(x_i), draws the correction at the first
+ * rejection from the normalised positive part of P_H - P_S, or the bonus token after k acceptances from P_H, both with
+ * u_final_dev[b]; the emitted tokens are then distributed as the full model's own samples.  The three DEVICE float
+ * arrays ([max_batch][max_k], [max_batch][max_k], [max_batch], values in [0,1)) are read by the kernels of every
+ * following round: the caller refills them between rounds (stream-ordered) and keeps them alive.  An inverse-CDF draw
+ * takes the smallest index whose cumulative weight exceeds u * total.  Synchronises; HS_ERR_ORDER inside a round. */
+int hs_set_sampling(hs_model *m, float temperature, const float *u_draft_dev, const float *u_accept_dev, const float *u_final_dev);
+
 /* Verification phase (paper Sec. 3.3, "Verification phase": M_H, Eq. 2 / Eq. 3, processes the prefix and the
  * drafts in a single forward pass; here incrementally from the cached state) over k+1 candidates per sequence
  * at positions kv_len[b]..kv_len[b]+k.  k is passed explicitly so that k = 0 (plain autoregressive decoding,

@@ -572,7 +572,7 @@ int or_round_sampled(or_seq *s, int k, double tau, const double *u_draft, const 
     int next;
     if (n < k) { or_residual(pS + (size_t)n * V, pH + (size_t)n * V, V, r); next = or_sample_cdf(r, V, u_final, &margins[2 * k]); }
     else next = or_sample_cdf(pH + (size_t)k * V, V, u_final, &margins[2 * k]);
-    if (next < 0) { next = 0; for (int j = 1; j < V; ++j) if (pH[(size_t)n * V + j] > pH[(size_t)n * V + next]) next = j; margins[2 * k] = 0.0; }
+    if (next < 0) next = or_sample_cdf(pH + (size_t)n * V, V, u_final, &margins[2 * k]);   /* empty residual (P_H <= P_S everywhere, i.e. equal): P_H itself */
     if (forced_next >= 0) next = forced_next;
     if (emitted) { for (int i = 0; i < n; ++i) emitted[i] = cand[i + 1]; emitted[n] = next; }
     rstate_copy(m, &s->st, &snap[n]);

@@ -20,7 +20,7 @@ STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
-           "hs_set_attn_geometry", "hs_set_draft_plan", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
+           "hs_set_attn_geometry", "hs_set_sampling", "hs_set_draft_plan", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
            "hs_selftest_wait_timeout", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
@@ -75,6 +75,7 @@ def load_library(path: str | None = None):
     L.hs_launch_count.argtypes = [vp]
     L.hs_set_attn_geometry.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     L.hs_set_draft_plan.argtypes = [vp, vp]
+    L.hs_set_sampling.argtypes = [vp, f32, vp, vp, vp]
     L.hs_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     L.hs_profile.argtypes = [vp, ctypes.c_int]
     L.hs_profile_read.argtypes = [vp, vp, vp, vp]
@@ -313,6 +314,16 @@ class Engine:
     def set_attn_geometry(self, chunk, tiles=1):
         """Fix the KV split of verify-mode attention (chunk keys x tiles per CTA); chunk = 0: automatic."""
         self._ck(lib().hs_set_attn_geometry(self.h, int(chunk), int(tiles)))
+
+    def set_sampling(self, temperature, u_draft=None, u_accept=None, u_final=None):
+        """Temperature > 0: speculative sampling (Eq. 6) with the given device tensors of uniforms (float32,
+        [max_batch, max_k], [max_batch, max_k], [max_batch]); the engine keeps them alive.  0: greedy."""
+        self._sampling = (u_draft, u_accept, u_final)
+        if temperature > 0:
+            for t, n in ((u_draft, self.max_batch * self.max_k), (u_accept, self.max_batch * self.max_k), (u_final, self.max_batch)):
+                if t is None or t.dtype != self.torch.float32 or not t.is_contiguous() or t.numel() != n or t.device != self.device:
+                    raise HsError(-1, "sampling needs contiguous float32 device tensors [max_batch, max_k] x2 and [max_batch]")
+        self._ck(lib().hs_set_sampling(self.h, float(temperature), _ptr(u_draft), _ptr(u_accept), _ptr(u_final)))
 
     def set_draft_plan(self, plan=None):
         """Per-layer draft plan (0 skip, 1 recurrent pathway only, 2 whole layer), or None for the component-aware draft."""

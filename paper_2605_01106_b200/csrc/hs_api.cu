@@ -127,7 +127,7 @@ Derived derive(const hs_config &c) {
 // layout of the work buffer; base may be null to only measure
 struct WorkLayout {
     int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters;
-    int64_t rope, h, zx, gbuf, obuf, abuf, logits, att_acc, att_ml, am_part, xb, total;
+    int64_t rope, h, zx, gbuf, obuf, abuf, logits, dlogits, att_acc, att_ml, am_part, xb, total;
 };
 
 WorkLayout work_layout(const hs_config &c, const Derived &v) {
@@ -145,6 +145,7 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.obuf = take((int64_t)4 * v.R * c.qh * c.hd);
     w.abuf = take((int64_t)4 * v.R * c.ff);
     w.logits = take((int64_t)4 * v.R * c.V);
+    w.dlogits = take((int64_t)4 * v.B * std::max(c.max_k, 1) * c.V);
     w.att_acc = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * c.hd);
     w.att_ml = take((int64_t)4 * v.B * c.kvh * v.att_nch * HS_MAX_GT * 2);
     w.am_part = take((int64_t)16 * v.R * HS_ARGMAX_CHUNKS);
@@ -380,11 +381,18 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
     GemvArgs lm{};
     lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->hbuf[cur]; lm.ldx0 = d; lm.xparts = hparts; lm.xpstride = hps;
     lm.norm_w = m->final_norm; lm.eps = c.eps;
-    lm.O = c.V; lm.out = m->logits; lm.ldo = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
+    // a draft step at temperature > 0 keeps its logits (Eq. 6 needs P_S of every draft position at verification time)
+    const bool sampled = draft && m->tau > 0.f;
+    const int64_t dstride = (int64_t)std::max(c.max_k, 1) * c.V;
+    lm.O = c.V; lm.nrows = rows; lm.epi = EPI_STORE;
+    if (sampled) { lm.out = m->dlogits + (size_t)b0 * dstride + (size_t)step * c.V; lm.ldo = (int)dstride; }
+    else { lm.out = m->logits; lm.ldo = c.V; }
     lm.early_trigger = 1;
     lm.xb = m->xb; lm.xb_rows = m->xb_rows;
     PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
-    if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, m->am_part, m->ctrl.am_counters, s), "argmax");
+    if (sampled) PROF(HS_PROF_ARGMAX, 0, launch_sample(m->dlogits + (size_t)step * c.V, dstride, c.V, m->Tm, b0, nb, m->tau, m->u_draft, c.max_k, step,
+                                                       m->ctrl.cand, step + 1, s), "draft draw");
+    else if (draft) PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, 1, b0, nb, m->Tm, m->ctrl.cand, step + 1, nullptr, m->am_part, m->ctrl.am_counters, s), "argmax");
     else PROF(HS_PROF_ARGMAX, 0, launch_argmax(m->logits, c.V, T, b0, nb, m->Tm, m->ctrl.g, 0, m->ctrl.margin, m->am_part, m->ctrl.am_counters, s), "argmax");
     ++m->launches;
     m->last_rows = rows;
@@ -529,7 +537,8 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters); m->ctrl.am_counters = (int32_t *)(w + wl.am_counters);
     m->rope = (float2 *)(w + wl.rope);
     m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
-    m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits);
+    m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits); m->dlogits = (float *)(w + wl.dlogits);
+    m->tau = 0.f; m->u_draft = m->u_accept = m->u_final = nullptr;
     m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part; m->xb = v.R > 16 ? (__nv_bfloat16 *)(w + wl.xb) : nullptr; m->xb_rows = gemm_tc_rows(v.R);
     // conv buffer: committed windows | verify history | draft ping-pong
     float *cv = (float *)bufs->conv;
@@ -640,6 +649,7 @@ int hs_draft(hs_model *m, int k) {
         if (rc) return rc;
     }
     m->phase = 1; m->last_k = k;
+    m->sampled_draft = m->tau > 0.f;
     return HS_OK;
 }
 
@@ -651,6 +661,7 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     const int nb = m->batch, T = k + 1;
     int rc = check_capacity(m, T, 0, nb);
     if (rc) return rc;
+    if (cand_dev) m->sampled_draft = false;      // the kept draft distributions belong to other candidates
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
@@ -665,6 +676,15 @@ int hs_accept_rollback(hs_model *m, const int32_t *forced_n_dev, const int32_t *
     if (!m) return HS_ERR_INVALID_ARG;
     if (m->phase != 2) return fail(m, HS_ERR_ORDER, "accept_rollback needs a preceding verify");
     const int k = m->last_k, nb = m->batch, T = k + 1;
+    if (m->tau > 0.f && !forced_n_dev) {
+        // Eq. 6: the accept length and the correction / bonus token are drawn on the device, then applied like forced ones
+        if (!m->sampled_draft && k > 0) return fail(m, HS_ERR_ORDER, "sampling needs the draft distributions of this round: hs_draft at the same temperature, or forced accept lengths");
+        PROF(HS_PROF_ACCEPT, 0, launch_spec_accept(m->dlogits, (int64_t)std::max(m->c.max_k, 1) * m->c.V, m->logits, m->ctrl.cand, m->u_accept, m->u_final,
+                                                   m->c.max_k, m->ctrl.stage_n, m->ctrl.stage_next, m->c.V, m->Tm, k, 0, nb, m->tau, m->stream), "sampled accept");
+        ++m->launches;
+        forced_n_dev = m->ctrl.stage_n;
+        if (!forced_next_dev) forced_next_dev = m->ctrl.stage_next;
+    }
     int rc = enqueue_accept(m, k, 0, nb, forced_n_dev, forced_next_dev);
     if (rc) return rc;
     m->phase = 0;
@@ -831,6 +851,21 @@ int hs_set_draft_plan(hs_model *m, const int32_t *plan_host) {
     CK(cudaStreamSynchronize(m->stream), "plan sync");
     m->plan = plan; m->plan_attn = attn;
     for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);     // the draft graphs were captured for the old plan
+    m->graphs.clear(); m->graph_launches.clear();
+    return HS_OK;
+}
+
+int hs_set_sampling(hs_model *m, float temperature, const float *u_draft_dev, const float *u_accept_dev, const float *u_final_dev) {
+    if (!m) return HS_ERR_INVALID_ARG;
+    if (m->phase != 0) return fail(m, HS_ERR_ORDER, "the sampling mode changes between rounds only");
+    const bool on = temperature > 0.f;
+    if (on && (!u_draft_dev || !u_accept_dev || !u_final_dev)) return fail(m, HS_ERR_INVALID_ARG, "sampling needs the three uniform arrays");
+    if (!(temperature >= 0.f)) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "sampling sync");
+    m->tau = on ? temperature : 0.f;
+    m->u_draft = on ? u_draft_dev : nullptr; m->u_accept = on ? u_accept_dev : nullptr; m->u_final = on ? u_final_dev : nullptr;
+    m->sampled_draft = false;
+    for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);     // the draft graphs depend on the mode and the pointers
     m->graphs.clear(); m->graph_launches.clear();
     return HS_OK;
 }

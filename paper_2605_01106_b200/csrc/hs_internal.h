@@ -68,6 +68,9 @@ struct hs_model {
     float2 *rope;             // [cap][hd/2] (cos, sin)
     float *hbuf[2];            // residual stream, ping-pong; each [HS_H_PARTS][B*Tm][d] partial sums
     float *zx, *gbuf, *obuf, *abuf, *logits;
+    float *dlogits;            // [B][max(max_k,1)][V] logits of the draft steps (kept for Eq. 6)
+    float tau;                 // sampling temperature; 0: greedy
+    const float *u_draft, *u_accept, *u_final;   // DEVICE uniforms of the round: [B][max_k], [B][max_k], [B]
     float *att_acc, *att_ml;
     __nv_bfloat16 *xb; int64_t xb_rows;   // packed activation operand of the many-row projection kernel
     void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
@@ -79,6 +82,7 @@ struct hs_model {
     std::vector<int> kv_upper; // upper bound of kv_len per sequence (exact after a host readback)
     int phase;                 // 0 idle, 1 drafted, 2 verified
     int last_k;                // k of the last draft / verify
+    bool sampled_draft;        // the draft logits buffer holds the distributions of the candidates now in `cand`
     int last_draft_k;          // draft length of the draft being enqueued (scratch KV rows of a plan that keeps attention)
     int last_rows;             // rows of logits of the last pass
     int64_t launches;
@@ -234,3 +238,9 @@ struct AcceptArgs {
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s);
 cudaError_t launch_wait_probe(int32_t *status, int polls, cudaStream_t s);
+// speculative sampling (Eq. 6): a draft draw from softmax(logits / tau), and the accept / correction / bonus decision
+cudaError_t launch_sample(const float *logits, int64_t row_stride, int V, int Tm, int b0, int nb, float tau,
+                          const float *u, int u_stride, int u_col, int32_t *tok_out, int tok_col, cudaStream_t s);
+cudaError_t launch_spec_accept(const float *dlogits, int64_t d_seq_stride, const float *vlogits, const int32_t *cand,
+                               const float *u_acc, const float *u_final, int u_stride, int32_t *n_out, int32_t *next_out,
+                               int V, int Tm, int k, int b0, int nb, float tau, cudaStream_t s);

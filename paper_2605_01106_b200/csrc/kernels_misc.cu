@@ -169,6 +169,146 @@ __global__ void accept_kernel(AcceptArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Speculative sampling at temperature > 0 (paper Sec. 3.3, Eq. 6).  One block per sequence; a logits row is
+// walked in per-thread contiguous segments so that every sum has a fixed order (reproducible draws).
+constexpr int SP_THREADS = 1024;
+
+struct RowStat { float mx, Z; };
+
+// max and sum of exp((l - max) / tau) of one row; every thread returns the same values
+__device__ __forceinline__ RowStat sp_row_stat(const float *row, int V, float inv_tau, float *red_s) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    float mx = -INFINITY;
+    for (int j = tid; j < V; j += SP_THREADS) mx = fmaxf(mx, __ldcg(row + j));
+    mx = warp_max(mx);
+    __syncthreads();
+    if (lane == 0) red_s[warp] = mx;
+    __syncthreads();
+    mx = red_s[0];
+    for (int w = 1; w < SP_THREADS / 32; ++w) mx = fmaxf(mx, red_s[w]);
+    float z = 0.f;
+    for (int j = tid; j < V; j += SP_THREADS) z += expf((__ldcg(row + j) - mx) * inv_tau);
+    z = warp_sum(z);
+    __syncthreads();
+    if (lane == 0) red_s[warp] = z;
+    __syncthreads();
+    z = 0.f;
+    for (int w = 0; w < SP_THREADS / 32; ++w) z += red_s[w];
+    return RowStat{mx, z};
+}
+
+// Inverse-CDF draw from the unnormalised weights wf(j) >= 0: the smallest j whose cumulative weight exceeds u * total.
+// Thread t owns the contiguous segment [t * S, (t + 1) * S); segment sums are scanned in thread order.  Returns the
+// index (the same in every thread), or -1 if the total is not positive.
+template <class WF>
+__device__ __forceinline__ int sp_draw(WF wf, int V, float u, float *seg_s, int *pick_s) {
+    const int tid = threadIdx.x;
+    const int S = (V + SP_THREADS - 1) / SP_THREADS, j0 = tid * S, j1 = min(V, j0 + S);
+    float seg = 0.f;
+    for (int j = j0; j < j1; ++j) seg += wf(j);
+    __syncthreads();
+    seg_s[tid] = seg;
+    if (tid == 0) { pick_s[0] = 0x7fffffff; pick_s[1] = 0; }
+    __syncthreads();
+    // exclusive prefix of this thread's segment and the total: plain ordered sums (1024 adds, once per draw)
+    float excl = 0.f, tot = 0.f;
+    for (int i = 0; i < SP_THREADS; ++i) { const float v = seg_s[i]; if (i < tid) excl += v; tot += v; }
+    if (!(tot > 0.f)) return -1;
+    const float t = u * tot;
+    if (seg > 0.f && excl + seg > t) atomicMin(pick_s, tid);       // the first segment that reaches past the threshold
+    __syncthreads();
+    int owner = *pick_s;
+    __syncthreads();
+    if (owner == 0x7fffffff) {                                     // u * total rounded up to the total: the last positive segment
+        if (seg > 0.f) atomicMax(pick_s + 1, tid);
+        __syncthreads();
+        owner = pick_s[1];
+    }
+    if (tid == owner) {
+        float c = excl; int pick = -1, lastpos = j0;
+        for (int j = j0; j < j1; ++j) {
+            const float w = wf(j);
+            if (w > 0.f) { lastpos = j; c += w; if (c > t) { pick = j; break; } }
+        }
+        pick_s[2] = pick >= 0 ? pick : lastpos;
+    }
+    __syncthreads();
+    return pick_s[2];
+}
+
+struct SampleArgs {
+    const float *logits; int64_t row_stride;   // row of sequence b at logits + b * row_stride
+    int V, Tm, b0; float inv_tau;
+    const float *u; int u_stride, u_col;       // uniform of sequence b at u[b * u_stride + u_col]
+    int32_t *tok_out; int tok_col;             // cand[b][tok_col]
+};
+
+// draft step: token ~ softmax(logits / tau)
+__global__ void __launch_bounds__(SP_THREADS) sample_kernel(const SampleArgs a) {
+    __shared__ float red_s[SP_THREADS / 32], seg_s[SP_THREADS];
+    __shared__ int pick_s[4];
+    const int b = a.b0 + blockIdx.x;
+    pdl_trigger();
+    pdl_wait();
+    const float *row = a.logits + (size_t)b * a.row_stride;
+    const RowStat st = sp_row_stat(row, a.V, a.inv_tau, red_s);
+    const float u = __ldcg(a.u + (size_t)b * a.u_stride + a.u_col);
+    int tok = sp_draw([&](int j) { return expf((__ldcg(row + j) - st.mx) * a.inv_tau); }, a.V, u, seg_s, pick_s);
+    if (tok < 0) tok = 0;
+    if (threadIdx.x == 0) a.tok_out[b * a.Tm + a.tok_col] = tok;
+}
+
+struct SpecAcceptArgs {
+    const float *dlogits; int64_t d_seq_stride;     // draft logits: row i of sequence b at dlogits + b * d_seq_stride + i * V
+    const float *vlogits;                           // verify logits: row (b - b0) * T + i, V floats each
+    const int32_t *cand;                            // [B][Tm]
+    const float *u_acc, *u_final; int u_stride;     // u_acc[b * u_stride + i], u_final[b]
+    int32_t *n_out, *next_out;                      // [B]: accept length and correction / bonus token
+    int V, Tm, k, b0; float inv_tau;
+};
+
+// Eq. 6 for one sequence: accept draft i+1 iff u_i < P_H(x) / P_S(x); at the first rejection draw the correction from
+// the positive part of P_H - P_S, after k acceptances draw the bonus token from P_H.
+__global__ void __launch_bounds__(SP_THREADS) spec_accept_kernel(const SpecAcceptArgs a) {
+    __shared__ float red_s[SP_THREADS / 32], seg_s[SP_THREADS];
+    __shared__ int pick_s[4];
+    const int lb = blockIdx.x, b = a.b0 + lb, T = a.k + 1;
+    pdl_trigger();
+    pdl_wait();
+    const float *drow = a.dlogits + (size_t)b * a.d_seq_stride, *vrow = a.vlogits + (size_t)lb * T * a.V;
+    int n = 0;
+    RowStat sS{0.f, 1.f}, sH{0.f, 1.f};
+    for (; n < a.k; ++n) {
+        sS = sp_row_stat(drow + (size_t)n * a.V, a.V, a.inv_tau, red_s);
+        sH = sp_row_stat(vrow + (size_t)n * a.V, a.V, a.inv_tau, red_s);
+        const int x = __ldcg(a.cand + b * a.Tm + n + 1);
+        const float pS = expf((__ldcg(drow + (size_t)n * a.V + x) - sS.mx) * a.inv_tau) / sS.Z;
+        const float pH = expf((__ldcg(vrow + (size_t)n * a.V + x) - sH.mx) * a.inv_tau) / sH.Z;
+        const float ratio = pS > 0.f ? pH / pS : 1.f;
+        if (!(ratio >= 1.f) && !(__ldcg(a.u_acc + (size_t)b * a.u_stride + n) < ratio)) break;      // rejected
+    }
+    const float uf = __ldcg(a.u_final + b);
+    int tok;
+    if (n < a.k) {
+        const float *dr = drow + (size_t)n * a.V, *vr = vrow + (size_t)n * a.V;
+        const float iS = 1.f / sS.Z, iH = 1.f / sH.Z;
+        tok = sp_draw([&](int j) {
+            const float d = expf((__ldcg(vr + j) - sH.mx) * a.inv_tau) * iH - expf((__ldcg(dr + j) - sS.mx) * a.inv_tau) * iS;
+            return d > 0.f ? d : 0.f; }, a.V, uf, seg_s, pick_s);
+    } else {
+        sH = sp_row_stat(vrow + (size_t)a.k * a.V, a.V, a.inv_tau, red_s);
+        tok = -1;
+    }
+    if (tok < 0) {                                   // bonus draw, or an empty residual: draw from P_H of that position
+        const float *vr = vrow + (size_t)n * a.V;
+        if (n < a.k) sH = sp_row_stat(vr, a.V, a.inv_tau, red_s);
+        tok = sp_draw([&](int j) { return expf((__ldcg(vr + j) - sH.mx) * a.inv_tau); }, a.V, uf, seg_s, pick_s);
+        if (tok < 0) tok = 0;
+    }
+    if (threadIdx.x == 0) { a.n_out[b] = n; a.next_out[b] = tok; }
+}
+
 // Self-test of the bounded wait every copy-fed kernel uses: one warp arms an mbarrier for bytes that no copy
 // will ever deliver, polls it `polls` times, gives up, records HS_ERR_TIMEOUT and returns.  Nothing is in flight
 // when it exits, so the context stays usable.
@@ -183,6 +323,19 @@ __global__ void wait_probe_kernel(int32_t *status, int polls) {
 }
 
 }  // namespace
+
+cudaError_t launch_sample(const float *logits, int64_t row_stride, int V, int Tm, int b0, int nb, float tau,
+                          const float *u, int u_stride, int u_col, int32_t *tok_out, int tok_col, cudaStream_t s) {
+    SampleArgs a{logits, row_stride, V, Tm, b0, 1.0f / tau, u, u_stride, u_col, tok_out, tok_col};
+    return launch_pdl(sample_kernel, dim3(nb), dim3(SP_THREADS), 0, s, a);
+}
+
+cudaError_t launch_spec_accept(const float *dlogits, int64_t d_seq_stride, const float *vlogits, const int32_t *cand,
+                               const float *u_acc, const float *u_final, int u_stride, int32_t *n_out, int32_t *next_out,
+                               int V, int Tm, int k, int b0, int nb, float tau, cudaStream_t s) {
+    SpecAcceptArgs a{dlogits, d_seq_stride, vlogits, cand, u_acc, u_final, u_stride, n_out, next_out, V, Tm, k, b0, 1.0f / tau};
+    return launch_pdl(spec_accept_kernel, dim3(nb), dim3(SP_THREADS), 0, s, a);
+}
 
 cudaError_t launch_wait_probe(int32_t *status, int polls, cudaStream_t s) {
     wait_probe_kernel<<<1, 32, 0, s>>>(status, polls);

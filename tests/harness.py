@@ -183,6 +183,70 @@ def run_rounds(eng, seqs, shape, k, rounds, forced=None, rep=None, check_states_
     return rep
 
 
+# a draw or an accept test whose uniform lies closer than this to a decision boundary (in the oracle's double
+# arithmetic) may come out differently in float32: such rounds are listed and the GPU is given the oracle's outcome
+CDF_MARGIN = 5e-3
+ACCEPT_MARGIN = 2e-2
+
+
+def run_rounds_sampled(eng, seqs, shape, k, rounds, tau, seed=11, rep=None):
+    """Rounds at temperature tau > 0 (Eq. 6) with the same float32 uniforms on both sides.  The library draws the
+    drafts, decides the accept length and draws the correction / bonus token on the device; everything must equal the
+    oracle's round wherever the oracle's decision margins are wide.  Returns (report, rounds compared in full)."""
+    import torch
+    rep = rep or Report()
+    B, T, dev, mk = len(seqs), k + 1, eng.device, eng.max_k
+    ud = torch.zeros((eng.max_batch, mk), dtype=torch.float32, device=dev)
+    ua = torch.zeros((eng.max_batch, mk), dtype=torch.float32, device=dev)
+    uf = torch.zeros((eng.max_batch,), dtype=torch.float32, device=dev)
+    eng.set_sampling(tau, ud, ua, uf)
+    full = 0
+    for r in range(rounds):
+        u = np.stack([hi.uniform01(seed, 1000 * b + r, 2 * mk + 1).astype(np.float32) for b in range(B)])
+        u = np.minimum(u, np.float32(1.0 - 2.0 ** -24))            # keep [0, 1) after rounding to float32
+        with torch.cuda.stream(eng.stream):
+            ud[:B].copy_(torch.from_numpy(u[:, :mk]).to(dev)); ua[:B].copy_(torch.from_numpy(u[:, mk:2 * mk]).to(dev))
+            uf[:B].copy_(torch.from_numpy(u[:, 2 * mk]).to(dev))
+        ora = [o.round_sampled(k, tau, u[b, :k].astype(np.float64), u[b, mk:mk + k].astype(np.float64), float(u[b, 2 * mk]))
+               for b, o in enumerate(seqs)]
+        eng.draft(k)
+        eng.last_k = k
+        gc, _, _ = eng.get_round(k)
+        resync = False
+        for b in range(B):
+            mg = ora[b]["margins"]
+            for i in range(1, T):
+                if gc[b, i] != ora[b]["cand"][i]:
+                    assert mg[i - 1] <= CDF_MARGIN, ("draft draw differs at a wide margin", r, b, i, mg[i - 1])
+                    rep.listed.append((r, b, "draft draw", i, float(mg[i - 1])))
+                    resync = True
+                    break
+        cand_all = np.stack([o["cand"] for o in ora]).astype(np.int32)
+        eng.verify(k, torch.from_numpy(cand_all).to(dev) if resync else None)
+        narrow = resync
+        for b in range(B):
+            mg, n = ora[b]["margins"], ora[b]["n"]
+            if any(mg[k + i] <= ACCEPT_MARGIN for i in range(min(n + 1, k))) or mg[2 * k] <= CDF_MARGIN:
+                narrow = True
+                rep.listed.append((r, b, "accept / final draw", n, float(min(mg[k:].min(), mg[2 * k]))))
+        if narrow:       # hand the GPU the oracle's outcome for this round (states stay comparable)
+            fn = torch.tensor([o["n"] for o in ora], dtype=torch.int32, device=dev)
+            fx = torch.tensor([int(o["emitted"][-1]) for o in ora], dtype=torch.int32, device=dev)
+            n, em = eng.accept_rollback(fn, fx, readback=True)
+        else:
+            n, em = eng.accept_rollback(readback=True)
+            full += 1
+        for b in range(B):
+            assert n[b] == ora[b]["n"], ("accept length", r, b, n[b], ora[b]["n"], ora[b]["margins"])
+            assert np.array_equal(em[b, : n[b] + 1], ora[b]["emitted"]), ("emitted", r, b, em[b], ora[b]["emitted"], ora[b]["margins"])
+            rep.n_hist[int(n[b])] = rep.n_hist.get(int(n[b]), 0) + 1
+            rep.tokens += int(n[b]) + 1
+        rep.rounds += 1
+        compare_states(eng, seqs, shape, rep, kv_rows=2 * T + 2)
+    eng.set_sampling(0.0)
+    return rep, full
+
+
 def inject_context(eng, oseq, shape, b, kv_len, pending, seed=3):
     """Give GPU sequence b and the oracle sequence `oseq` (or None: GPU only, recurrent state only) the same
     synthetic context: seeded recurrent state, conv window and kv_len KV rows per layer, plus the pending token."""

@@ -150,6 +150,32 @@ def test_draft_plans_match_oracle(env, name, kind, flags):
     assert eng.device_status() == 0
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("name,tau", [("cfg1_tiny", 0.01), ("cfg1_tiny", 0.05), ("test_seq", 0.02)])
+def test_speculative_sampling_matches_oracle(env, name, tau, flags):
+    # temperature > 0 (Eq. 6): draft draws, accept tests and the correction / bonus draw happen on the device with the
+    # uniforms the oracle gets; tokens, accept lengths and states must agree wherever the oracle's margins are wide
+    s, eng, model, seqs = setup(env, name, [hi.CONFIGS[name].prompt_len, 19], max_k=4, cap=512, flags=flags)
+    rep, full = env["harness"].run_rounds_sampled(eng, seqs, s, 4, 10, tau)
+    rep, full2 = env["harness"].run_rounds_sampled(eng, seqs, s, 2, 6, tau, seed=12, rep=rep)
+    print(name, tau, flags, rep, "rounds compared in full:", full + full2)
+    assert full + full2 >= 8                    # most rounds are decided by the device and compared as such
+    assert eng.device_status() == 0
+    # back to greedy: the next rounds are the oracle's greedy rounds
+    env["harness"].run_rounds(eng, seqs, s, 2, 3)
+
+
+def test_sampling_with_the_full_model_as_draft_accepts_everything(env):
+    # P_S = P_H when the draft plan keeps every layer whole: Eq. 6 accepts with probability 1
+    s, eng, model, seqs = setup(env, "cfg1_tiny", [33], max_k=4, cap=256, flags=1)
+    plan = hi.draft_plan(s, "full")
+    eng.set_draft_plan(plan); model.set_draft_plan(plan)
+    rep, full = env["harness"].run_rounds_sampled(eng, seqs, s, 4, 6, 0.02)
+    assert set(rep.n_hist) == {4}, rep.n_hist
+    with pytest.raises(env["hs"].HsError):           # no uniforms given
+        eng.set_sampling(0.5)
+
+
 def test_prefill_ragged_batch_matches_oracle(env):
     # prompts of different lengths go through prefill together, chunk by chunk; shorter ones drop out of later passes
     lens = [9, 31, 30, 30, 5]
