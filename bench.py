@@ -328,9 +328,12 @@ def run_ours(args):
     peak, peak_src = measured_peak()
     inject = s.prompt_len > 1024 or B > 4              # long or many prompts: injected context instead of hs_prefill
     blob, table = hi.make_weights(s, 0, "unit")
-    lens = hi.context_lengths(B, 4096, 16384) if s.name == "cfg5_b64" else np.full(B, s.prompt_len, np.int32)
+    lens = hi.context_lengths(B, 4096, 16384) if (s.name == "cfg5_b64" and args.prompt_len is None) else np.full(B, s.prompt_len, np.int32)
     cap = int(lens.max()) + (steps + warm + 4) * (max_k + 1) * 2 + 64
     eng = hs.Engine(s, blob, max_batch=B, max_k=max_k, kv_capacity=cap, flags=hs.HS_FLAG_GRAPHS, device=str(dev))
+    if args.attn_geometry:
+        ck, tl = (int(x) for x in args.attn_geometry.split("x"))
+        eng.set_attn_geometry(ck, tl)
     if inject:
         fresh_context = inject_random_context(torch, eng, s, B, lens)
     else:
@@ -498,6 +501,7 @@ def main():
     ap.add_argument("--all-k", dest="all_k", action="store_true", default=True)
     ap.add_argument("--one-k", dest="all_k", action="store_false")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--attn-geometry", default=None, help="CHUNKxTILES: fix the KV split of the verify attention (profiling runs)")
     ap.add_argument("--no-configs", dest="by_config", action="store_false", default=True,
                     help="skip the legs on the other workloads (profiling and quick runs)")
     args = ap.parse_args()

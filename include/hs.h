@@ -228,8 +228,10 @@ int64_t hs_launch_count(const hs_model *m);
  * CTAs to `tiles` tiles of `chunk` keys per CTA for all following verify passes; chunk = 0 restores the
  * automatic choice (made per launch from the batch and the context lengths).  chunk is a multiple of 16 up to 128,
  * tiles 1..32, and chunk * tiles must be at least the chunk the workspace was laid out for (128, or less
- * for small batch * capacity): otherwise HS_ERR_INVALID_ARG and nothing changes.  Results do not depend on
- * the setting beyond fp32 summation order. */
+ * for small batch * capacity): otherwise HS_ERR_INVALID_ARG and nothing changes.  A negative `tiles` with chunk = 128
+ * selects the streaming form (-tiles tiles of 128 keys per CTA, partials merged by the last CTA to arrive) wherever the
+ * attention runs as a launch of its own; it needs (qh / kvh) * (max_k + 1) <= 32.  Results do not depend on the setting
+ * beyond fp32 summation order. */
 int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);
 /* Tuning / measurement hook: switch a kernel choice on (value != 0) or off.  The choices are process-wide (they
  * apply to every handle); the handle's captured graphs are dropped so that the next step is captured afresh.
@@ -240,8 +242,10 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);
  *   HS_OPT_GEMM_TC         more than 16 activation rows on tcgen05 (default on; off: several 16-row launches)
  *   HS_OPT_PDL             programmatic dependent launch between the kernels of a pass (default on)
  *   HS_OPT_ATTN_SMALL      verify attention with at most 16 query rows per KV head over caches of up to 1024 keys
- *                          (2048 in a sequential hybrid) in its latency-lean form (default on; off: the general form) */
-enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4 };
+ *                          (2048 in a sequential hybrid) in its latency-lean form (default on; off: the general form)
+ *   HS_OPT_ATTN_STREAM     verify attention over long caches at large batch (a launch of its own, at most 32 query rows
+ *                          per KV head) in its streaming form (default on; off: the general form) */
+enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4, HS_OPT_ATTN_STREAM = 5 };
 int hs_set_option(hs_model *m, int option, int value);
 /* Measurement hook.  hs_profile(m, 1) brackets every following kernel launch with two CUDA events on
  * the launching stream (graph replay is bypassed while it is on); hs_profile_read synchronises and

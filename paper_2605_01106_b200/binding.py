@@ -332,7 +332,7 @@ class Engine:
             raise HsError(-1, "draft plan needs one entry per layer")
         self._ck(lib().hs_set_draft_plan(self.h, _ptr(p)))
 
-    OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL = range(5)
+    OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL, OPT_ATTN_STREAM = range(6)
 
     def set_option(self, option, value):
         """Switch a kernel choice (process-wide) on or off; see hs_set_option."""

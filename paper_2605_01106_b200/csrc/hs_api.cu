@@ -7,6 +7,7 @@
 #include <algorithm>
 
 bool g_hs_attn_small = true;   // short caches and few query rows use the latency-lean attention form
+bool g_hs_attn_stream = true;  // long caches at large batch use the streaming attention form
 
 namespace {
 
@@ -199,24 +200,35 @@ double gemv_bytes(const GemvArgs &a) {
 // Few query rows (G * T <= 16) over caches that fit one cluster: the latency-lean attention form, keys per CTA in
 // steps of 32 up to 128 (parallel blocks: the mixer CTAs of the fused launch get the same shared memory) or 256.
 struct AttnGeom {
-    int chunk, tiles, small;
-    int code() const { return small * 512 + (chunk / 16 - 1) * 32 + tiles - 1; }   // < 1024, part of the graph key
+    int chunk, tiles, small, stream;
+    int code() const { return stream * 1024 + small * 512 + (chunk / 16 - 1) * 32 + tiles - 1; }   // < 2048, part of the graph key
 };
 // Tq: query positions per sequence of the launch; T: rows the pass may append beyond the upper bound of kv_len
 // (the same for a verify pass; a draft that keeps attention appends one row per step, k in all)
 AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
-    if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles, 0};
+    if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles < 0 ? -m->att_force_tiles : m->att_force_tiles, 0, m->att_force_tiles < 0 ? 1 : 0};
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
     {
         const int limit = m->c.arch == HS_ARCH_PARALLEL ? 128 : 256;
         int ck = 32;
         while (ck < limit && 8 * ck < maxlen + T) ck += 32;
-        if (g_hs_attn_small && (m->c.qh / m->c.kvh) * Tq <= 16 && 8 * ck >= maxlen + T) return AttnGeom{ck, 1, 1};
+        if (g_hs_attn_small && (m->c.qh / m->c.kvh) * Tq <= 16 && 8 * ck >= maxlen + T) return AttnGeom{ck, 1, 1, 0};
     }
     int want = 32;
     while (want < 128 && 8 * want < maxlen + T) want += 32;
-    AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1, 0};
+    // Long caches at a batch that fills the GPU several times over, in a launch of its own (not fused with the mixer):
+    // the streaming form - 128-key tiles, as many per CTA (up to 16) as still leave every SM a few CTAs.
+    {
+        const bool own_launch = m->c.arch == HS_ARCH_SEQUENTIAL || (int64_t)(m->c.P / 16) * m->c.H * nb > 4 * 148;
+        const int64_t ctas128 = (int64_t)nb * m->c.kvh * ((maxlen + T + 127) / 128);
+        if (g_hs_attn_stream && own_launch && (m->c.qh / m->c.kvh) * Tq <= 32 && ctas128 >= 2 * 148) {
+            int tiles = (int)(ctas128 / (4 * 148));
+            tiles = tiles < 1 ? 1 : tiles > 16 ? 16 : tiles;
+            return AttnGeom{128, tiles, 0, 1};
+        }
+    }
+    AttnGeom g{want > m->att_chunk ? want : m->att_chunk, 1, 0, 0};
     const int64_t ctas64 = (int64_t)nb * m->c.kvh * ((maxlen + T + 63) / 64);
     const int64_t fill = 148 * 8;             // CTAs that keep every SM busy for several rounds
     if (g.chunk == 128 && ctas64 >= 4 * fill) {
@@ -320,7 +332,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
             aa.Kc = m->Kc + ly.al * per_layer; aa.Vc = m->Vc + ly.al * per_layer; aa.cap = c.kv_capacity;
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
-            aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles; aa.small = at_geom.small;
+            aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles; aa.small = at_geom.small; aa.stream = at_geom.stream;
             aa.len_off = draft ? step : 0;
             aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
             bool fused = false;
@@ -831,7 +843,10 @@ int64_t hs_launch_count(const hs_model *m) { return m ? m->launches : -1; }
 int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
     if (!m) return HS_ERR_INVALID_ARG;
     if (chunk == 0) { m->att_force_chunk = m->att_force_tiles = 0; return HS_OK; }
-    if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
+    if (tiles < 0) {        // the streaming form: 128-key tiles, -tiles of them per CTA
+        if (chunk != 128 || tiles < -32 || (m->c.qh / m->c.kvh) * (m->c.max_k + 1) > 32)
+            return fail(m, HS_ERR_INVALID_ARG, "streaming attention: chunk 128, 1..32 tiles, at most 32 query rows per KV head");
+    } else if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
         return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk a multiple of 16 up to 128, tiles 1..32, chunk * tiles >= workspace chunk");
     m->att_force_chunk = chunk; m->att_force_tiles = tiles;
     return HS_OK;
@@ -874,7 +889,7 @@ int hs_set_option(hs_model *m, int option, int value) {
     if (!m) return HS_ERR_INVALID_ARG;
     bool *flag = option == HS_OPT_CLUSTER_REDUCE ? &g_hs_cluster_reduce : option == HS_OPT_GEMM_MMA ? &g_hs_gemm_mma
                : option == HS_OPT_GEMM_TC ? &g_hs_gemm_tc : option == HS_OPT_PDL ? &g_hs_pdl
-               : option == HS_OPT_ATTN_SMALL ? &g_hs_attn_small : nullptr;
+               : option == HS_OPT_ATTN_SMALL ? &g_hs_attn_small : option == HS_OPT_ATTN_STREAM ? &g_hs_attn_stream : nullptr;
     if (!flag) return fail(m, HS_ERR_INVALID_ARG, "unknown option");
     CK(cudaStreamSynchronize(m->stream), "option sync");
     *flag = value != 0;

@@ -217,6 +217,7 @@ struct AttnArgs {
     float *part_acc, *part_ml; int32_t *counters; int32_t *status;
     int chunk, tiles, nch;              // keys per tile, tiles per CTA, CTAs (key ranges) that cover the cache capacity
     int len_off;                        // the new rows start at kv_len[b] + len_off (draft step i of a plan that keeps attention: i)
+    int stream;                         // 1: the streaming form for long caches (stand-alone launches: chunk = 128, at most 32 query rows)
     int small;                          // 1: the latency-lean form (G*T <= 16 rows, every cache within one cluster of 8 CTAs x chunk keys)
     int T, b0, nb;
 };

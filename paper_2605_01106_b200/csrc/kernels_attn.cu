@@ -818,6 +818,399 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Long caches (the KV read is the step's largest byte stream): the streaming form.  One CTA of eight warps owns a
+// range of `tiles` tiles of 128 cached keys and walks it with two tile buffers: while the warps work on tile t, the
+// copies of tile t+1 (K and V, 64 KB) are in flight - one block-wide barrier per tile and nothing else.  The work on a
+// tile is warp-local, as in the latency-lean form: warp w takes keys [16 w, 16 w + 16) of the tile, computes their
+// scores for all query rows on the tensor cores, keeps the probabilities in registers, folds them into its own running
+// (max, sum) and accumulates its own partial output over the whole head dimension.  After the last tile the eight warp
+// partials are merged through shared memory (over the tile buffers); a range that is the whole cache writes the
+// result, otherwise the CTA publishes its partial and the CTA of the sequence and KV head that arrives last (ticket
+// counter, no spinning) merges the ranges in order, so the result does not depend on timing.  No clusters: every SM
+// takes the next CTA as soon as it is free.
+constexpr int A2_THREADS = 256, A2_WARPS = 8, A2_CK = 128;
+
+struct Attn2Layout { int kstr, trows; size_t tile_off, q_off, new_off, rope_off, ml_off, total; };
+__host__ __device__ inline Attn2Layout attn2_layout(int hd, int mt) {
+    Attn2Layout L;
+    L.kstr = hd + 8;
+    L.trows = A2_CK + 16;                  // a tile: 128 cached keys + room for the new rows, rounded to the MMA k step
+    size_t o = 128;
+    L.tile_off = o; o += (size_t)4 * L.trows * L.kstr * 2;        // K0 | V0 | K1 | V1; later the warp partials
+    L.q_off = o; o += (size_t)2 * mt * 16 * L.kstr * 2;           // bf16 head | remainder
+    L.new_off = o; o += (size_t)2 * HS_MAX_T * L.kstr * 2;        // the new K | V rows as they are cached
+    L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
+    L.ml_off = o; o += (size_t)(A2_WARPS + 1) * mt * 16 * 2 * 4;  // per warp (max, sum) per row, then the merged pair
+    L.total = (o + 127) / 128 * 128;
+    return L;
+}
+
+template <int HD, int MT>
+__global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    constexpr int CK = A2_CK, GTB = MT * 16, NT = HD / 8;
+    const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
+    const int G = a.qh / a.kvh, T = a.T, GT = G * T;
+    const Attn2Layout L = attn2_layout(HD, MT);
+    const int KSTR = L.kstr;
+    __nv_bfloat16 *tile_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.tile_off);
+    auto Kbuf = [&](int i) { return tile_s + (size_t)(2 * i) * L.trows * KSTR; };
+    auto Vbuf = [&](int i) { return tile_s + (size_t)(2 * i + 1) * L.trows * KSTR; };
+    __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.q_off);        // [GTB][KSTR]
+    __nv_bfloat16 *Ql_s = Qh_s + (size_t)GTB * KSTR;
+    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.new_off);      // [T][KSTR]
+    __nv_bfloat16 *Vn_s = Kn_s + (size_t)HS_MAX_T * KSTR;
+    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);
+    float *wml_s = reinterpret_cast<float *>(smraw + L.ml_off);                      // [A2_WARPS + 1][GTB][2]
+    __shared__ int ticket_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t tinv = (65536u + T - 1) / T;
+    pdl_trigger();
+
+    // ---- before the wait: kv_len, the first tile, the RoPE rows
+    const int len = __ldcg(a.kv_len + b) + a.len_off;
+    const int SPAN = CK * a.tiles;
+    const int nsplit = max(1, (len + SPAN - 1) / SPAN);
+    if (split >= nsplit) return;                   // beyond the cache
+    if (len + T > a.cap) {
+        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
+        return;
+    }
+    const bool last = split == nsplit - 1;
+    const int c0 = split * SPAN, rc = max(0, min(len, c0 + SPAN) - c0);
+    const int ntile = last ? max(1, (rc + CK - 1) / CK) : (rc + CK - 1) / CK;
+    // the new rows join the last tile behind its cached keys; if they do not fit its 16 spare rows they get a tile of their own
+    const int lastc = rc - (ntile - 1) * CK;                       // cached keys of the last tile
+    const int nt_all = (last && lastc + T > L.trows) ? ntile + 1 : ntile;
+    __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
+    auto fetch = [&](int t) {              // cached rows of tile t into buffer t & 1: one commit group, possibly empty
+        const int n = t < ntile ? max(0, min(CK, rc - t * CK)) : 0;
+        __nv_bfloat16 *kd = Kbuf(t & 1), *vd = Vbuf(t & 1);
+        const __nv_bfloat16 *ks = Kb + (size_t)(c0 + t * CK) * HD, *vs = Vb + (size_t)(c0 + t * CK) * HD;
+#pragma unroll 4
+        for (int idx = tid; idx < n * (HD / 8); idx += A2_THREADS) {
+            const int j = idx / (HD / 8), c = idx - j * (HD / 8);
+            cp_async16(kd + (size_t)j * KSTR + 8 * c, ks + (size_t)j * HD + 8 * c);
+            cp_async16(vd + (size_t)j * KSTR + 8 * c, vs + (size_t)j * HD + 8 * c);
+        }
+        cp_async_commit();
+    };
+    fetch(0);
+#pragma unroll 1
+    for (int idx = tid; idx < T * (HD / 2); idx += A2_THREADS) {
+        const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+        rope_s[idx] = a.rope[(size_t)(len + i) * (HD / 2) + e];
+    }
+#pragma unroll 1
+    for (int idx = tid; idx < (GTB - GT) * (HD / 8); idx += A2_THREADS) {      // query rows that do not exist are zero
+        const int r = GT + idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4 *>(Qh_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(Ql_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+    }
+    pdl_wait();
+    __syncthreads();                        // rope_s complete
+
+    // ---- queries (RoPE, scale, bf16 head + remainder) and, in the last range, the new K / V rows
+    const int rowbase = lb * T;
+    const float scale = rsqrtf((float)HD);
+    {
+        constexpr int HP = HD / 2, NH = A2_THREADS / HP;
+        const int e = tid % HP, part = tid / HP;
+#pragma unroll 1
+        for (int q0 = part; q0 < GT; q0 += 4 * NH) {
+            float x0[4], x1[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                x0[u] = x1[u] = 0.f;
+                if (qi < GT) {
+                    const int gq = (int)((qi * tinv) >> 16);
+                    const float *src = a.zx + (size_t)(rowbase + qi - gq * T) * a.in_ld + a.q_off + (kh * G + gq) * HD;
+                    x0[u] = __ldcg(src + e); x1[u] = __ldcg(src + e + HP);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int qi = q0 + u * NH;
+                if (qi < GT) {
+                    const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
+                    __nv_bfloat16 h, l;
+                    split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                    split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
+                    Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
+                }
+            }
+        }
+    }
+    if (last) {
+#pragma unroll 1
+        for (int idx = tid; idx < T * (HD / 2); idx += A2_THREADS) {
+            const int i = idx / (HD / 2), e = idx - i * (HD / 2);
+            const float *row = a.zx + (size_t)(rowbase + i) * a.in_ld;
+            const float2 cs = rope_s[idx];
+            const float x0 = __ldcg(row + a.k_off + kh * HD + e), x1 = __ldcg(row + a.k_off + kh * HD + e + HD / 2);
+            const __nv_bfloat16 k0 = __float2bfloat16_rn(x0 * cs.x - x1 * cs.y);
+            const __nv_bfloat16 k1 = __float2bfloat16_rn(x1 * cs.x + x0 * cs.y);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e));
+            const __nv_bfloat16 v1 = __float2bfloat16_rn(__ldcg(row + a.v_off + kh * HD + e + HD / 2));
+            Kn_s[i * KSTR + e] = k0; Kn_s[i * KSTR + e + HD / 2] = k1;
+            Vn_s[i * KSTR + e] = v0; Vn_s[i * KSTR + e + HD / 2] = v1;
+            Kb[(size_t)(len + i) * HD + e] = k0; Kb[(size_t)(len + i) * HD + e + HD / 2] = k1;
+            Vb[(size_t)(len + i) * HD + e] = v0; Vb[(size_t)(len + i) * HD + e + HD / 2] = v1;
+        }
+    }
+    __syncthreads();                        // queries and new rows in place
+
+    const int g8 = lane >> 2, t4 = lane & 3;
+    float O[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { O[mt][nt][0] = O[mt][nt][1] = O[mt][nt][2] = O[mt][nt][3] = 0.f; }
+    float m_run[MT][2], l_run[MT][2];
+    int ti[MT][2];                          // position index of each of this lane's rows among the T new ones
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            m_run[mt][r] = -INFINITY; l_run[mt][r] = 0.f;
+            const int row = mt * 16 + g8 + 8 * r;
+            ti[mt][r] = row - (int)((row * tinv) >> 16) * T;
+        }
+
+#pragma unroll 1
+    for (int t = 0; t < nt_all; ++t) {
+        const bool own = t >= ntile;                              // a tile of the new rows alone
+        const int ncache = own ? 0 : max(0, min(CK, rc - t * CK));
+        const bool with_new = last && t == nt_all - 1;
+        const int nkeys = ncache + (with_new ? T : 0);
+        const int nkp = (nkeys + 15) & ~15;
+        cp_async_wait_all();                // this thread's copies of tile t have landed
+        if (with_new) {                     // the new rows behind the cached keys; finite V rows for the padding keys
+            __nv_bfloat16 *kd = Kbuf(t & 1), *vd = Vbuf(t & 1);
+#pragma unroll 1
+            for (int idx = tid; idx < T * (HD / 8); idx += A2_THREADS) {
+                const int i = idx / (HD / 8), c = idx - i * (HD / 8);
+                *reinterpret_cast<uint4 *>(kd + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Kn_s + (size_t)i * KSTR + 8 * c);
+                *reinterpret_cast<uint4 *>(vd + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Vn_s + (size_t)i * KSTR + 8 * c);
+            }
+        }
+        __syncthreads();                    // tile t complete for everybody; everybody is done with tile t-1
+        if (with_new) {
+            // (the new rows were copied by other threads: visible after the barrier above; padding rows now)
+            __nv_bfloat16 *vd = Vbuf(t & 1);
+#pragma unroll 1
+            for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
+                const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
+                *reinterpret_cast<uint4 *>(vd + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+            }
+            __syncthreads();
+        } else if (nkp != nkeys) {          // a ragged cached tile (only the last one can be): zero its padding V rows
+            __nv_bfloat16 *vd = Vbuf(t & 1);
+#pragma unroll 1
+            for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
+                const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
+                *reinterpret_cast<uint4 *>(vd + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+            }
+            __syncthreads();
+        }
+        if (t + 1 < nt_all) fetch(t + 1);   // into the other buffer, free since the barrier
+        const __nv_bfloat16 *K_s = Kbuf(t & 1), *V_s = Vbuf(t & 1);
+        // 16 keys per warp; the new rows behind a full tile make a ninth group, which warp 0 takes as well
+#pragma unroll 1
+        for (int kb = warp * 16; kb < nkp; kb += A2_WARPS * 16) {
+        // ---- scores of this warp's 16 keys for all query rows (two accumulator sets per tile row: the k steps alternate)
+        float S[MT][2][4];
+        {
+            float Sp[2][MT][2][4];
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) { Sp[c][mt][nt][0] = Sp[c][mt][nt][1] = Sp[c][mt][nt][2] = Sp[c][mt][nt][3] = 0.f; }
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                uint32_t bk[4];
+                ldsm_x4(bk, K_s + (size_t)(kb + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    uint32_t ah[4], al[4];
+                    const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
+                    ldsm_x4(ah, Qh_s + qo);
+                    ldsm_x4(al, Ql_s + qo);
+                    mma_bf16(Sp[0][mt][0], ah, bk[0], bk[1]); mma_bf16(Sp[0][mt][1], ah, bk[2], bk[3]);
+                    mma_bf16(Sp[1][mt][0], al, bk[0], bk[1]); mma_bf16(Sp[1][mt][1], al, bk[2], bk[3]);
+                }
+            }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) S[mt][nt][e] = Sp[0][mt][nt][e] + Sp[1][mt][nt][e];
+        }
+        // ---- masks, running softmax, probabilities as operand fragments
+        uint32_t ph[MT][4], pl[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = kb + nt * 8 + 2 * t4 + (e & 1);
+                    if (key >= nkeys || (with_new && key >= ncache && key - ncache > ti[mt][e >> 1])) S[mt][nt][e] = -INFINITY;
+                    mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
+                }
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                const float mnew = fmaxf(m_run[mt][r], mx[r]);
+                const float muse = mnew == -INFINITY ? 0.f : mnew;
+                const float corr = __expf(m_run[mt][r] - muse);
+                m_run[mt][r] = mnew;
+                float sum = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    const float p0 = __expf(S[mt][nt][2 * r] - muse), p1 = __expf(S[mt][nt][2 * r + 1] - muse);
+                    sum += p0 + p1;
+                    __nv_bfloat16 h0, l0, h1, l1;
+                    split_bf16(p0, h0, l0); split_bf16(p1, h1, l1);
+                    ph[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                    pl[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                }
+                l_run[mt][r] = fmaf(l_run[mt][r], corr, sum);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) { O[mt][nt][2 * r] *= corr; O[mt][nt][2 * r + 1] *= corr; }
+            }
+        }
+        // ---- partial output += P V over the whole head dimension
+#pragma unroll
+        for (int p = 0; p < NT / 2; ++p) {
+            uint32_t bv[4];
+            ldsm_x4_t(bv, V_s + (size_t)(kb + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + p * 16 + (lane >> 4) * 8);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                mma_bf16(O[mt][2 * p], ph[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], ph[mt], bv[2], bv[3]);
+                mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
+            }
+        }
+        }
+    }
+    cp_async_wait_all();
+    __syncthreads();                        // everybody is done with the tile buffers
+
+    // ---- merge the eight warp partials through shared memory (the tile buffers are free now)
+    float *wo_s = reinterpret_cast<float *>(smraw + L.tile_off);            // [A2_WARPS][GTB][HD]
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float l = l_run[mt][r];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int row = mt * 16 + g8 + 8 * r;
+            if (t4 == 0) { wml_s[((size_t)warp * GTB + row) * 2] = m_run[mt][r]; wml_s[((size_t)warp * GTB + row) * 2 + 1] = l; }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                *reinterpret_cast<float2 *>(wo_s + ((size_t)warp * GTB + row) * HD + nt * 8 + 2 * t4) = make_float2(O[mt][nt][2 * r], O[mt][nt][2 * r + 1]);
+        }
+    __syncthreads();
+    float *o_base = a.o + (size_t)rowbase * (a.qh * HD);
+    const size_t pslot = ((size_t)b * a.kvh + kh) * a.nch + split;
+    float *mrg_s = wml_s + (size_t)A2_WARPS * GTB * 2;                       // [GTB][2] merged (M, den)
+    constexpr int DV4 = HD / 4;
+#pragma unroll 1
+    for (int idx = tid; idx < GT * DV4; idx += A2_THREADS) {
+        const int qi = idx / DV4, d = (idx - qi * DV4) * 4;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < A2_WARPS; ++w) M = fmaxf(M, wml_s[((size_t)w * GTB + qi) * 2]);
+        float den = 0.f;
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < A2_WARPS; ++w) {
+            const float mw = wml_s[((size_t)w * GTB + qi) * 2];
+            const float wt = mw == -INFINITY ? 0.f : __expf(mw - M);
+            den = fmaf(wt, wml_s[((size_t)w * GTB + qi) * 2 + 1], den);
+            const float4 v = *reinterpret_cast<const float4 *>(wo_s + ((size_t)w * GTB + qi) * HD + d);
+            sum.x = fmaf(wt, v.x, sum.x); sum.y = fmaf(wt, v.y, sum.y); sum.z = fmaf(wt, v.z, sum.z); sum.w = fmaf(wt, v.w, sum.w);
+        }
+        if (nsplit == 1) {
+            const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
+            const float inv = 1.0f / den;
+            *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
+                make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
+        } else {
+            *reinterpret_cast<float4 *>(a.part_acc + pslot * HS_MAX_GT * HD + (size_t)qi * HD + d) = sum;
+            if (d == 0) { mrg_s[2 * qi] = M; mrg_s[2 * qi + 1] = den; }
+        }
+    }
+    if (nsplit == 1) return;
+    __syncthreads();
+    if (tid < 2 * GT) a.part_ml[pslot * HS_MAX_GT * 2 + tid] = mrg_s[tid];
+    // ---- several ranges: the CTA that arrives last merges their partials in order
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) ticket_s = atomicAdd(a.counters + b * a.kvh + kh, 1);
+    __syncthreads();
+    if (ticket_s != nsplit - 1) return;
+    __threadfence();
+    if (tid == 0) a.counters[b * a.kvh + kh] = 0;          // ready for the next launch
+    const size_t pbase = ((size_t)b * a.kvh + kh) * a.nch;
+    const float *pa0 = a.part_acc + pbase * HS_MAX_GT * HD;
+    const float *pm0 = a.part_ml + pbase * HS_MAX_GT * 2;
+    for (int qi = warp; qi < GT; qi += A2_WARPS) {
+        float M = -INFINITY;
+        for (int c = lane; c < nsplit; c += 32) M = fmaxf(M, __ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+        M = warp_max(M);
+        float den = 0.f;
+        for (int c = lane; c < nsplit; c += 32) {
+            const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2));
+            den = fmaf(__expf(mlv.x - M), mlv.y, den);
+        }
+        den = warp_sum(den);
+        if (lane == 0) { mrg_s[2 * qi] = M; mrg_s[2 * qi + 1] = den; }
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int idx = tid; idx < GT * DV4; idx += A2_THREADS) {
+        const int qi = idx / DV4, d = (idx - qi * DV4) * 4;
+        const float M = mrg_s[2 * qi];
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int c = 0; c < nsplit; ++c) {
+            const float wt = __expf(__ldcg(pm0 + ((size_t)c * HS_MAX_GT + qi) * 2) - M);
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(pa0 + ((size_t)c * HS_MAX_GT + qi) * HD + d));
+            sum.x = fmaf(wt, v.x, sum.x); sum.y = fmaf(wt, v.y, sum.y); sum.z = fmaf(wt, v.z, sum.z); sum.w = fmaf(wt, v.w, sum.w);
+        }
+        const int gq = (int)((qi * tinv) >> 16), i = qi - gq * T;
+        const float inv = 1.0f / mrg_s[2 * qi + 1];
+        *reinterpret_cast<float4 *>(o_base + (size_t)i * (a.qh * HD) + (kh * G + gq) * HD + d) =
+            make_float4(sum.x * inv, sum.y * inv, sum.z * inv, sum.w * inv);
+    }
+}
+
+template <int HD, int MT>
+cudaError_t launch_attn2_t(const AttnArgs &a, cudaStream_t s) {
+    static bool configured = false;
+    const size_t smem = attn2_layout(HD, MT).total;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn2_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn2_kernel<HD, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_pdl(attn2_kernel<HD, MT>, dim3(a.nch, a.kvh, a.nb), dim3(A2_THREADS), smem, s, a);
+}
+
 template <int HD, int MT>
 __global__ void __launch_bounds__(AT_THREADS) attn_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
@@ -915,6 +1308,12 @@ cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
         if (GT > 16 || a.chunk < 16 || a.chunk > AT_SMALL_MAXCHUNK || (a.chunk & 15)) return cudaErrorInvalidValue;
         return a.hd == 128 ? launch_small_t<128>(a, s) : a.hd == 64 ? launch_small_t<64>(a, s) : cudaErrorInvalidValue;
     }
+    if (a.stream) {          // the streaming form: 128-key tiles, a.tiles of them per CTA, at most 32 query rows
+        if (GT > 32 || a.chunk != A2_CK || a.tiles < 1) return cudaErrorInvalidValue;
+        if (a.hd == 128) return GT <= 16 ? launch_attn2_t<128, 1>(a, s) : launch_attn2_t<128, 2>(a, s);
+        if (a.hd == 64) return GT <= 16 ? launch_attn2_t<64, 1>(a, s) : launch_attn2_t<64, 2>(a, s);
+        return cudaErrorInvalidValue;
+    }
     if (GT > HS_MAX_GT || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || a.tiles < 1) return cudaErrorInvalidValue;
     const int mt = (GT + 15) / 16;
 #define CASE(hd_, m_) if (a.hd == hd_ && mt == m_) return launch_t<hd_, m_>(a, s)
@@ -930,6 +1329,10 @@ cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s
     const int GT = (a.qh / a.kvh) * a.T, mt = a.small ? 0 : (GT + 15) / 16;
     *fused = false;
     if (ssm_wide(sa) || GT > HS_MAX_GT || a.tiles < 1 || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || sa.P % 16) return cudaSuccess;
+    // In the fused launch every mixer block carries the attention's shared-memory allocation.  With a few blocks per SM
+    // (batch 1) that costs nothing and saves a kernel on the dependent chain; with many (larger batches) it caps the
+    // number of resident mixer blocks and with it the state bandwidth: then the two kernels go out separately.
+    if ((int64_t)(sa.P / 16) * sa.H * sa.nb > 4 * 148) return cudaSuccess;
     if (a.small && GT > 16) return cudaErrorInvalidValue;
 #define CASE(n_, e_, hd_, m_) if (sa.N == n_ && a.hd == hd_ && mt == m_) { *fused = true; return a.T <= 3 ? launch_fused_t<e_, hd_, m_, 3>(sa, a, s) : launch_fused_t<e_, hd_, m_, HS_MAX_T>(sa, a, s); }
 #define CASES(n_, e_) CASE(n_, e_, 128, 0) CASE(n_, e_, 64, 0) CASE(n_, e_, 128, 1) CASE(n_, e_, 128, 2) CASE(n_, e_, 128, 3) CASE(n_, e_, 64, 1) CASE(n_, e_, 64, 2) CASE(n_, e_, 64, 3)

@@ -88,6 +88,38 @@ def test_cfg2_attention_geometries(env):
     assert rep.rounds == 9
 
 
+def test_streaming_attention_edge_cases(env):
+    # the streaming form (128-key tiles walked with two buffers, warp-local running softmax, ranges merged by the last
+    # CTA to arrive) on the small sequential stack, where attention is a launch of its own: contexts that end exactly on
+    # a tile boundary (the new rows then form a ninth key group), one key short of and one past it, a single short
+    # range, several tiles per CTA, one and two 16-row query tiles (k = 4: 10 rows, k = 8: 18 rows)
+    lens = [1152, 1151, 1153, 640, 77, 1279]
+    s, eng, model, seqs = make(env, "test_seq", len(lens), 8, 1500, set(range(len(lens))), lens)
+    rep = None
+    for tiles, k in ((-1, 4), (-2, 8), (-4, 4), (-16, 8), (-3, 1)):
+        eng.set_attn_geometry(128, tiles)
+        forced = [hi.forced_accept(k, 1, seq=40 + b - tiles) for b in range(len(lens))]
+        rep = env["harness"].run_rounds(eng, seqs, s, k, 1, forced=forced, rep=rep)
+        assert eng.device_status() == 0, (tiles, k)
+    with pytest.raises(RuntimeError):
+        eng.set_attn_geometry(64, -2)
+    print(rep)
+    assert rep.rounds == 5
+
+
+def test_streaming_attention_batched_parallel_hybrid(env):
+    # a batch large enough that the verify attention of the parallel hybrid runs as its own launch in the streaming form
+    # (chosen automatically); three sequences carry their context on both sides, the others run beside them
+    lens = [1152, 1151, 640] + [1000 + 7 * b for b in range(21)]
+    s, eng, model, seqs = make(env, "cfg1_tiny", len(lens), 4, 1400, {0, 1, 2}, lens)
+    forced = [hi.forced_accept(4, 2, seq=b) for b in range(len(lens))]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 2, forced=forced)
+    forced = [hi.forced_accept(2, 2, seq=50 + b) for b in range(len(lens))]
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 2, forced=forced, rep=rep)
+    print(rep)
+    assert eng.device_status() == 0 and rep.rounds == 4
+
+
 def test_cfg4_sequential_full_size(env):
     s, eng, model, seqs = make(env, "cfg4_seq", 1, 4, 1100, {0}, [1024])
     rep = env["harness"].run_rounds(eng, seqs, s, 2, 2, forced=[hi.forced_accept(2, 2, seq=1)])
