@@ -830,38 +830,42 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
 // result, otherwise the CTA publishes its partial and the CTA of the sequence and KV head that arrives last (ticket
 // counter, no spinning) merges the ranges in order, so the result does not depend on timing.  No clusters: every SM
 // takes the next CTA as soon as it is free.
-constexpr int A2_THREADS = 256, A2_WARPS = 8, A2_CK = 128;
+constexpr int A2_THREADS = 256, A2_WARPS = 8, A2_CK = 128, A2_NBUF = 3;
 
-struct Attn2Layout { int kstr, trows; size_t tile_off, q_off, new_off, rope_off, ml_off, total; };
+// Tile buffers hold 128 keys x HD bf16 without padding; the 16-byte chunk c of row r sits at chunk position
+// c ^ (r & 7), which keeps the eight rows of an ldmatrix 8x8 block on different banks.  Three K and three V buffers:
+// two tiles (128 KB at HD = 128) are in flight while the warps work on a third.
+struct Attn2Layout { int kstr; size_t tile_bytes, tile_off, q_off, new_off, rope_off, ml_off, total; };
 __host__ __device__ inline Attn2Layout attn2_layout(int hd, int mt) {
     Attn2Layout L;
-    L.kstr = hd + 8;
-    L.trows = A2_CK + 16;                  // a tile: 128 cached keys + room for the new rows, rounded to the MMA k step
+    L.kstr = hd + 8;                       // padded rows of the query and new-row buffers
+    L.tile_bytes = (size_t)A2_CK * hd * 2;
     size_t o = 128;
-    L.tile_off = o; o += (size_t)4 * L.trows * L.kstr * 2;        // K0 | V0 | K1 | V1; later the warp partials
-    L.q_off = o; o += (size_t)2 * mt * 16 * L.kstr * 2;           // bf16 head | remainder
-    L.new_off = o; o += (size_t)2 * HS_MAX_T * L.kstr * 2;        // the new K | V rows as they are cached
+    L.tile_off = o; o += 2 * A2_NBUF * L.tile_bytes;               // K0 V0 K1 V1 K2 V2; later the warp partials
+    L.q_off = o; o += (size_t)2 * mt * 16 * L.kstr * 2;            // bf16 head | remainder
+    L.new_off = o; o += (size_t)2 * 16 * L.kstr * 2;               // the new K | V rows as they are cached: a 16-key group of their own
     L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
-    L.ml_off = o; o += (size_t)(A2_WARPS + 1) * mt * 16 * 2 * 4;  // per warp (max, sum) per row, then the merged pair
+    L.ml_off = o; o += (size_t)(A2_WARPS + 1) * mt * 16 * 2 * 4;   // per warp (max, sum) per row, then the merged pair
     L.total = (o + 127) / 128 * 128;
     return L;
 }
+__device__ __forceinline__ void cp_async_wait_but_two() { asm volatile("cp.async.wait_group 2;" ::: "memory"); }
 
 template <int HD, int MT>
 __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
-    constexpr int CK = A2_CK, GTB = MT * 16, NT = HD / 8;
+    constexpr int CK = A2_CK, GTB = MT * 16, NT = HD / 8, RB = HD * 2;       // RB: bytes of a tile row
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int G = a.qh / a.kvh, T = a.T, GT = G * T;
     const Attn2Layout L = attn2_layout(HD, MT);
     const int KSTR = L.kstr;
-    __nv_bfloat16 *tile_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.tile_off);
-    auto Kbuf = [&](int i) { return tile_s + (size_t)(2 * i) * L.trows * KSTR; };
-    auto Vbuf = [&](int i) { return tile_s + (size_t)(2 * i + 1) * L.trows * KSTR; };
+    unsigned char *tile_s = smraw + L.tile_off;
+    auto Kbuf = [&](int i) { return tile_s + (size_t)(2 * i) * L.tile_bytes; };
+    auto Vbuf = [&](int i) { return tile_s + (size_t)(2 * i + 1) * L.tile_bytes; };
     __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.q_off);        // [GTB][KSTR]
     __nv_bfloat16 *Ql_s = Qh_s + (size_t)GTB * KSTR;
-    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.new_off);      // [T][KSTR]
-    __nv_bfloat16 *Vn_s = Kn_s + (size_t)HS_MAX_T * KSTR;
+    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.new_off);      // [16][KSTR]
+    __nv_bfloat16 *Vn_s = Kn_s + (size_t)16 * KSTR;
     float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);
     float *wml_s = reinterpret_cast<float *>(smraw + L.ml_off);                      // [A2_WARPS + 1][GTB][2]
     __shared__ int ticket_s;
@@ -870,7 +874,7 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     const uint32_t tinv = (65536u + T - 1) / T;
     pdl_trigger();
 
-    // ---- before the wait: kv_len, the first tile, the RoPE rows
+    // ---- before the wait: kv_len, the first two tiles, the RoPE rows
     const int len = __ldcg(a.kv_len + b) + a.len_off;
     const int SPAN = CK * a.tiles;
     const int nsplit = max(1, (len + SPAN - 1) / SPAN);
@@ -881,25 +885,25 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     }
     const bool last = split == nsplit - 1;
     const int c0 = split * SPAN, rc = max(0, min(len, c0 + SPAN) - c0);
-    const int ntile = last ? max(1, (rc + CK - 1) / CK) : (rc + CK - 1) / CK;
-    // the new rows join the last tile behind its cached keys; if they do not fit its 16 spare rows they get a tile of their own
-    const int lastc = rc - (ntile - 1) * CK;                       // cached keys of the last tile
-    const int nt_all = (last && lastc + T > L.trows) ? ntile + 1 : ntile;
+    const int ntile = (rc + CK - 1) / CK;
+    const int nitem = ntile + (last ? 1 : 0);      // the range that ends the cache also takes the new rows, as one more item
     __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
     __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    auto fetch = [&](int t) {              // cached rows of tile t into buffer t & 1: one commit group, possibly empty
-        const int n = t < ntile ? max(0, min(CK, rc - t * CK)) : 0;
-        __nv_bfloat16 *kd = Kbuf(t & 1), *vd = Vbuf(t & 1);
+    auto fetch = [&](int t) {              // cached rows of tile t into buffer t % 3: one commit group, possibly empty
+        const int n = t < ntile ? min(CK, rc - t * CK) : 0;
+        unsigned char *kd = Kbuf(t % A2_NBUF), *vd = Vbuf(t % A2_NBUF);
         const __nv_bfloat16 *ks = Kb + (size_t)(c0 + t * CK) * HD, *vs = Vb + (size_t)(c0 + t * CK) * HD;
 #pragma unroll 4
         for (int idx = tid; idx < n * (HD / 8); idx += A2_THREADS) {
             const int j = idx / (HD / 8), c = idx - j * (HD / 8);
-            cp_async16(kd + (size_t)j * KSTR + 8 * c, ks + (size_t)j * HD + 8 * c);
-            cp_async16(vd + (size_t)j * KSTR + 8 * c, vs + (size_t)j * HD + 8 * c);
+            const int so = j * RB + ((c ^ (j & 7)) << 4);
+            cp_async16(kd + so, ks + (size_t)j * HD + 8 * c);
+            cp_async16(vd + so, vs + (size_t)j * HD + 8 * c);
         }
         cp_async_commit();
     };
     fetch(0);
+    fetch(1);
 #pragma unroll 1
     for (int idx = tid; idx < T * (HD / 2); idx += A2_THREADS) {
         const int i = idx / (HD / 2), e = idx - i * (HD / 2);
@@ -911,8 +915,13 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
         *reinterpret_cast<uint4 *>(Qh_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4 *>(Ql_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
     }
+#pragma unroll 1
+    for (int idx = tid; idx < 16 * (HD / 8); idx += A2_THREADS) {              // finite V rows behind the new ones
+        const int r = idx / (HD / 8), c = idx % (HD / 8);
+        *reinterpret_cast<uint4 *>(Vn_s + (size_t)r * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
+    }
     pdl_wait();
-    __syncthreads();                        // rope_s complete
+    __syncthreads();                        // rope_s complete, Vn_s cleared
 
     // ---- queries (RoPE, scale, bf16 head + remainder) and, in the last range, the new K / V rows
     const int rowbase = lb * T;
@@ -983,125 +992,114 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
             ti[mt][r] = row - (int)((row * tinv) >> 16) * T;
         }
 
+    // An item is a tile of cached keys (a buffer of the ring, swizzled rows of RB bytes) or, last, the new rows (their own
+    // padded buffer): the same code serves both, told apart by base address, row pitch and swizzle mask.
 #pragma unroll 1
-    for (int t = 0; t < nt_all; ++t) {
-        const bool own = t >= ntile;                              // a tile of the new rows alone
-        const int ncache = own ? 0 : max(0, min(CK, rc - t * CK));
-        const bool with_new = last && t == nt_all - 1;
-        const int nkeys = ncache + (with_new ? T : 0);
+    for (int t = 0; t < nitem; ++t) {
+        const bool newrows = t >= ntile;
+        const int nkeys = newrows ? T : min(CK, rc - t * CK);
         const int nkp = (nkeys + 15) & ~15;
-        cp_async_wait_all();                // this thread's copies of tile t have landed
-        if (with_new) {                     // the new rows behind the cached keys; finite V rows for the padding keys
-            __nv_bfloat16 *kd = Kbuf(t & 1), *vd = Vbuf(t & 1);
+        if (!newrows) {
+            cp_async_wait_but_one();        // this thread's copies of tile t have landed (tile t + 1 may be in flight)
+            if (nkp != nkeys) {             // a ragged tile (only the last can be): finite V rows for its padding keys
+                unsigned char *vd = Vbuf(t % A2_NBUF);
 #pragma unroll 1
-            for (int idx = tid; idx < T * (HD / 8); idx += A2_THREADS) {
-                const int i = idx / (HD / 8), c = idx - i * (HD / 8);
-                *reinterpret_cast<uint4 *>(kd + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Kn_s + (size_t)i * KSTR + 8 * c);
-                *reinterpret_cast<uint4 *>(vd + (size_t)(ncache + i) * KSTR + 8 * c) = *reinterpret_cast<const uint4 *>(Vn_s + (size_t)i * KSTR + 8 * c);
+                for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS)
+                    *reinterpret_cast<uint4 *>(vd + (size_t)(nkeys + idx / (HD / 8)) * RB + ((idx % (HD / 8)) << 4)) = make_uint4(0, 0, 0, 0);
             }
+            __syncthreads();                // tile t complete for everybody; everybody is done with tile t - 1
+            fetch(t + 2);                   // into the buffer tile t - 1 used (an empty group beyond the range)
         }
-        __syncthreads();                    // tile t complete for everybody; everybody is done with tile t-1
-        if (with_new) {
-            // (the new rows were copied by other threads: visible after the barrier above; padding rows now)
-            __nv_bfloat16 *vd = Vbuf(t & 1);
+        const unsigned char *K_s = newrows ? reinterpret_cast<const unsigned char *>(Kn_s) : Kbuf(t % A2_NBUF);
+        const unsigned char *V_s = newrows ? reinterpret_cast<const unsigned char *>(Vn_s) : Vbuf(t % A2_NBUF);
+        const int pitch = newrows ? KSTR * 2 : RB, swz = newrows ? 0 : 7;
+        // 16 keys per warp; the new rows are one group, given to the warp that a ragged last tile leaves idle most often
 #pragma unroll 1
-            for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
-                const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
-                *reinterpret_cast<uint4 *>(vd + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
-            }
-            __syncthreads();
-        } else if (nkp != nkeys) {          // a ragged cached tile (only the last one can be): zero its padding V rows
-            __nv_bfloat16 *vd = Vbuf(t & 1);
-#pragma unroll 1
-            for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
-                const int j = nkeys + idx / (HD / 8), c = idx % (HD / 8);
-                *reinterpret_cast<uint4 *>(vd + (size_t)j * KSTR + 8 * c) = make_uint4(0, 0, 0, 0);
-            }
-            __syncthreads();
-        }
-        if (t + 1 < nt_all) fetch(t + 1);   // into the other buffer, free since the barrier
-        const __nv_bfloat16 *K_s = Kbuf(t & 1), *V_s = Vbuf(t & 1);
-        // 16 keys per warp; the new rows behind a full tile make a ninth group, which warp 0 takes as well
-#pragma unroll 1
-        for (int kb = warp * 16; kb < nkp; kb += A2_WARPS * 16) {
-        // ---- scores of this warp's 16 keys for all query rows (two accumulator sets per tile row: the k steps alternate)
-        float S[MT][2][4];
-        {
-            float Sp[2][MT][2][4];
+        for (int kb = (newrows ? (warp == A2_WARPS - 1 ? 0 : nkp) : warp * 16); kb < nkp; kb += A2_WARPS * 16) {
+            // ---- scores of this warp's 16 keys for all query rows (two accumulator sets: head and remainder products)
+            float S[MT][2][4];
+            {
+                float Sp[2][MT][2][4];
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int nt = 0; nt < 2; ++nt) { Sp[c][mt][nt][0] = Sp[c][mt][nt][1] = Sp[c][mt][nt][2] = Sp[c][mt][nt][3] = 0.f; }
+                const int krow = kb + (lane & 7) + (lane >> 4) * 8;
+                const unsigned char *krp = K_s + (size_t)krow * pitch;
+                const int ksw = krow & swz, kc0 = (lane >> 3) & 1;
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks) {
+                    uint32_t bk[4];
+                    ldsm_x4(bk, krp + (((ks * 2 + kc0) ^ ksw) << 4));
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        uint32_t ah[4], al[4];
+                        const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
+                        ldsm_x4(ah, Qh_s + qo);
+                        ldsm_x4(al, Ql_s + qo);
+                        mma_bf16(Sp[0][mt][0], ah, bk[0], bk[1]); mma_bf16(Sp[0][mt][1], ah, bk[2], bk[3]);
+                        mma_bf16(Sp[1][mt][0], al, bk[0], bk[1]); mma_bf16(Sp[1][mt][1], al, bk[2], bk[3]);
+                    }
+                }
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) { Sp[c][mt][nt][0] = Sp[c][mt][nt][1] = Sp[c][mt][nt][2] = Sp[c][mt][nt][3] = 0.f; }
+                    for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int ks = 0; ks < HD / 16; ++ks) {
-                uint32_t bk[4];
-                ldsm_x4(bk, K_s + (size_t)(kb + (lane & 7) + (lane >> 4) * 8) * KSTR + ks * 16 + ((lane >> 3) & 1) * 8);
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    uint32_t ah[4], al[4];
-                    const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
-                    ldsm_x4(ah, Qh_s + qo);
-                    ldsm_x4(al, Ql_s + qo);
-                    mma_bf16(Sp[0][mt][0], ah, bk[0], bk[1]); mma_bf16(Sp[0][mt][1], ah, bk[2], bk[3]);
-                    mma_bf16(Sp[1][mt][0], al, bk[0], bk[1]); mma_bf16(Sp[1][mt][1], al, bk[2], bk[3]);
-                }
+                        for (int e = 0; e < 4; ++e) S[mt][nt][e] = Sp[0][mt][nt][e] + Sp[1][mt][nt][e];
             }
+            // ---- masks, running softmax, probabilities as operand fragments
+            uint32_t ph[MT][4], pl[MT][4];
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
+            for (int mt = 0; mt < MT; ++mt) {
+                float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) S[mt][nt][e] = Sp[0][mt][nt][e] + Sp[1][mt][nt][e];
-        }
-        // ---- masks, running softmax, probabilities as operand fragments
-        uint32_t ph[MT][4], pl[MT][4];
+                    for (int e = 0; e < 4; ++e) {
+                        const int key = kb + nt * 8 + 2 * t4 + (e & 1);
+                        if (key >= nkeys || (newrows && key > ti[mt][e >> 1])) S[mt][nt][e] = -INFINITY;
+                        mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
+                    }
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            float mx[2] = {-INFINITY, -INFINITY};
+                for (int r = 0; r < 2; ++r) {
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                    const float mnew = fmaxf(m_run[mt][r], mx[r]);
+                    const float muse = mnew == -INFINITY ? 0.f : mnew;
+                    const float corr = __expf(m_run[mt][r] - muse);
+                    m_run[mt][r] = mnew;
+                    float sum = 0.f;
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
+                    for (int nt = 0; nt < 2; ++nt) {
+                        const float p0 = __expf(S[mt][nt][2 * r] - muse), p1 = __expf(S[mt][nt][2 * r + 1] - muse);
+                        sum += p0 + p1;
+                        __nv_bfloat16 h0, l0, h1, l1;
+                        split_bf16(p0, h0, l0); split_bf16(p1, h1, l1);
+                        ph[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                        pl[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                    }
+                    l_run[mt][r] = fmaf(l_run[mt][r], corr, sum);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int key = kb + nt * 8 + 2 * t4 + (e & 1);
-                    if (key >= nkeys || (with_new && key >= ncache && key - ncache > ti[mt][e >> 1])) S[mt][nt][e] = -INFINITY;
-                    mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
+                    for (int nt = 0; nt < NT; ++nt) { O[mt][nt][2 * r] *= corr; O[mt][nt][2 * r + 1] *= corr; }
                 }
+            }
+            // ---- partial output += P V over the whole head dimension
+            const int vrow = kb + (lane & 7) + ((lane >> 3) & 1) * 8;
+            const unsigned char *vrp = V_s + (size_t)vrow * pitch;
+            const int vsw = vrow & swz, vc0 = lane >> 4;
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-                const float mnew = fmaxf(m_run[mt][r], mx[r]);
-                const float muse = mnew == -INFINITY ? 0.f : mnew;
-                const float corr = __expf(m_run[mt][r] - muse);
-                m_run[mt][r] = mnew;
-                float sum = 0.f;
+            for (int p = 0; p < NT / 2; ++p) {
+                uint32_t bv[4];
+                ldsm_x4_t(bv, vrp + (((p * 2 + vc0) ^ vsw) << 4));
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-                    const float p0 = __expf(S[mt][nt][2 * r] - muse), p1 = __expf(S[mt][nt][2 * r + 1] - muse);
-                    sum += p0 + p1;
-                    __nv_bfloat16 h0, l0, h1, l1;
-                    split_bf16(p0, h0, l0); split_bf16(p1, h1, l1);
-                    ph[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    pl[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                for (int mt = 0; mt < MT; ++mt) {
+                    mma_bf16(O[mt][2 * p], ph[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], ph[mt], bv[2], bv[3]);
+                    mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
                 }
-                l_run[mt][r] = fmaf(l_run[mt][r], corr, sum);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) { O[mt][nt][2 * r] *= corr; O[mt][nt][2 * r + 1] *= corr; }
             }
-        }
-        // ---- partial output += P V over the whole head dimension
-#pragma unroll
-        for (int p = 0; p < NT / 2; ++p) {
-            uint32_t bv[4];
-            ldsm_x4_t(bv, V_s + (size_t)(kb + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + p * 16 + (lane >> 4) * 8);
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                mma_bf16(O[mt][2 * p], ph[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], ph[mt], bv[2], bv[3]);
-                mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
-            }
-        }
         }
     }
     cp_async_wait_all();
