@@ -85,6 +85,12 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// two floats rounded to bf16 (nearest even) and packed: lo in bits 0-15, hi in bits 16-31
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 // x = head + remainder, both bf16 (round to nearest): exact to 2^-17 relative
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &h, __nv_bfloat16 &l) {
     h = __float2bfloat16_rn(x);
@@ -1051,18 +1057,25 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                         for (int e = 0; e < 4; ++e) S[mt][nt][e] = Sp[0][mt][nt][e] + Sp[1][mt][nt][e];
             }
             // ---- masks, running softmax, probabilities as operand fragments
+            const bool edge = newrows || kb + 16 > nkeys;
             uint32_t ph[MT][4], pl[MT][4];
+            float corr_all[MT][2];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 float mx[2] = {-INFINITY, -INFINITY};
+                if (edge) {                 // only a ragged last group and the new rows have anything to mask
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int key = kb + nt * 8 + 2 * t4 + (e & 1);
+                            if (key >= nkeys || (newrows && key > ti[mt][e >> 1])) S[mt][nt][e] = -INFINITY;
+                        }
+                }
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int key = kb + nt * 8 + 2 * t4 + (e & 1);
-                        if (key >= nkeys || (newrows && key > ti[mt][e >> 1])) S[mt][nt][e] = -INFINITY;
-                        mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
-                    }
+                    for (int e = 0; e < 4; ++e) mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
                     mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
@@ -1070,21 +1083,33 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                     const float mnew = fmaxf(m_run[mt][r], mx[r]);
                     const float muse = mnew == -INFINITY ? 0.f : mnew;
                     const float corr = __expf(m_run[mt][r] - muse);
+                    corr_all[mt][r] = corr;
                     m_run[mt][r] = mnew;
                     float sum = 0.f;
 #pragma unroll
                     for (int nt = 0; nt < 2; ++nt) {
                         const float p0 = __expf(S[mt][nt][2 * r] - muse), p1 = __expf(S[mt][nt][2 * r + 1] - muse);
                         sum += p0 + p1;
-                        __nv_bfloat16 h0, l0, h1, l1;
-                        split_bf16(p0, h0, l0); split_bf16(p1, h1, l1);
-                        ph[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                        pl[mt][r + 2 * nt] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                        // two probabilities at a time: bf16 heads packed by one conversion, remainders from the exact differences
+                        const uint32_t hh = pack_bf16x2(p0, p1);
+                        ph[mt][r + 2 * nt] = hh;
+                        pl[mt][r + 2 * nt] = pack_bf16x2(p0 - __uint_as_float(hh << 16), p1 - __uint_as_float(hh & 0xffff0000u));
                     }
                     l_run[mt][r] = fmaf(l_run[mt][r], corr, sum);
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) { O[mt][nt][2 * r] *= corr; O[mt][nt][2 * r + 1] *= corr; }
                 }
+            }
+            // the accumulators are rescaled only when some row's running maximum moved (rare after the first tiles)
+            bool moved = false;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) moved = moved || corr_all[mt][0] != 1.f || corr_all[mt][1] != 1.f;
+            if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        O[mt][nt][0] *= corr_all[mt][0]; O[mt][nt][1] *= corr_all[mt][0];
+                        O[mt][nt][2] *= corr_all[mt][1]; O[mt][nt][3] *= corr_all[mt][1];
+                    }
             }
             // ---- partial output += P V over the whole head dimension
             const int vrow = kb + (lane & 7) + ((lane >> 3) & 1) * 8;
