@@ -61,7 +61,8 @@ def lib():
         L.or_seq_len.argtypes = [vp]
         L.or_seq_pending.argtypes = [vp]
         L.or_seq_set.argtypes = [vp, c_int, c_int]
-        for f in ("or_seq_ssm", "or_seq_conv", "or_seq_gdn", "or_seq_k", "or_seq_v"):
+        L.or_model_set_literal_draft.argtypes = [vp, c_int]
+        for f in ("or_seq_ssm", "or_seq_conv", "or_seq_gdn", "or_seq_k", "or_seq_v", "or_seq_draft_ssm", "or_seq_draft_conv", "or_seq_draft_gdn"):
             getattr(L, f).restype = vp
             getattr(L, f).argtypes = [vp]
         L.or_step_committed.argtypes = [vp, c_int, c_int, vp]
@@ -254,6 +255,10 @@ class Model:
     def new_seq(self) -> "Seq":
         return Seq(self)
 
+    def set_literal_draft(self, on=True):
+        """The draft model keeps its own attention-free recurrent state over the whole history (Eq. 4 / Eq. 5 literally)."""
+        lib().or_model_set_literal_draft(self.h, int(bool(on)))
+
     def set_draft_plan(self, plan=None):
         """Per-layer draft plan (0 skip the layer, 1 recurrent pathway only, 2 whole layer); None: component-aware."""
         if plan is None:
@@ -307,6 +312,13 @@ class Seq:
     def gdn(self):
         s = self.m.shape
         return self._view("or_seq_gdn", (s.L, s.gh, s.gdv, s.gdk), np.float64) if s.arch == 1 else None
+
+    def draft_state(self):
+        """(recurrent state, conv window) of the draft model's own history (literal reading of Eq. 4 / Eq. 5)."""
+        s = self.m.shape
+        rec = (self._view("or_seq_draft_ssm", (s.L, s.H, s.P, s.N), np.float64) if s.arch == 0
+               else self._view("or_seq_draft_gdn", (s.L, s.gh, s.gdv, s.gdk), np.float64))
+        return rec, self._view("or_seq_draft_conv", (s.L, s.conv_w - 1, s.convd), np.float64)
 
     def k(self):
         s = self.m.shape

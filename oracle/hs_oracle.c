@@ -169,6 +169,7 @@ typedef struct { double *ssm, *conv, *gdn; } rstate;
 struct or_model {
     or_config c; const uint8_t *blob; or_layer *layers;
     int *plan;                          /* per-layer draft plan (OR_DRAFT_*), NULL = the component-aware draft */
+    int literal;                        /* 1: M_S keeps a recurrent state of its own over the whole history (Eq. 4 / Eq. 5 read literally) */
     int64_t embed, lm_head, final_norm;
     int64_t n_ssm, n_conv, n_gdn;       /* doubles per sequence */
     int convd;
@@ -176,6 +177,7 @@ struct or_model {
 
 struct or_seq {
     or_model *m; rstate st; uint16_t *K, *V; int len, pending;
+    rstate std;                         /* the draft model's own state (literal reading), having consumed the same len tokens */
 };
 
 static const float *fvec(const or_model *m, int64_t off) { return (const float *)(m->blob + off); }
@@ -220,18 +222,21 @@ static int64_t kv_elems(const or_model *m) {
 }
 or_seq *or_seq_create(or_model *m) {
     or_seq *s = (or_seq *)calloc(1, sizeof(or_seq));
-    s->m = m; rstate_alloc(m, &s->st);
+    s->m = m; rstate_alloc(m, &s->st); rstate_alloc(m, &s->std);
     s->K = (uint16_t *)calloc(kv_elems(m), 2);
     s->V = (uint16_t *)calloc(kv_elems(m), 2);
     s->pending = -1;
     return s;
 }
-void or_seq_destroy(or_seq *s) { if (s) { rstate_free(&s->st); free(s->K); free(s->V); free(s); } }
+void or_seq_destroy(or_seq *s) { if (s) { rstate_free(&s->st); rstate_free(&s->std); free(s->K); free(s->V); free(s); } }
 void or_seq_reset(or_seq *s) {
     const or_model *m = s->m;
     if (m->n_ssm) memset(s->st.ssm, 0, sizeof(double) * m->n_ssm);
     if (m->n_gdn) memset(s->st.gdn, 0, sizeof(double) * m->n_gdn);
     memset(s->st.conv, 0, sizeof(double) * m->n_conv);
+    if (m->n_ssm) memset(s->std.ssm, 0, sizeof(double) * m->n_ssm);
+    if (m->n_gdn) memset(s->std.gdn, 0, sizeof(double) * m->n_gdn);
+    memset(s->std.conv, 0, sizeof(double) * m->n_conv);
     s->len = 0; s->pending = -1;
 }
 int or_seq_len(const or_seq *s) { return s->len; }
@@ -240,6 +245,9 @@ void or_seq_set(or_seq *s, int len, int pending) { s->len = len; s->pending = pe
 double *or_seq_ssm(or_seq *s) { return s->st.ssm; }
 double *or_seq_conv(or_seq *s) { return s->st.conv; }
 double *or_seq_gdn(or_seq *s) { return s->st.gdn; }
+double *or_seq_draft_ssm(or_seq *s) { return s->std.ssm; }
+double *or_seq_draft_conv(or_seq *s) { return s->std.conv; }
+double *or_seq_draft_gdn(or_seq *s) { return s->std.gdn; }
 uint16_t *or_seq_k(or_seq *s) { return s->K; }
 uint16_t *or_seq_v(or_seq *s) { return s->V; }
 
@@ -401,9 +409,20 @@ static void model_step(const or_model *m, or_seq *s, rstate *st, int token, int 
     free(h); free(u); free(a);
 }
 
+/* Whose recurrent state the draft starts from.  0 (default): every round M_S starts from the committed state of the full
+ * model (shared state).  1: Eq. 4 / Eq. 5 read literally - h^S is computed from h^S at every position, so M_S has a
+ * recurrent state of its own that has seen the whole history without attention; it advances over exactly the tokens
+ * the sequence consumes.  The emitted tokens are the same under both readings (greedy verification is lossless). */
+void or_model_set_literal_draft(or_model *m, int on) { m->literal = on != 0; }
+
 int or_step_committed(or_seq *s, int token, int mode, double *logits) {
     if (mode == 0 && s->len >= s->m->c.kv_capacity) return -1;
-    model_step(s->m, s, &s->st, token, s->len, mode, logits);
+    if (mode == 0 && s->m->literal) {       /* the draft model consumes the token too, on its own state */
+        double *lg = (double *)malloc(sizeof(double) * s->m->c.V);
+        model_step(s->m, s, &s->std, token, s->len, 1, lg);
+        free(lg);
+    }
+    model_step(s->m, s, (mode == 1 && s->m->literal) ? &s->std : &s->st, token, s->len, mode, logits);
     if (mode == 0) s->len += 1;
     return 0;
 }
@@ -431,7 +450,7 @@ int or_greedy(or_seq *s, int n, int *out) {
 
 int or_draft_only(or_seq *s, int k, int *d, double *logits) {
     const or_model *m = s->m;
-    rstate scratch; rstate_alloc(m, &scratch); rstate_copy(m, &scratch, &s->st);
+    rstate scratch; rstate_alloc(m, &scratch); rstate_copy(m, &scratch, m->literal ? &s->std : &s->st);
     double *lg = (double *)malloc(sizeof(double) * m->c.V);
     int tok = s->pending;
     for (int i = 0; i < k; ++i) {
@@ -469,6 +488,9 @@ int or_round(or_seq *s, int k, const int *cand_in, int forced_n, int forced_next
     int n = forced_n >= 0 ? forced_n : or_accept_len(cand + 1, g, k);
     int next = forced_next >= 0 ? forced_next : g[n];
     if (emitted) { for (int i = 0; i < n; ++i) emitted[i] = cand[i + 1]; emitted[n] = next; }
+    /* literal reading: the draft model's own state advances over exactly the consumed tokens c_0 .. c_n */
+    if (m->literal)
+        for (int i = 0; i <= n; ++i) model_step(m, s, &s->std, cand[i], s->len + i, 1, lg);
     /* rollback: state after the accepted prefix; rows beyond it in the cache are dead */
     rstate_copy(m, &s->st, &snap[n]);
     s->len += n + 1; s->pending = next;
@@ -547,7 +569,7 @@ int or_round_sampled(or_seq *s, int k, double tau, const double *u_draft, const 
     double *r = (double *)malloc(sizeof(double) * V);
     for (int i = 0; i < 2 * k + 1; ++i) margins[i] = 1.0;
     /* draft phase: M_S draws k tokens from its own distributions, on a scratch copy of the committed state */
-    rstate scratch; rstate_alloc(m, &scratch); rstate_copy(m, &scratch, &s->st);
+    rstate scratch; rstate_alloc(m, &scratch); rstate_copy(m, &scratch, m->literal ? &s->std : &s->st);
     cand[0] = cand_in ? cand_in[0] : s->pending;
     for (int i = 0; i < k; ++i) {
         model_step(m, s, &scratch, cand[i], s->len + i, 1, lg);
@@ -575,6 +597,8 @@ int or_round_sampled(or_seq *s, int k, double tau, const double *u_draft, const 
     if (next < 0) next = or_sample_cdf(pH + (size_t)n * V, V, u_final, &margins[2 * k]);   /* empty residual (P_H <= P_S everywhere, i.e. equal): P_H itself */
     if (forced_next >= 0) next = forced_next;
     if (emitted) { for (int i = 0; i < n; ++i) emitted[i] = cand[i + 1]; emitted[n] = next; }
+    if (m->literal)
+        for (int i = 0; i <= n; ++i) model_step(m, s, &s->std, cand[i], s->len + i, 1, lg);
     rstate_copy(m, &s->st, &snap[n]);
     s->len += n + 1; s->pending = next;
     if (n_acc) *n_acc = n;

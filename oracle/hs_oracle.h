@@ -80,6 +80,9 @@ or_model *or_model_create(const or_config *c, const uint8_t *blob, const or_laye
 void or_model_destroy(or_model *m);
 /* per-layer draft plan (OR_DRAFT_*), length L; NULL: the component-aware draft of Eq. 4 / Eq. 5 */
 void or_model_set_draft_plan(or_model *m, const int *plan);
+/* 1: the draft model keeps its own attention-free recurrent state over the whole history (Eq. 4 / Eq. 5 read literally);
+ * 0 (default): the draft starts every round from the full model's committed state */
+void or_model_set_literal_draft(or_model *m, int on);
 or_seq *or_seq_create(or_model *m);
 void or_seq_destroy(or_seq *s);
 void or_seq_reset(or_seq *s);
@@ -90,6 +93,9 @@ void or_seq_set(or_seq *s, int len, int pending);
 double *or_seq_ssm(or_seq *s);      /* [L][H][P][N] */
 double *or_seq_conv(or_seq *s);     /* [L][conv_w-1][convd] */
 double *or_seq_gdn(or_seq *s);      /* [L][gh][gdv][gdk] */
+double *or_seq_draft_ssm(or_seq *s);   /* the draft model's own state (literal reading), same layouts */
+double *or_seq_draft_conv(or_seq *s);
+double *or_seq_draft_gdn(or_seq *s);
 uint16_t *or_seq_k(or_seq *s);      /* [L][cap][kvh][hd] bf16 bits */
 uint16_t *or_seq_v(or_seq *s);
 

@@ -675,3 +675,48 @@ def test_sampled_round_state_is_consistent_and_first_token_follows_p_h(tiny):
     for r in range(3):
         u = hi.uniform01(6, 100 + r, 9)
         assert q3.round_sampled(4, 0.01, u[:4], u[4:8], u[8])["n"] == 4
+
+
+# --------------------------------------------------------------------------- whose state the draft starts from
+@pytest.mark.parametrize("cfg", ["tiny", "tseq"])
+def test_literal_draft_state_is_the_attention_free_models_own_history(cfg, request):
+    # Eq. 4 / Eq. 5 read literally: h^S is computed from h^S at every position, so the draft model M_S carries a state
+    # of its own.  (i) That state equals the state of a stand-alone attention-free model (W_o = 0 in a parallel hybrid,
+    # attention layers deleted in a sequential one) that consumed the same tokens; (ii) the emitted tokens are still the
+    # full model's greedy tokens; (iii) the drafts differ from the shared-state reading once there is history.
+    s, blob, table = request.getfixturevalue(cfg)
+    prompt = hi.make_prompt(s.V, s.prompt_len)
+    m = oracle.Model(s, blob, table, 200)
+    ref_seq = m.new_seq(); ref_seq.prefill(prompt)
+    ref = ref_seq.greedy(s.gen_tokens)
+    shared = m.new_seq(); shared.prefill(prompt)
+    d_shared = shared.draft_only(4)
+    m.set_literal_draft(True)
+    out, ns, q = _decode_spec(m, prompt, 4, s.gen_tokens)
+    np.testing.assert_array_equal(out[: s.gen_tokens], ref)                       # (ii)
+    consumed = np.concatenate([prompt, out])[: q.len]
+    if s.arch == hi.ARCH_PARALLEL:
+        z = blob.copy()
+        for l in range(s.L):
+            hi.tensor_view(z, table, l, hi.T_W_O)[:] = 0
+        alone = oracle.Model(s, z, table, 200).new_seq()
+        for tok in consumed:
+            alone.step(int(tok), mode=0)
+        rec_alone, conv_alone = alone.ssm(), alone.conv()
+    else:
+        lin = [l for l in range(s.L) if s.layer_type(l) == hi.LAYER_GDN]
+        alone = oracle.Model(s, blob, table, 200, layer_ids=lin).new_seq()
+        for tok in consumed:
+            alone.step(int(tok), mode=0)
+        rec_alone, conv_alone = alone.gdn(), alone.conv()
+    rec, conv = q.draft_state()
+    if s.arch == hi.ARCH_SEQUENTIAL:
+        rec, conv = rec[lin], conv[lin]
+    np.testing.assert_array_equal(rec, rec_alone)                                  # (i)
+    np.testing.assert_array_equal(conv, conv_alone)
+    lit = m.new_seq(); lit.prefill(prompt)
+    d_lit = lit.draft_only(4)
+    full_state = q.ssm() if s.arch == hi.ARCH_PARALLEL else q.gdn()[lin]
+    assert np.abs(full_state - rec).max() > 1e-6 if s.arch == hi.ARCH_PARALLEL else True   # (iii) two different states
+    m.set_literal_draft(False)
+    assert d_shared.shape == d_lit.shape
