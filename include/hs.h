@@ -68,11 +68,20 @@ typedef struct hs_config {
 
 enum {
     HS_FLAG_GRAPHS = 1,        /* replay each (mode, k, batch) step as a captured CUDA graph */
-    HS_FLAG_REPLAY = 2         /* rollback by replay: verify keeps no per-position state snapshots but a small log of
+    HS_FLAG_REPLAY = 2,        /* rollback by replay: verify keeps no per-position state snapshots but a small log of
                                   the k+1 state updates (Mamba-2: decay, dt*x, B; DeltaNet: alpha, beta, k, v), and
                                   hs_accept_rollback applies the accepted n+1 updates to the committed state in place.
                                   State traffic per verify round: 3 state units (read, read, write) instead of k+2;
                                   the snapshot buffer shrinks to one state per sequence plus the log.  Same results. */
+    HS_FLAG_LITERAL_DRAFT = 4  /* whose recurrent state the draft starts from.  Default (flag clear): every round the draft
+                                  starts from the committed state of the full model.  With the flag, Eq. 4 / Eq. 5 are read
+                                  literally: the draft model M_S keeps a recurrent state and conv window of its own, which have
+                                  seen the whole history without attention and advance over exactly the tokens a round
+                                  consumes (hs_prefill runs M_S over the prompt as well; a round runs k+1 draft steps, the
+                                  last one only to consume d_k).  The emitted tokens are the same (greedy verification is
+                                  lossless); the acceptance rate of real weights and the cost of a round differ.  The draft
+                                  scratch buffer grows to max_k+2 states per sequence.  Only with draft plans that keep no
+                                  attention. */
 };
 
 /* Bytes the caller must provide (each buffer 256-byte aligned). */
@@ -210,7 +219,9 @@ enum { HS_STATE_SSM = 0,   /* f32 [H][P][N] committed Mamba-2 state of (layer, s
        HS_STATE_GDN = 2,   /* f32 [gh][gdv][gdk] committed DeltaNet state */
        HS_STATE_K = 3,     /* bf16 [rows][kvh][hd], rows = bytes / (kvh*hd*2), from row 0 */
        HS_STATE_V = 4,
-       HS_STATE_DRAFT = 5  /* f32 draft scratch state after the last hs_draft (export only) */ };
+       HS_STATE_DRAFT = 5, /* f32 draft scratch state after the last hs_draft; with HS_FLAG_LITERAL_DRAFT the draft
+                              model's own committed state (export only) */
+       HS_STATE_DRAFT_CONV = 6 /* f32 [3][channels] the draft model's own committed conv window (HS_FLAG_LITERAL_DRAFT; export only) */ };
 int hs_export_state(hs_model *m, int layer, int seq, int kind, void *host, int64_t bytes);
 int hs_import_state(hs_model *m, int layer, int seq, int kind, const void *host, int64_t bytes);
 /* Declare sequence `seq` to hold kv_len consumed tokens and the given pending token (after imports);

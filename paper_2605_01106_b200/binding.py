@@ -16,7 +16,8 @@ i32, i64, f32, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_voi
 
 HS_FLAG_GRAPHS = 1
 HS_FLAG_REPLAY = 2
-STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT = range(6)
+HS_FLAG_LITERAL_DRAFT = 4
+STATE_SSM, STATE_CONV, STATE_GDN, STATE_K, STATE_V, STATE_DRAFT, STATE_DRAFT_CONV = range(7)
 EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "hs_prefill", "hs_draft", "hs_verify",
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
@@ -283,7 +284,7 @@ class Engine:
             return (s.gh, s.gdv, s.gdk), np.float32
         if kind == STATE_DRAFT:
             return ((s.H, s.P, s.N) if s.arch == 0 else (s.gh, s.gdv, s.gdk)), np.float32
-        if kind == STATE_CONV:
+        if kind in (STATE_CONV, STATE_DRAFT_CONV):
             return (s.conv_w - 1, s.convd), np.float32
         return (rows, s.kvh, s.hd), np.uint16
 

@@ -97,6 +97,7 @@ bool valid_config(const hs_config &c) {
 struct Derived {
     int B, Tm, R, n_rl, n_al, convd, gw, in_rows_max, att_chunk, att_nch;
     int nslot, log_w;         // state slots per (layer, sequence); floats of one logged update (rollback by replay)
+    int literal;              // the draft model keeps its own state: a ring of Tm + 1 draft slots, a second set of conv buffers
     int64_t state_elems;
 };
 
@@ -116,6 +117,7 @@ Derived derive(const hs_config &c) {
     v.state_elems = c.arch == HS_ARCH_PARALLEL ? (int64_t)c.H * c.P * c.N : (int64_t)c.gh * c.gdv * c.gdk;
     const bool replay = (c.flags & HS_FLAG_REPLAY) != 0;
     v.nslot = replay ? 1 : v.Tm;
+    v.literal = (c.flags & HS_FLAG_LITERAL_DRAFT) ? 1 : 0;
     v.log_w = !replay ? 0 : c.arch == HS_ARCH_PARALLEL ? c.H + c.H * c.P + c.N : c.gh * (2 + c.gdk + c.gdv);
     // keys per attention CTA: the largest of 128 / 64 / 32 that still gives about two CTAs per SM
     int chunk = 128;
@@ -127,7 +129,7 @@ Derived derive(const hs_config &c) {
 
 // layout of the work buffer; base may be null to only measure
 struct WorkLayout {
-    int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters;
+    int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters, dslot;
     int64_t rope, h, zx, gbuf, obuf, abuf, logits, dlogits, att_acc, att_ml, am_part, xb, total;
 };
 
@@ -139,6 +141,7 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.n_acc = take(4 * v.B); w.emitted = take(4 * v.R);
     w.stage_n = take(4 * v.B); w.stage_next = take(4 * v.B);
     w.status = take(4); w.counters = take((int64_t)4 * v.B * c.kvh); w.am_counters = take((int64_t)4 * v.R);
+    w.dslot = take(4 * v.B);
     w.rope = take((int64_t)c.kv_capacity * (c.hd / 2) * 8);
     w.h = take((int64_t)4 * 2 * HS_H_PARTS * v.R * c.d);
     w.zx = take((int64_t)4 * v.R * v.in_rows_max);
@@ -245,7 +248,9 @@ inline bool draft_runs(const hs_model *m, int l) {
 
 // first = true: this pass opens an API call (its predecessor in the stream may be the accept kernel of the last
 // round): its first kernel goes out in plain stream order, see hs_device.cuh.
-int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool first) {
+// chunk = true (literal draft state only): the DRAFT model over T positions of every sequence on its own state buffers,
+// like a verify pass of M_S (prompt chunks; candidates supplied by the caller); head = false: no LM head / token choice.
+int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool first, bool chunk = false, bool head = true) {
     const hs_config &c = m->c;
     const AttnGeom at_geom = draft ? attn_geom(m, 1, m->last_draft_k, b0, nb) : attn_geom(m, T, T, b0, nb);
     cudaStream_t s = m->stream;
@@ -281,13 +286,19 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         if (ly.type != HS_LAYER_ATT) {
             const size_t lrB = (size_t)ly.rl * m->B;
             const float *win_in; float *win_out = nullptr, *hist = nullptr;
+            const size_t half = (size_t)m->n_rl * m->B * 3 * m->convd;
+            const bool lit = draft && m->literal;          // the draft model runs on its own state buffers
             if (!draft) { win_in = m->cw + lrB * 3 * m->convd; hist = m->hist + lrB * m->Tm * m->convd; }
+            else if (chunk) { win_in = m->dcwc + lrB * 3 * m->convd; hist = m->dhist + lrB * m->Tm * m->convd; }
             else {
-                const size_t half = (size_t)m->n_rl * m->B * 3 * m->convd;
-                win_in = step == 0 ? m->cw + lrB * 3 * m->convd : m->dcw + ((step - 1) & 1) * half + lrB * 3 * m->convd;
+                const float *committed = lit ? m->dcwc : m->cw;
+                win_in = step == 0 ? committed + lrB * 3 * m->convd : m->dcw + ((step - 1) & 1) * half + lrB * 3 * m->convd;
                 win_out = m->dcw + (step & 1) * half + lrB * 3 * m->convd;
+                if (lit) hist = m->dhist + lrB * m->Tm * m->convd + (size_t)step * m->convd;     // raw inputs of draft position `step`
             }
             const float *st_in; int64_t in_seq, in_slot; float *st_out; int64_t out_seq, out_slot;
+            const int32_t *slot_arr = m->ctrl.slot;
+            int in_add = 0, out_rel = 0, out_add = 0, slot_mod = 0;
             // snapshots: slot i of (layer, sequence) holds the state after position i and `slot` names the committed one;
             // rollback by replay: one slot, the committed state, and the verify pass writes the update log instead
             const int64_t ns = m->nslot;
@@ -295,6 +306,15 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
             float *snap_l = m->snap + lrB * ns * se, *dst_l = m->dstate + lrB * se;
             float *log_l = (!draft && replay) ? m->ulog + lrB * m->Tm * m->log_w : nullptr;
             if (!draft) { st_in = snap_l; in_seq = ns * se; in_slot = replay ? 0 : se; st_out = snap_l; out_seq = ns * se; out_slot = replay ? 0 : se; }
+            else if (lit) {
+                // literal draft state: a ring of Tm + 1 slots per (layer, sequence); the committed slot dslot[b] is never
+                // overwritten during a round: draft position i reads slot dslot + i and writes slot dslot + i + 1
+                const int64_t dn = m->Tm + 1;
+                float *ring = m->dstate + lrB * dn * se;
+                st_in = ring; in_seq = dn * se; in_slot = se; st_out = ring; out_seq = dn * se; out_slot = se;
+                slot_arr = m->ctrl.dslot; slot_mod = (int)dn; out_rel = 1;
+                in_add = chunk ? 0 : step; out_add = chunk ? 1 : step + 1;
+            }
             else if (step == 0) { st_in = snap_l; in_seq = ns * se; in_slot = replay ? 0 : se; st_out = dst_l; out_seq = se; out_slot = 0; }
             else { st_in = dst_l; in_seq = se; in_slot = 0; st_out = dst_l; out_seq = se; out_slot = 0; }
             if (ly.type == HS_LAYER_PAR) {
@@ -304,7 +324,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 sa.win_in = win_in; sa.win_out = win_out; sa.hist = hist;
                 sa.state_in = st_in; sa.in_seq_stride = in_seq; sa.in_slot_stride = in_slot;
                 sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
-                sa.slot = m->ctrl.slot; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
+                sa.slot = slot_arr; sa.in_add = in_add; sa.out_rel = out_rel; sa.out_add = out_add; sa.slot_mod = slot_mod; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
                 sa.log = log_l; sa.log_w = m->log_w;
                 if (with_attn) { ssm_args = sa; ssm_deferred = true; }      // goes out together with the attention
                 else PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
@@ -315,7 +335,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 gd.win_in = win_in; gd.win_out = win_out; gd.hist = hist;
                 gd.state_in = st_in; gd.in_seq_stride = in_seq; gd.in_slot_stride = in_slot;
                 gd.state_out = st_out; gd.out_seq_stride = out_seq; gd.out_slot_stride = out_slot;
-                gd.slot = m->ctrl.slot; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
+                gd.slot = slot_arr; gd.in_add = in_add; gd.out_rel = out_rel; gd.out_add = out_add; gd.slot_mod = slot_mod; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
                 gd.log = log_l; gd.log_w = m->log_w;
                 PROF(HS_PROF_MIXER, 0, launch_gdn(gd, s), "gdn");
             }
@@ -389,6 +409,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, st_w, s, &m->launches, &hparts), "down");
         cur ^= 1;
     }
+    if (!head) { m->last_rows = 0; return HS_OK; }       // the draft model only had to consume these positions
     // final norm + LM head, then greedy argmax
     GemvArgs lm{};
     lm.W0 = m->lm_head; lm.ldw0 = d; lm.K0 = d; lm.x0 = m->hbuf[cur]; lm.ldx0 = d; lm.xparts = hparts; lm.xpstride = hps;
@@ -415,6 +436,9 @@ int enqueue_draft(hs_model *m, int k, int b0, int nb) {
     // a draft that keeps attention reads, in a step's attention prologue, the scratch KV row the previous step wrote:
     // then every step opens in plain stream order
     for (int st = 0; st < k; ++st) { int rc = model_pass(m, true, 1, st, b0, nb, st == 0 || m->plan_attn); if (rc) return rc; }
+    // literal draft state: the draft model must also have consumed the last candidate (d_k; the pending token when k = 0)
+    // if the round accepts everything - one more step without the LM head
+    if (m->literal) { int rc = model_pass(m, true, 1, k, b0, nb, k == 0, false, false); if (rc) return rc; }
     return HS_OK;
 }
 
@@ -422,6 +446,7 @@ int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const 
     AcceptArgs a{};
     a.k = k; a.Tm = m->Tm; a.b0 = b0; a.nb = nb; a.n_rl = m->n_rl; a.B = m->B; a.convd = m->convd; a.V = m->c.V;
     a.ctrl = m->ctrl; a.forced_n = fn; a.forced_next = fx; a.cw = m->cw; a.hist = m->hist; a.replay = m->log_w != 0;
+    if (m->literal) { a.dcw = m->dcwc; a.dhist = m->dhist; a.dslot = m->ctrl.dslot; a.dslot_mod = m->Tm + 1; }
     PROF(HS_PROF_ACCEPT, 0, launch_accept(a, m->stream), "accept");
     ++m->launches;
     if (m->log_w && m->n_rl > 0) {
@@ -480,8 +505,8 @@ int hs_query_sizes(const hs_config *cfg, hs_sizes *out) {
     Derived v = derive(c);
     out->weights = blob_offset(c, c.L, 0);
     out->snap = up((int64_t)4 * v.n_rl * v.B * (v.nslot * v.state_elems + (int64_t)v.Tm * v.log_w));
-    out->dstate = up((int64_t)4 * v.n_rl * v.B * v.state_elems);
-    out->conv = up((int64_t)4 * v.n_rl * v.B * v.convd * (3 + v.Tm + 6));
+    out->dstate = up((int64_t)4 * v.n_rl * v.B * v.state_elems * (v.literal ? v.Tm + 1 : 1));
+    out->conv = up((int64_t)4 * v.n_rl * v.B * v.convd * (3 + v.Tm + 6 + (v.literal ? 3 + v.Tm : 0)));
     out->kv = up((int64_t)2 * 2 * v.n_al * v.B * c.kvh * c.kv_capacity * c.hd);
     out->work = work_layout(c, v).total;
     return HS_OK;
@@ -547,6 +572,7 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->ctrl.n_acc = (int32_t *)(w + wl.n_acc); m->ctrl.emitted = (int32_t *)(w + wl.emitted);
     m->ctrl.stage_n = (int32_t *)(w + wl.stage_n); m->ctrl.stage_next = (int32_t *)(w + wl.stage_next);
     m->ctrl.status = (int32_t *)(w + wl.status); m->ctrl.counters = (int32_t *)(w + wl.counters); m->ctrl.am_counters = (int32_t *)(w + wl.am_counters);
+    m->ctrl.dslot = (int32_t *)(w + wl.dslot);
     m->rope = (float2 *)(w + wl.rope);
     m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
     m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits); m->dlogits = (float *)(w + wl.dlogits);
@@ -556,6 +582,8 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     float *cv = (float *)bufs->conv;
     const size_t win = (size_t)v.n_rl * v.B * 3 * v.convd;
     m->cw = cv; m->hist = cv + win; m->dcw = m->hist + (size_t)v.n_rl * v.B * v.Tm * v.convd;
+    m->literal = v.literal != 0;
+    m->dcwc = m->dcw + 2 * win; m->dhist = m->dcwc + win;        // used with the literal draft state only
     m->Kc = (__nv_bfloat16 *)bufs->kv;
     m->Vc = m->Kc + (size_t)v.n_al * v.B * c.kvh * c.kv_capacity * c.hd;
     m->snap = (float *)bufs->snap; m->dstate = (float *)bufs->dstate;
@@ -632,6 +660,7 @@ int hs_prefill(hs_model *m, const int32_t *tokens_host, const int32_t *lens_host
             if (Tb[b0] > 0) {
                 int rc = model_pass(m, false, Tb[b0], 0, b0, nb, true);
                 if (rc) return rc;
+                if (m->literal) { rc = model_pass(m, true, Tb[b0], 0, b0, nb, true, true, false); if (rc) return rc; }
                 rc = enqueue_accept(m, Tb[b0] - 1, b0, nb, m->ctrl.stage_n, nullptr);
                 if (rc) return rc;
                 for (int b = b0; b < b0 + nb; ++b) m->kv_upper[b] += Tb[b0];
@@ -648,7 +677,7 @@ int hs_draft(hs_model *m, int k) {
     if (!m || k < 0 || k > m->c.max_k) return HS_ERR_INVALID_ARG;
     if (m->batch < 1) return fail(m, HS_ERR_ORDER, "no active sequences: prefill or set_context first");
     if (m->phase == 2) return fail(m, HS_ERR_ORDER, "draft after verify: the snapshots hold the verified positions until accept_rollback");
-    if (k > 0) {
+    if (k > 0 || m->literal) {
         const int nb = m->batch;
         m->last_draft_k = k;
         uint64_t geo = 0;
@@ -677,6 +706,11 @@ int hs_verify(hs_model *m, int k, const int32_t *cand_dev) {
     if (cand_dev)
         CK(cudaMemcpy2DAsync(m->ctrl.cand, sizeof(int32_t) * m->Tm, cand_dev, sizeof(int32_t) * T, sizeof(int32_t) * T, nb,
                              cudaMemcpyDeviceToDevice, m->stream), "candidates");
+    if (m->literal && (cand_dev || m->phase != 1)) {
+        // the draft model's own state must follow the candidates that are verified, not the ones it drafted (or none)
+        rc = model_pass(m, true, T, 0, 0, nb, true, true, false);
+        if (rc) return rc;
+    }
     rc = run_maybe_graph(m, (2ull << 60) | ((uint64_t)attn_geom(m, T, T, 0, nb).code() << 32) | ((uint64_t)k << 20) | nb, [&] { return model_pass(m, false, T, 0, 0, nb, true); });
     if (rc) return rc;
     m->phase = 2; m->last_k = k;
@@ -753,7 +787,11 @@ static int state_xfer(hs_model *m, int layer, int seq, int kind, void *host, int
         float *dev;
         if (kind == HS_STATE_DRAFT) {
             if (!to_host) return HS_ERR_INVALID_ARG;
-            dev = m->dstate + ((size_t)ly.rl * m->B + seq) * m->state_elems;
+            if (m->literal) {
+                int32_t ds = 0;
+                CK(cudaMemcpy(&ds, m->ctrl.dslot + seq, 4, cudaMemcpyDeviceToHost), "draft slot read");
+                dev = m->dstate + (((size_t)ly.rl * m->B + seq) * (m->Tm + 1) + ds) * m->state_elems;
+            } else dev = m->dstate + ((size_t)ly.rl * m->B + seq) * m->state_elems;
         } else {
             int32_t slot = 0;
             if (to_host) CK(cudaMemcpy(&slot, m->ctrl.slot + seq, 4, cudaMemcpyDeviceToHost), "slot read");
@@ -763,10 +801,11 @@ static int state_xfer(hs_model *m, int layer, int seq, int kind, void *host, int
         CK(to_host ? cudaMemcpy(host, dev, bytes, dir) : cudaMemcpy(dev, host, bytes, dir), "state copy");
         return HS_OK;
     }
-    if (kind == HS_STATE_CONV) {
+    if (kind == HS_STATE_CONV || kind == HS_STATE_DRAFT_CONV) {
         if (ly.rl < 0) return fail(m, HS_ERR_INVALID_ARG, "layer has no conv window");
+        if (kind == HS_STATE_DRAFT_CONV && (!m->literal || !to_host)) return HS_ERR_INVALID_ARG;
         if (bytes != (int64_t)4 * 3 * m->convd) return fail(m, HS_ERR_SIZE, "conv window size mismatch");
-        float *dev = m->cw + ((size_t)ly.rl * m->B + seq) * 3 * m->convd;
+        float *dev = (kind == HS_STATE_CONV ? m->cw : m->dcwc) + ((size_t)ly.rl * m->B + seq) * 3 * m->convd;
         CK(to_host ? cudaMemcpy(host, dev, bytes, dir) : cudaMemcpy(dev, host, bytes, dir), "conv copy");
         return HS_OK;
     }
@@ -863,6 +902,7 @@ int hs_set_draft_plan(hs_model *m, const int32_t *plan_host) {
             plan[l] = plan_host[l];
             if (plan[l] == HS_DRAFT_FULL && m->layers[l].type != HS_LAYER_GDN) attn = true;
         }
+    if (attn && m->literal) return fail(m, HS_ERR_INVALID_ARG, "the literal draft state goes with draft plans that keep no attention");
     CK(cudaStreamSynchronize(m->stream), "plan sync");
     m->plan = plan; m->plan_attn = attn;
     for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);     // the draft graphs were captured for the old plan

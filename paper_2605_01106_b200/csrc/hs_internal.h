@@ -31,6 +31,7 @@ struct HsCtrl {
     int32_t *status;      // [1]   first error a kernel recorded
     int32_t *counters;    // [B][kvh] split-KV arrival tickets (zero between launches)
     int32_t *am_counters; // [B][Tm] argmax arrival tickets (zero between launches)
+    int32_t *dslot;       // [B]   slot of the draft model's own committed state (literal draft state)
 };
 
 struct HsLayer {
@@ -76,6 +77,8 @@ struct hs_model {
     void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
     // conv buffers
     float *cw, *hist, *dcw;
+    float *dcwc, *dhist;       // literal draft state: the draft model's committed conv window and per-step raw inputs
+    bool literal;              // the draft model keeps its own state over the whole history
     __nv_bfloat16 *Kc, *Vc;
     float *snap, *dstate;
     // host bookkeeping
@@ -172,6 +175,9 @@ struct SsmArgs {
     float *state_out;                   // verify: snapshots (slot i at i*out_slot_stride); draft: scratch
     int64_t out_seq_stride, out_slot_stride;
     const int32_t *slot;                // [B] committed slot (used when in_slot_stride != 0)
+    // slot addressing: the state is read from slot (slot[b] + in_add) % slot_mod (slot_mod = 0: no wrap) and the state
+    // after position i goes to slot i, or, with out_rel, to slot (slot[b] + out_add + i) % slot_mod
+    int in_add, out_rel, out_add, slot_mod;
     float *g;                           // [rows][di] gated output y * silu(z)
     int T, Tm, b0, nb;
     float *log; int log_w;              // verify with rollback by replay: [B][Tm][log_w] update log (decay[H] | dt*x[di] | B[N]);
@@ -187,6 +193,7 @@ struct GdnArgs {
     const float *state_in; int64_t in_seq_stride, in_slot_stride;
     float *state_out; int64_t out_seq_stride, out_slot_stride;
     const int32_t *slot;
+    int in_add, out_rel, out_add, slot_mod;   // as in SsmArgs
     float *g;                           // [rows][gh*dv]
     int T, Tm, b0, nb;
     float *log; int log_w;              // rollback by replay: [B][Tm][log_w] (alpha[gh] | beta[gh] | k[gh*dk] | v[gh*dv]); NULL otherwise
@@ -236,6 +243,8 @@ struct AcceptArgs {
     HsCtrl ctrl;
     const int32_t *forced_n, *forced_next;
     float *cw; const float *hist;       // [n_rl][B][3][convd], [n_rl][B][Tm][convd]
+    float *dcw; const float *dhist;     // the draft model's own committed window and raw inputs (literal draft state), or NULL
+    int32_t *dslot; int dslot_mod;      // its committed slot advances by n + 1 (mod dslot_mod)
 };
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t s);
 cudaError_t launch_wait_probe(int32_t *status, int polls, cudaStream_t s);

@@ -144,17 +144,20 @@ __global__ void accept_kernel(AcceptArgs a) {
     }
     // conv windows: sequence of raw inputs = [w0 w1 w2 | hist_0 .. hist_k]; new window = entries n+1..n+3
     if (rl < a.n_rl) {
-        float *cw = a.cw + ((size_t)rl * a.B + b) * 3 * a.convd;
-        const float *hist = a.hist + ((size_t)rl * a.B + b) * Tm * a.convd;
-        for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < a.convd; c += gridDim.x * blockDim.x) {
-            float v[3];
+        // the full model's window, then (literal draft state) the draft model's own: the same selection on its buffers
+        for (int which = 0; which < (a.dcw ? 2 : 1); ++which) {
+            float *cw = (which ? a.dcw : a.cw) + ((size_t)rl * a.B + b) * 3 * a.convd;
+            const float *hist = (which ? a.dhist : a.hist) + ((size_t)rl * a.B + b) * Tm * a.convd;
+            for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < a.convd; c += gridDim.x * blockDim.x) {
+                float v[3];
 #pragma unroll
-            for (int j = 0; j < 3; ++j) {
-                int e = n + 1 + j;
-                v[j] = e < 3 ? __ldcg(cw + e * a.convd + c) : __ldcg(hist + (e - 3) * a.convd + c);
+                for (int j = 0; j < 3; ++j) {
+                    int e = n + 1 + j;
+                    v[j] = e < 3 ? __ldcg(cw + e * a.convd + c) : __ldcg(hist + (e - 3) * a.convd + c);
+                }
+#pragma unroll
+                for (int j = 0; j < 3; ++j) cw[j * a.convd + c] = v[j];
             }
-#pragma unroll
-            for (int j = 0; j < 3; ++j) cw[j * a.convd + c] = v[j];
         }
     }
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
@@ -164,6 +167,7 @@ __global__ void accept_kernel(AcceptArgs a) {
         for (int i = 0; i <= k; ++i) em[i] = i < n ? d[i] : (i == n ? next : -1);
         a.ctrl.n_acc[b] = n;
         a.ctrl.slot[b] = a.replay ? 0 : n;
+        if (a.dslot) a.dslot[b] = (__ldcg(a.dslot + b) + 1 + n) % a.dslot_mod;
         a.ctrl.kv_len[b] = __ldcg(a.ctrl.kv_len + b) + n + 1;
         a.ctrl.cand[b * Tm] = next;
     }

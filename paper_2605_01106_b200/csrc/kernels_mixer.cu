@@ -36,8 +36,9 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
     pdl_trigger();          // the next kernel (out-projection) only streams weights before its own wait
     const int nk = a.gh * DK, nv = a.gh * dv;
 
-    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
-                        (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) + (size_t)h * dv * DK;
+    const int cslot = (a.in_slot_stride || a.out_rel) ? __ldcg(a.slot + b) : 0;
+    const int islot = a.slot_mod ? (cslot + a.in_add) % a.slot_mod : cslot;
+    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride + (a.in_slot_stride ? (size_t)islot * a.in_slot_stride : 0) + (size_t)h * dv * DK;
     float s[RPW][2];
     const bool rows_ok = warp * RPW < dv;
     // before the wait the state is only pulled towards L2 (it was written by an earlier kernel); it is loaded
@@ -145,7 +146,8 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
         const float o = xreduce<RPW>(part, lane);
         if (rows_ok && (lane & (LPV - 1)) == 0) os[i][warp * RPW + lane / LPV] = o * 0.125f;   // 1/sqrt(64)
         if (rows_ok && !a.log) {
-            float *dst = sout + (size_t)i * a.out_slot_stride;
+            const int oslot = a.out_rel ? (cslot + a.out_add + i) % a.slot_mod : i;
+            float *dst = sout + (size_t)oslot * a.out_slot_stride;
 #pragma unroll
             for (int r = 0; r < RPW; ++r)
                 *reinterpret_cast<float2 *>(dst + (warp * RPW + r) * DK + 2 * lane) = make_float2(s[r][0], s[r][1]);

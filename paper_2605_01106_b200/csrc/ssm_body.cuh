@@ -32,8 +32,9 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
     // ---- before the wait only parameters are read; the recurrent state (written by an earlier kernel of
     //      the step or of the previous round) is merely pulled towards L2 and loaded after the wait, together
     //      with the in-projection's outputs, so that this kernel may start as early as its predecessor allows
-    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride +
-                        (a.in_slot_stride ? (size_t)__ldcg(a.slot + b) * a.in_slot_stride : 0) +
+    const int cslot = (a.in_slot_stride || a.out_rel) ? __ldcg(a.slot + b) : 0;
+    const int islot = a.slot_mod ? (cslot + a.in_add) % a.slot_mod : cslot;
+    const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride + (a.in_slot_stride ? (size_t)islot * a.in_slot_stride : 0) +
                         ((size_t)h * a.P + p0 + warp * RPW) * N;
 #pragma unroll
     for (int r = 0; r < RPW; ++r)
@@ -189,7 +190,8 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
         }
         // state after position i (verify: snapshot i; draft: the scratch state; rollback by replay: nothing)
         if (a.log) continue;
-        float *dst = sout + (size_t)i * a.out_slot_stride;
+        const int oslot = a.out_rel ? (cslot + a.out_add + i) % a.slot_mod : i;
+        float *dst = sout + (size_t)oslot * a.out_slot_stride;
 #pragma unroll
         for (int r = 0; r < RPW; ++r)
 #pragma unroll

@@ -33,8 +33,10 @@ class Report:
 
 
 def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
-    """Committed recurrent state, conv window and KV rows of every sequence against the oracle."""
+    """Committed recurrent state, conv window and KV rows of every sequence against the oracle (and, with the literal
+    draft state, the draft model's own committed state and window)."""
     worst = 0.0
+    literal = bool(eng.cfg.flags & hs.HS_FLAG_LITERAL_DRAFT)
     for b, o in enumerate(seqs):
         if o is None:
             continue
@@ -53,6 +55,15 @@ def compare_states(eng, seqs, shape, rep=None, kv_rows=None):
                 gotc = eng.export_state(l, b, hs.STATE_CONV)
                 errc = np.abs(gotc - conv[l]).max() / max(np.abs(conv[l]).max(), 1e-30)
                 assert errc <= STATE_TOL, ("conv", l, b, errc)
+                if literal:
+                    drec, dconv = o.draft_state()
+                    gotd = eng.export_state(l, b, hs.STATE_DRAFT)
+                    errd = np.abs(gotd - drec[l]).max() / max(np.abs(drec[l]).max(), 1e-30)
+                    assert errd <= STATE_TOL, ("draft model's own state", l, b, errd)
+                    gotdc = eng.export_state(l, b, hs.STATE_DRAFT_CONV)
+                    errdc = np.abs(gotdc - dconv[l]).max() / max(np.abs(dconv[l]).max(), 1e-30)
+                    assert errdc <= STATE_TOL, ("draft model's own conv window", l, b, errdc)
+                    worst = max(worst, errd)
         n = o.len if kv_rows is None else min(kv_rows, o.len)
         for l in range(shape.L):
             if shape.layer_type(l) == hi.LAYER_GDN or n == 0:

@@ -32,6 +32,8 @@ def setup(env, name, prompt_lens, max_k, cap, flags=0, seed_seq0=0):
     blob, table = weights(name)
     eng = env["hs"].Engine(s, blob, max_batch=len(prompt_lens), max_k=max_k, kv_capacity=cap, flags=flags)
     model = env["oracle"].Model(s, blob, table, cap)
+    if flags & env["hs"].HS_FLAG_LITERAL_DRAFT:
+        model.set_literal_draft(True)
     prompts = [hi.make_prompt(s.V, n, seq=seed_seq0 + b) for b, n in enumerate(prompt_lens)]
     seqs = []
     for p in prompts:
@@ -184,6 +186,29 @@ def test_prefill_ragged_batch_matches_oracle(env):
     s, eng, model, seqs = setup(env, "test_seq", [17, 17, 4], max_k=8, cap=128, flags=1)
     env["harness"].compare_states(eng, seqs, s, kv_rows=None)
     assert eng.device_status() == 0
+
+
+@pytest.mark.parametrize("flags", [4, 5, 7])
+@pytest.mark.parametrize("name", ["cfg1_tiny", "test_seq"])
+def test_literal_draft_state_matches_oracle(env, name, flags):
+    # HS_FLAG_LITERAL_DRAFT: the draft model keeps its own attention-free state over the whole history (Eq. 4 / Eq. 5
+    # read literally): prefill runs it over the prompt, a round advances it over the consumed tokens.  Candidates,
+    # accept lengths, tokens, the full model's state AND the draft model's own state and conv window follow the oracle,
+    # with real acceptance, forced accept lengths (every n from 0 to k), k = 0 rounds, ragged prompts, graphs, replay.
+    lens = [hi.CONFIGS[name].prompt_len, 7, 22]
+    s, eng, model, seqs = setup(env, name, lens, max_k=4, cap=512, flags=flags)
+    env["harness"].compare_states(eng, seqs, s)
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 5)
+    forced = [hi.forced_accept(4, 8, seq=30 + b) for b in range(3)]
+    rep = env["harness"].run_rounds(eng, seqs, s, 4, 8, forced=forced, rep=rep)
+    rep = env["harness"].run_rounds(eng, seqs, s, 0, 2, rep=rep)
+    rep = env["harness"].run_rounds(eng, seqs, s, 2, 3, rep=rep)
+    print(name, flags, rep)
+    assert len(rep.n_hist) >= 3 and eng.device_status() == 0
+    env["harness"].run_rounds_async(eng, seqs, [2, 0, 4, 1, 0, 2])
+    env["harness"].compare_states(eng, seqs, s, kv_rows=None)
+    with pytest.raises(env["hs"].HsError):           # this reading goes with attention-free draft plans only
+        eng.set_draft_plan(hi.draft_plan(s, "full"))
 
 
 def test_draft_leaves_cache_and_committed_state_untouched(env):
