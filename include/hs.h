@@ -249,14 +249,20 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);
  * Results are the same within fp32 summation order.  Synchronises the stream.
  *   HS_OPT_CLUSTER_REDUCE  residual projections with 4..16 activation rows add the partial sums of their K split
  *                          inside a thread-block cluster (default on; off: the consumers add the parts)
- *   HS_OPT_GEMM_MMA        4..16 activation rows on the warp-level tensor path (default on; off: CUDA cores)
- *   HS_OPT_GEMM_TC         more than 16 activation rows on tcgen05 (default on; off: several 16-row launches)
+ *   HS_OPT_GEMM_MMA        4..16 activation rows below the tcgen05 threshold on the warp-level tensor path (default on;
+ *                          off: CUDA cores)
+ *   HS_OPT_GEMM_TC         projections from HS_OPT_TC_MIN_ROWS activation rows on run on tcgen05 (default on; off: the
+ *                          warp-level path, more than 16 rows as several 16-row launches)
  *   HS_OPT_PDL             programmatic dependent launch between the kernels of a pass (default on)
  *   HS_OPT_ATTN_SMALL      verify attention with at most 16 query rows per KV head over caches of up to 1024 keys
  *                          (2048 in a sequential hybrid) in its latency-lean form (default on; off: the general form)
  *   HS_OPT_ATTN_STREAM     verify attention over long caches at large batch (a launch of its own, at most 32 query rows
- *                          per KV head) in its streaming form (default on; off: the general form) */
-enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4, HS_OPT_ATTN_STREAM = 5 };
+ *                          per KV head) in its streaming form (default on; off: the general form)
+ *   HS_OPT_TC_MIN_ROWS     not a switch: the smallest number of activation rows (2..17) whose projections run on
+ *                          tcgen05; 0 restores the automatic choice (7; 5 for models whose weight matrices are large
+ *                          enough that the kernel's fixed cost is small beside the time to stream them) */
+enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4, HS_OPT_ATTN_STREAM = 5,
+       HS_OPT_TC_MIN_ROWS = 6 };
 int hs_set_option(hs_model *m, int option, int value);
 /* Measurement hook.  hs_profile(m, 1) brackets every following kernel launch with two CUDA events on
  * the launching stream (graph replay is bypassed while it is on); hs_profile_read synchronises and
@@ -275,6 +281,16 @@ int hs_clear_status(hs_model *m);
  * mbarrier nothing will ever complete, gives up and records HS_ERR_TIMEOUT, which hs_device_status then returns.
  * The kernel ends by itself; the handle stays usable (hs_clear_status).  Async. */
 int hs_selftest_wait_timeout(hs_model *m, int polls);
+/* Self-test of the kernels' own range checks: overwrites ONE device control word of sequence `seq` without the
+ * validation every other entry point applies - HS_CTRL_KV_LEN (the cache length the attention kernels start from) or
+ * HS_CTRL_SLOT (the index of the committed state snapshot the mixers start from).  Every kernel that turns such a
+ * word into an address checks it first (cache length within [0, kv_capacity - rows], slot within the snapshot ring):
+ * a block that finds it out of range touches neither the cache nor the state, and the status word becomes
+ * HS_ERR_CAPACITY (cache too long) or HS_ERR_DEVICE.  The round's results are then meaningless; hs_reset or
+ * hs_set_context + hs_import_state restore a consistent sequence, hs_clear_status the status word.  The host-side bounds
+ * are not updated.  Synchronises.  HS_ERR_INVALID_ARG for a bad handle, sequence or word. */
+enum { HS_CTRL_KV_LEN = 0, HS_CTRL_SLOT = 1 };
+int hs_poke_control(hs_model *m, int seq, int word, int32_t value);
 const char *hs_last_error(const hs_model *m);
 
 /* Greedy argmax for callers that cannot allocate device memory.  (The paper has no counterpart: this is

@@ -22,7 +22,7 @@ EXPORTS = ["hs_query_sizes", "hs_weight_offset", "hs_init_model", "hs_reset", "h
            "hs_accept_rollback", "hs_round_host", "hs_export_state", "hs_import_state", "hs_set_context",
            "hs_set_batch", "hs_get_context", "hs_get_logits", "hs_get_round", "hs_launch_count",
            "hs_set_attn_geometry", "hs_set_sampling", "hs_set_draft_plan", "hs_set_option", "hs_profile", "hs_profile_read", "hs_device_status", "hs_clear_status",
-           "hs_selftest_wait_timeout", "hs_last_error", "hs_destroy", "hs_argmax_static"]
+           "hs_selftest_wait_timeout", "hs_poke_control", "hs_last_error", "hs_destroy", "hs_argmax_static"]
 
 
 class HsError(RuntimeError):
@@ -83,6 +83,7 @@ def load_library(path: str | None = None):
     L.hs_device_status.argtypes = [vp]
     L.hs_clear_status.argtypes = [vp]
     L.hs_selftest_wait_timeout.argtypes = [vp, ctypes.c_int]
+    L.hs_poke_control.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32]
     L.hs_last_error.restype = ctypes.c_char_p
     L.hs_last_error.argtypes = [vp]
     L.hs_destroy.argtypes = [vp]
@@ -333,7 +334,7 @@ class Engine:
             raise HsError(-1, "draft plan needs one entry per layer")
         self._ck(lib().hs_set_draft_plan(self.h, _ptr(p)))
 
-    OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL, OPT_ATTN_STREAM = range(6)
+    OPT_CLUSTER_REDUCE, OPT_GEMM_MMA, OPT_GEMM_TC, OPT_PDL, OPT_ATTN_SMALL, OPT_ATTN_STREAM, OPT_TC_MIN_ROWS = range(7)
 
     def set_option(self, option, value):
         """Switch a kernel choice (process-wide) on or off; see hs_set_option."""
@@ -360,6 +361,12 @@ class Engine:
 
     def selftest_wait_timeout(self, polls=1000):
         self._ck(lib().hs_selftest_wait_timeout(self.h, int(polls)))
+
+    CTRL_KV_LEN, CTRL_SLOT = 0, 1
+
+    def poke_control(self, seq, word, value):
+        """Overwrite a device control word without validation (self-test of the kernels' range checks)."""
+        self._ck(lib().hs_poke_control(self.h, int(seq), int(word), int(value)))
 
     def check_guards(self):
         """True if the guard bytes behind every buffer the library was given are untouched (synchronises)."""

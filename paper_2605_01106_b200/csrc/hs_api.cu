@@ -130,7 +130,7 @@ Derived derive(const hs_config &c) {
 // layout of the work buffer; base may be null to only measure
 struct WorkLayout {
     int64_t kv_len, slot, cand, g, margin, n_acc, emitted, stage_n, stage_next, status, counters, am_counters, dslot;
-    int64_t rope, h, zx, gbuf, obuf, abuf, logits, dlogits, att_acc, att_ml, am_part, xb, total;
+    int64_t rope, h, zx, gbuf, obuf, abuf, logits, dlogits, att_acc, att_ml, am_part, xb, xb_h, xb_a, ssbuf, total;
 };
 
 WorkLayout work_layout(const hs_config &c, const Derived &v) {
@@ -155,7 +155,13 @@ WorkLayout work_layout(const hs_config &c, const Derived &v) {
     w.am_part = take((int64_t)16 * v.R * HS_ARGMAX_CHUNKS);
     {   // packed bf16 activation operand of the many-row projection kernel: [2][rows][widest reduction]
         const int64_t kmax = std::max<int64_t>(std::max<int64_t>(c.d, c.ff), (int64_t)v.gw + c.qh * c.hd);
-        w.xb = take(v.R > 16 ? (int64_t)2 * 2 * gemm_tc_rows(v.R) * kmax : 0);
+        const int64_t pr = gemm_tc_rows(v.R);
+        w.xb = take((int64_t)2 * 2 * pr * kmax);
+        // the same for the residual stream and the MLP activations, written by the producing projection's epilogue,
+        // and the partial sums of squares (one per 128 model dimensions) of the residual stream's rows
+        w.xb_h = take((int64_t)2 * 2 * pr * c.d);
+        w.xb_a = take((int64_t)2 * 2 * pr * c.ff);
+        w.ssbuf = take((int64_t)4 * pr * ((c.d + 127) / 128));
     }
     w.total = off;
     return w;
@@ -261,6 +267,12 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
     int cur = 0, hparts = 1;
     const int64_t hps = (int64_t)m->B * m->Tm * d;
     int32_t *st_w = m->ctrl.status;
+    // many rows: every projection of the pass runs on the tcgen05 kernel, and the projections hand each other their
+    // results in the packed form that kernel consumes (only the mixer's output and the embedding are packed by a
+    // kernel of their own)
+    const bool tc_pass = gemv_uses_tc(rows, m->xb != nullptr);
+    const int ss_parts = (d + 127) / 128;
+    bool h_packed = false;                  // xb_h / ssbuf hold the current residual stream
     PROF(HS_PROF_EMBED, 0, launch_embed(m->embed, d, c.V, m->ctrl.cand, m->Tm, draft ? step : 0, T, b0, nb, m->hbuf[0], st_w, first, s), "embed");
     ++m->launches;
     for (int l = 0; l < c.L; ++l) {
@@ -279,6 +291,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         ga.pf_ptr = ly.type == HS_LAYER_ATT ? ly.W_o : ly.W_out;
         ga.pf_bytes = 2 * (int64_t)d * (ly.type == HS_LAYER_ATT ? c.qh * c.hd : m->gw);
         ga.xb = m->xb; ga.xb_rows = m->xb_rows;
+        if (tc_pass && h_packed) { ga.pk_in = m->xb_h; ga.ss_in = m->ssbuf; ga.ss_parts = ss_parts; }
         PROF(HS_PROF_GEMV, gemv_bytes(ga), launch_gemv(ga, st_w, s, &m->launches, nullptr), "in_proj");
         // (2) recurrent mixer
         SsmArgs ssm_args{};
@@ -326,6 +339,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 sa.state_out = st_out; sa.out_seq_stride = out_seq; sa.out_slot_stride = out_slot;
                 sa.slot = slot_arr; sa.in_add = in_add; sa.out_rel = out_rel; sa.out_add = out_add; sa.slot_mod = slot_mod; sa.g = m->gbuf; sa.T = T; sa.Tm = m->Tm; sa.b0 = b0; sa.nb = nb;
                 sa.log = log_l; sa.log_w = m->log_w;
+                sa.nslot = slot_mod ? slot_mod : (int)ns; sa.status = st_w;
                 if (with_attn) { ssm_args = sa; ssm_deferred = true; }      // goes out together with the attention
                 else PROF(HS_PROF_MIXER, 0, launch_ssm(sa, s), "ssm");
             } else {
@@ -337,6 +351,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 gd.state_out = st_out; gd.out_seq_stride = out_seq; gd.out_slot_stride = out_slot;
                 gd.slot = slot_arr; gd.in_add = in_add; gd.out_rel = out_rel; gd.out_add = out_add; gd.slot_mod = slot_mod; gd.g = m->gbuf; gd.T = T; gd.Tm = m->Tm; gd.b0 = b0; gd.nb = nb;
                 gd.log = log_l; gd.log_w = m->log_w;
+                gd.nslot = slot_mod ? slot_mod : (int)ns; gd.status = st_w;
                 PROF(HS_PROF_MIXER, 0, launch_gdn(gd, s), "gdn");
             }
             if (!ssm_deferred) ++m->launches;
@@ -381,6 +396,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         }
         go.early_trigger = 1; go.pf_ptr = ly.W_gu; go.pf_bytes = 2 * (int64_t)2 * c.ff * d;
         go.xb = m->xb; go.xb_rows = m->xb_rows;
+        if (tc_pass) { go.pk_out = m->xb_h; go.pk_ld = d; go.pk_nw = ly.norm2; go.ss_out = m->ssbuf; }
         PROF(HS_PROF_GEMV, gemv_bytes(go), launch_gemv(go, st_w, s, &m->launches, &hparts), "out_proj");
         cur ^= 1;
         // (5) RMSNorm + gate/up + SwiGLU, (6) down + residual
@@ -390,6 +406,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
         gu.O = 2 * c.ff; gu.out = m->abuf; gu.ldo = c.ff; gu.nrows = rows; gu.epi = EPI_SWIGLU;
         gu.early_trigger = 1; gu.pf_ptr = ly.W_down; gu.pf_bytes = 2 * (int64_t)d * c.ff;
         gu.xb = m->xb; gu.xb_rows = m->xb_rows;
+        if (tc_pass) { gu.pk_in = m->xb_h; gu.ss_in = m->ssbuf; gu.ss_parts = ss_parts; gu.pk_out = m->xb_a; gu.pk_ld = c.ff; }
         PROF(HS_PROF_GEMV, gemv_bytes(gu), launch_gemv(gu, st_w, s, &m->launches, nullptr), "gate_up");
         GemvArgs gdn{};
         gdn.W0 = ly.W_down; gdn.ldw0 = c.ff; gdn.K0 = c.ff; gdn.x0 = m->abuf; gdn.ldx0 = c.ff; gdn.xparts = 1;
@@ -404,10 +421,14 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
                 gdn.pf_ptr = m->layers[nl].W_in; gdn.pf_bytes = 2 * (int64_t)d * (na ? m->layers[nl].in_rows_full : m->layers[nl].in_rows_draft);
             }
             else { gdn.pf_ptr = m->lm_head; gdn.pf_bytes = 2 * (int64_t)c.V * d; }
+            // the consumer of this layer's output: the next layer that runs (its first norm), else the final norm
+            if (tc_pass) { gdn.pk_out = m->xb_h; gdn.pk_ld = d; gdn.pk_nw = nl < c.L ? m->layers[nl].norm1 : m->final_norm; gdn.ss_out = m->ssbuf; }
         }
         gdn.xb = m->xb; gdn.xb_rows = m->xb_rows;
+        if (tc_pass) gdn.pk_in = m->xb_a;
         PROF(HS_PROF_GEMV, gemv_bytes(gdn), launch_gemv(gdn, st_w, s, &m->launches, &hparts), "down");
         cur ^= 1;
+        h_packed = tc_pass;
     }
     if (!head) { m->last_rows = 0; return HS_OK; }       // the draft model only had to consume these positions
     // final norm + LM head, then greedy argmax
@@ -422,6 +443,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
     else { lm.out = m->logits; lm.ldo = c.V; }
     lm.early_trigger = 1;
     lm.xb = m->xb; lm.xb_rows = m->xb_rows;
+    if (tc_pass && h_packed) { lm.pk_in = m->xb_h; lm.ss_in = m->ssbuf; lm.ss_parts = ss_parts; }
     PROF(HS_PROF_GEMV, gemv_bytes(lm), launch_gemv(lm, st_w, s, &m->launches, nullptr), "lm_head");
     if (sampled) PROF(HS_PROF_ARGMAX, 0, launch_sample(m->dlogits + (size_t)step * c.V, dstride, c.V, m->Tm, b0, nb, m->tau, m->u_draft, c.max_k, step,
                                                        m->ctrl.cand, step + 1, s), "draft draw");
@@ -454,7 +476,7 @@ int enqueue_accept(hs_model *m, int k, int b0, int nb, const int32_t *fn, const 
         ReplayArgs r{};
         r.arch = m->c.arch; r.H = m->c.H; r.P = m->c.P; r.N = m->c.N; r.di = m->di; r.gh = m->c.gh; r.dk = m->c.gdk; r.dv = m->c.gdv;
         r.state = m->snap; r.log = m->ulog; r.log_w = m->log_w; r.n_acc = m->ctrl.n_acc; r.state_elems = m->state_elems;
-        r.n_rl = m->n_rl; r.B = m->B; r.Tm = m->Tm; r.b0 = b0; r.nb = nb;
+        r.n_rl = m->n_rl; r.B = m->B; r.Tm = m->Tm; r.b0 = b0; r.nb = nb; r.status = m->ctrl.status;
         PROF(HS_PROF_ACCEPT, 0, launch_replay(r, m->stream), "replay");
         ++m->launches;
     }
@@ -577,7 +599,12 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->hbuf[0] = (float *)(w + wl.h); m->hbuf[1] = m->hbuf[0] + (size_t)HS_H_PARTS * v.R * c.d; m->zx = (float *)(w + wl.zx); m->gbuf = (float *)(w + wl.gbuf);
     m->obuf = (float *)(w + wl.obuf); m->abuf = (float *)(w + wl.abuf); m->logits = (float *)(w + wl.logits); m->dlogits = (float *)(w + wl.dlogits);
     m->tau = 0.f; m->u_draft = m->u_accept = m->u_final = nullptr;
-    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part; m->xb = v.R > 16 ? (__nv_bfloat16 *)(w + wl.xb) : nullptr; m->xb_rows = gemm_tc_rows(v.R);
+    m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part; m->xb = (__nv_bfloat16 *)(w + wl.xb); m->xb_rows = gemm_tc_rows(v.R);
+    m->xb_h = (__nv_bfloat16 *)(w + wl.xb_h); m->xb_a = (__nv_bfloat16 *)(w + wl.xb_a); m->ssbuf = (float *)(w + wl.ssbuf);
+    // the tcgen05 kernel's fixed cost (operand packing, tensor-memory set-up, epilogue out of tensor memory) pays from
+    // 7 activation rows on, from 5 where the weight matrices are large (measured: model widths 1024 and 2560)
+    m->tc_min_rows_auto = (int64_t)4 * c.ff * c.d >= ((int64_t)64 << 20) ? 5 : 7;
+    g_hs_tc_min_rows = m->tc_min_rows_auto;
     // conv buffer: committed windows | verify history | draft ping-pong
     float *cv = (float *)bufs->conv;
     const size_t win = (size_t)v.n_rl * v.B * 3 * v.convd;
@@ -848,6 +875,14 @@ int hs_set_context(hs_model *m, int seq, int kv_len, int pending) {
     return HS_OK;
 }
 
+int hs_poke_control(hs_model *m, int seq, int word, int32_t value) {
+    if (!m || seq < 0 || seq >= m->B || (word != HS_CTRL_KV_LEN && word != HS_CTRL_SLOT)) return HS_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(m->stream), "hook sync");
+    int32_t *dst = (word == HS_CTRL_KV_LEN ? m->ctrl.kv_len : m->ctrl.slot) + seq;
+    CK(cudaMemcpy(dst, &value, 4, cudaMemcpyHostToDevice), "poke control word");
+    return HS_OK;
+}
+
 int hs_get_context(hs_model *m, int seq, int32_t *kv_len, int32_t *pending) {
     if (!m || seq < 0 || seq >= m->B) return HS_ERR_INVALID_ARG;
     CK(cudaStreamSynchronize(m->stream), "hook sync");
@@ -927,6 +962,14 @@ int hs_set_sampling(hs_model *m, float temperature, const float *u_draft_dev, co
 
 int hs_set_option(hs_model *m, int option, int value) {
     if (!m) return HS_ERR_INVALID_ARG;
+    if (option == HS_OPT_TC_MIN_ROWS) {
+        if (value != 0 && (value < 2 || value > 17)) return fail(m, HS_ERR_INVALID_ARG, "tcgen05 row threshold out of range");
+        CK(cudaStreamSynchronize(m->stream), "option sync");
+        g_hs_tc_min_rows = value ? value : m->tc_min_rows_auto;
+        for (auto &kv : m->graphs) cudaGraphExecDestroy(kv.second);
+        m->graphs.clear(); m->graph_launches.clear();
+        return HS_OK;
+    }
     bool *flag = option == HS_OPT_CLUSTER_REDUCE ? &g_hs_cluster_reduce : option == HS_OPT_GEMM_MMA ? &g_hs_gemm_mma
                : option == HS_OPT_GEMM_TC ? &g_hs_gemm_tc : option == HS_OPT_PDL ? &g_hs_pdl
                : option == HS_OPT_ATTN_SMALL ? &g_hs_attn_small : option == HS_OPT_ATTN_STREAM ? &g_hs_attn_stream : nullptr;

@@ -74,6 +74,8 @@ struct hs_model {
     const float *u_draft, *u_accept, *u_final;   // DEVICE uniforms of the round: [B][max_k], [B][max_k], [B]
     float *att_acc, *att_ml;
     __nv_bfloat16 *xb; int64_t xb_rows;   // packed activation operand of the many-row projection kernel
+    int tc_min_rows_auto;                 // the automatic row threshold of the tcgen05 kernel for this model
+    __nv_bfloat16 *xb_h, *xb_a; float *ssbuf;   // packed residual stream / MLP activations handed from projection to projection, row statistics
     void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
     // conv buffers
     float *cw, *hist, *dcw;
@@ -148,12 +150,23 @@ struct GemvArgs {
     __nv_bfloat16 *xb; int64_t xb_rows;     // scratch for the packed activation operand of the many-row kernel: [2][xb_rows][K0+K1]
     int early_trigger;        // 1: let the next kernel start before this one has waited for its predecessor
                               // (what a prologue may read before its own wait is stated in hs_device.cuh)
+    // Many-row kernel only: projections hand the packed operand to each other, so that no packing kernel sits on the
+    // dependent chain.  pk_in: the activations of this projection, already packed by the projection that produced them
+    // ([2][rows per plane][K0], norm weight folded in, WITHOUT 1/rms when ss_in is given: ss_in[p * rows per plane + r],
+    // p < ss_parts, are partial sums of squares of row r).  pk_out: where to leave this projection's result in packed
+    // form for its consumer (row length pk_ld, times pk_nw[output] if given), with the partial sums of squares of the
+    // residual epilogue's results in ss_out[128-row tile][rows per plane].
+    const __nv_bfloat16 *pk_in; const float *ss_in; int ss_parts;
+    __nv_bfloat16 *pk_out; int pk_ld; const float *pk_nw; float *ss_out;
 };
+// does a projection of nrows activation rows run on the many-row kernel?
+bool gemv_uses_tc(int nrows, bool have_xb);
 // *oparts receives the number of parts written to `out` (1 unless EPI_RESID split the reduction).
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
 cudaError_t configure_gemv();   // one-time kernel attributes; call outside stream capture
 // many activation rows (> 16): tcgen05 tensor-core contraction (kernels_gemm_tc.cu)
 extern bool g_hs_gemm_tc;
+extern int g_hs_tc_min_rows;      // projections with at least this many activation rows run on the tcgen05 kernel
 cudaError_t configure_gemm_tc();
 int gemm_tc_rows(int nrows);
 cudaError_t launch_gemm_tc(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts);
@@ -182,6 +195,8 @@ struct SsmArgs {
     int T, Tm, b0, nb;
     float *log; int log_w;              // verify with rollback by replay: [B][Tm][log_w] update log (decay[H] | dt*x[di] | B[N]);
                                         // no state is stored.  NULL otherwise
+    int nslot; int32_t *status;         // slot[b] must lie in [0, nslot): otherwise the block touches no state and
+                                        // reports HS_ERR_DEVICE through the status word
 };
 cudaError_t launch_ssm(const SsmArgs &a, cudaStream_t s);
 
@@ -197,6 +212,7 @@ struct GdnArgs {
     float *g;                           // [rows][gh*dv]
     int T, Tm, b0, nb;
     float *log; int log_w;              // rollback by replay: [B][Tm][log_w] (alpha[gh] | beta[gh] | k[gh*dk] | v[gh*dv]); NULL otherwise
+    int nslot; int32_t *status;         // as in SsmArgs
 };
 cudaError_t launch_gdn(const GdnArgs &a, cudaStream_t s);
 
@@ -207,9 +223,10 @@ struct ReplayArgs {
     int gh, dk, dv;                     // DeltaNet
     float *state;                       // [n_rl][B][state]
     const float *log; int log_w;        // [n_rl][B][Tm][log_w]
-    const int32_t *n_acc;               // [B]
+    const int32_t *n_acc;               // [B]; must lie in [0, Tm): otherwise nothing is applied and the status word reports it
     int64_t state_elems;
     int n_rl, B, Tm, b0, nb;
+    int32_t *status;
 };
 cudaError_t launch_replay(const ReplayArgs &a, cudaStream_t s);
 

@@ -139,8 +139,8 @@ __device__ __forceinline__ void attn_body(const AttnArgs &a, const int split, co
     const bool last = split == nsplit - 1;
     const int c0 = split * SPAN, rc = max(0, min(len, c0 + SPAN) - c0);
     const int ntile = last ? max(1, (rc + CK - 1) / CK) : (rc + CK - 1) / CK;
-    if (len + T > a.cap) {                        // never write past the cache; the host reports the status word
-        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
+    if (len < 0 || len + T > a.cap) {             // never read or write outside the cache; the host reports the status word
+        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, len < 0 ? (int)HS_ERR_DEVICE : (int)HS_ERR_CAPACITY);
         return;
     }
     __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
@@ -566,8 +566,8 @@ __device__ __forceinline__ void attn_small_body(const AttnArgs &a, const int spl
     // ---- before the wait: kv_len, the whole key range of this CTA, the RoPE rows
     const int len = __ldcg(a.kv_len + b) + a.len_off;
     const int nsplit = max(1, (len + CK - 1) / CK);
-    if (len + T > a.cap || nsplit > AT_CL) {      // never write past the cache; a cache longer than the host's bound is a host error
-        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, len + T > a.cap ? (int)HS_ERR_CAPACITY : (int)HS_ERR_DEVICE);
+    if (len < 0 || len + T > a.cap || nsplit > AT_CL) {      // never write past the cache; a cache longer than the host's bound is a host error
+        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (len >= 0 && len + T > a.cap) ? (int)HS_ERR_CAPACITY : (int)HS_ERR_DEVICE);
         return;
     }
     const int crank = split;                      // the grid has exactly one cluster along x
@@ -885,8 +885,8 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     const int SPAN = CK * a.tiles;
     const int nsplit = max(1, (len + SPAN - 1) / SPAN);
     if (split >= nsplit) return;                   // beyond the cache
-    if (len + T > a.cap) {
-        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, (int)HS_ERR_CAPACITY);
+    if (len < 0 || len + T > a.cap) {
+        if (tid == 0 && split == 0 && kh == 0) atomicCAS(a.status, 0, len < 0 ? (int)HS_ERR_DEVICE : (int)HS_ERR_CAPACITY);
         return;
     }
     const bool last = split == nsplit - 1;

@@ -652,6 +652,8 @@ cudaError_t configure_gemv() {
 
 // Launches the projection.  a.max_oparts > 1 allows a K split for the residual epilogue; the number
 // of parts written is returned in *oparts (1 for the other epilogues).
+bool gemv_uses_tc(int nrows, bool have_xb) { return (nrows > GV_MAXROWS || nrows >= g_hs_tc_min_rows) && g_hs_gemm_tc && have_xb; }
+
 cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int64_t *launches, int *oparts) {
     // One to three activation rows: the CUDA-core kernel.  4..16 rows: the tensor-core kernel.  More rows go in several
     // launches (the weights are streamed again for each).  g_hs_gemm_mma = false sends everything through the
@@ -671,7 +673,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int32_t *status, cudaStream_t s, int6
         return cudaSuccess;
     };
     const bool mma = g_hs_gemm_mma && a.nrows >= 4;       // measured: up to three rows the pruned FMA instances are faster
-    if (a.nrows > GV_MAXROWS && g_hs_gemm_tc && a.xb) return launch_gemm_tc(a, status, s, launches, oparts);   // a dense contraction: tcgen05
+    if (gemv_uses_tc(a.nrows, a.xb != nullptr)) return launch_gemm_tc(a, status, s, launches, oparts);   // a dense contraction: tcgen05
     if (a.nrows > GV_MAXROWS) return rows_launch(GV_MAXROWS);
     if (!mma && a.nrows > 4) {
         const int K = a.K0 > a.K1 ? a.K0 : a.K1;

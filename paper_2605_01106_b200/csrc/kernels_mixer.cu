@@ -37,6 +37,10 @@ __global__ void __launch_bounds__(GDN_THREADS) gdn_kernel(const GdnArgs a) {
     const int nk = a.gh * DK, nv = a.gh * dv;
 
     const int cslot = (a.in_slot_stride || a.out_rel) ? __ldcg(a.slot + b) : 0;
+    if ((unsigned)cslot >= (unsigned)a.nslot) {     // a control word out of range is never turned into an address
+        if (threadIdx.x == 0) atomicCAS(a.status, 0, (int)HS_ERR_DEVICE);
+        return;
+    }
     const int islot = a.slot_mod ? (cslot + a.in_add) % a.slot_mod : cslot;
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride + (a.in_slot_stride ? (size_t)islot * a.in_slot_stride : 0) + (size_t)h * dv * DK;
     float s[RPW][2];
@@ -180,6 +184,10 @@ __global__ void __launch_bounds__(SSM_THREADS) replay_ssm_kernel(const ReplayArg
     const float *lg = a.log + ((size_t)rl * a.B + b) * a.Tm * a.log_w;
     pdl_wait();
     const int n = __ldcg(a.n_acc + b);
+    if ((unsigned)n >= (unsigned)a.Tm) {            // the log holds Tm entries
+        if (threadIdx.x == 0) atomicCAS(a.status, 0, (int)HS_ERR_DEVICE);
+        return;
+    }
     float s[RPW][EPL];
 #pragma unroll
     for (int r = 0; r < RPW; ++r)
@@ -226,6 +234,10 @@ __global__ void __launch_bounds__(GDN_THREADS) replay_gdn_kernel(const ReplayArg
     const bool rows_ok = warp * RPW < dv;
     pdl_wait();
     const int n = __ldcg(a.n_acc + b);
+    if ((unsigned)n >= (unsigned)a.Tm) {            // the log holds Tm entries
+        if (threadIdx.x == 0) atomicCAS(a.status, 0, (int)HS_ERR_DEVICE);
+        return;
+    }
     float s[RPW][2];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {

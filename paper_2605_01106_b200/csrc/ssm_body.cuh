@@ -33,6 +33,10 @@ __device__ __forceinline__ void ssm_body(const SsmArgs &a, const int bx, const i
     //      the step or of the previous round) is merely pulled towards L2 and loaded after the wait, together
     //      with the in-projection's outputs, so that this kernel may start as early as its predecessor allows
     const int cslot = (a.in_slot_stride || a.out_rel) ? __ldcg(a.slot + b) : 0;
+    if ((unsigned)cslot >= (unsigned)a.nslot) {     // a control word out of range is never turned into an address
+        if (threadIdx.x == 0) atomicCAS(a.status, 0, (int)HS_ERR_DEVICE);
+        return;
+    }
     const int islot = a.slot_mod ? (cslot + a.in_add) % a.slot_mod : cslot;
     const float *sin_ = a.state_in + (size_t)b * a.in_seq_stride + (a.in_slot_stride ? (size_t)islot * a.in_slot_stride : 0) +
                         ((size_t)h * a.P + p0 + warp * RPW) * N;

@@ -88,6 +88,28 @@ def test_cfg2_attention_geometries(env):
     assert rep.rounds == 9
 
 
+def test_cfg2_projection_kernel_choices(env):
+    # which kernel a projection runs on is a matter of its activation-row count (CUDA cores up to 3 rows, the
+    # warp-level tensor path, tcgen05 from a threshold on): every choice must reproduce the oracle.  Threshold 17 keeps
+    # 6 and 10 rows on the warp-level path (one and two groups of eight rows), 2 sends even the two-row draft steps
+    # through tcgen05 (16- and 32-row tiles, K split over clusters), 0 restores the automatic threshold.
+    s, eng, model, seqs = make(env, "cfg2_0p5b", 2, 8, 700, {0, 1}, [512, 77])
+    with pytest.raises(RuntimeError):
+        eng.set_option(eng.OPT_TC_MIN_ROWS, 18)
+    rep = None
+    try:
+        for thr, ks in ((17, (2, 4)), (2, (0, 2, 8)), (0, (1, 4))):
+            eng.set_option(eng.OPT_TC_MIN_ROWS, thr)
+            for k in ks:
+                forced = [hi.forced_accept(k, 1, seq=thr + k + b) for b in range(2)]
+                rep = env["harness"].run_rounds(eng, seqs, s, k, 1, forced=forced, rep=rep)
+                assert eng.device_status() == 0, (thr, k)
+    finally:
+        eng.set_option(eng.OPT_TC_MIN_ROWS, 0)          # the choice is process-wide
+    print(rep)
+    assert rep.rounds == 7
+
+
 def test_streaming_attention_edge_cases(env):
     # the streaming form (128-key tiles walked with two buffers, warp-local running softmax, ranges merged by the last
     # CTA to arrive) on the small sequential stack, where attention is a launch of its own: contexts that end exactly on

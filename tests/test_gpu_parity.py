@@ -312,3 +312,40 @@ def test_bounded_wait_runs_out_and_reports(env):
     assert eng.device_status() == 0
     env["harness"].run_rounds(eng, seqs, s, 2, 2)
     assert eng.device_status() == 0
+
+
+@pytest.mark.parametrize("name", ["cfg1_tiny", "test_seq"])
+def test_control_words_out_of_range_are_not_used_as_addresses(env, name):
+    # The kernels that turn a device control word into an address check it first.  A self-test hook plants a bad word
+    # for one of two sequences (no host-side validation; the sequence is chosen so that even an unchecked access would
+    # stay inside the buffer): the blocks of that sequence must touch neither cache nor state,
+    # the status word must name the error, the guard bytes behind every buffer must be intact, and after a reset the
+    # handle must reproduce the oracle again.
+    k, cap = 4, 64
+    lens = [24, 17]
+    s, eng, model, seqs = setup(env, name, lens, max_k=k, cap=cap)
+    for seq, word, value, want in ((0, eng.CTRL_KV_LEN, cap - 2, -3),   # the k + 1 new rows would not fit: HS_ERR_CAPACITY
+                                   (1, eng.CTRL_KV_LEN, -5, -7),        # a negative cache length: HS_ERR_DEVICE
+                                   (0, eng.CTRL_SLOT, k + 3, -7)):      # a snapshot slot beyond the k + 1 that exist
+        eng.poke_control(seq, word, value)
+        eng.draft(k)
+        eng.verify(k)
+        assert eng.device_status() == want, (word, value)
+        assert eng.check_guards()
+        eng.accept_rollback()
+        eng.reset()
+        assert eng.device_status() == 0
+        prompts = [hi.make_prompt(s.V, n, seq=b) for b, n in enumerate(lens)]
+        seqs = []
+        for p in prompts:
+            q = model.new_seq()
+            q.prefill(p)
+            seqs.append(q)
+        eng.prefill(prompts)
+        env["harness"].run_rounds(eng, seqs, s, k, 2)
+        assert eng.device_status() == 0
+    with pytest.raises(RuntimeError):
+        eng.poke_control(0, 7, 0)
+    with pytest.raises(RuntimeError):
+        eng.poke_control(2, eng.CTRL_SLOT, 0)
+
