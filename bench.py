@@ -418,8 +418,10 @@ def run_ours(args):
     if world == 1 and args.by_config and args.config == "cfg2_0p5b":
         # (workload, batch, draft lengths, extra flags): the batched workloads also with rollback by replay
         # (HS_FLAG_REPLAY: an update log instead of k + 1 state snapshots per verify pass)
-        plan = [("cfg3_3b", 1, (2, 4), 0), ("cfg3_3b", 8, (4,), 0), ("cfg3_3b", 8, (4,), hs.HS_FLAG_REPLAY),
-                ("cfg4_seq", 1, (2, 4), 0), ("cfg5_b64", 64, (4,), 0), ("cfg5_b64", 64, (4,), hs.HS_FLAG_REPLAY)]
+        # k = 0 is plain autoregressive decoding with the full model: the denominator of Eq. 1 on that workload
+        plan = [("cfg3_3b", 1, (0, 2, 4), 0), ("cfg3_3b", 8, (0, 4), 0), ("cfg3_3b", 8, (4,), hs.HS_FLAG_REPLAY),
+                ("cfg4_seq", 1, (0, 2, 4), 0), ("cfg5_b64", 64, (0, 4), 0), ("cfg5_b64", 64, (4,), hs.HS_FLAG_REPLAY)]
+        ar_rate = {}
         blobs = {"cfg2_0p5b": blob}
         for name, nb, kset, xflags in plan:
             sc = hi.CONFIGS[name]
@@ -448,6 +450,10 @@ def run_ours(args):
                 # recurrent-state bytes one round really moves in its verify + rollback: snapshots: read 1, write k + 1;
                 # replay: read 1 in verify, read 1 + write 1 in the replay kernel (the algorithmic figure counts 2)
                 rep["state_traffic_bytes_per_round"] = unit * (3 if xflags & hs.HS_FLAG_REPLAY else kk + 2)
+                if kk == 0:
+                    ar_rate[(name, nb)] = rep["tokens_per_s"]
+                if (name, nb) in ar_rate:
+                    rep["speedup_vs_autoregressive"] = rep["tokens_per_s"] / ar_rate[(name, nb)]
                 entry["k%d" % kk] = rep
             by_config["%s@b%d%s" % (name, nb, "+replay" if xflags & hs.HS_FLAG_REPLAY else "")] = entry
             e.close()
