@@ -857,10 +857,16 @@ __host__ __device__ inline Attn2Layout attn2_layout(int hd, int mt) {
 }
 __device__ __forceinline__ void cp_async_wait_but_two() { asm volatile("cp.async.wait_group 2;" ::: "memory"); }
 
-template <int HD, int MT>
+// PK: the last 16-row query tile is "packed" - it holds at most 8 query rows, their bf16 heads in its rows 0-7 and
+// their bf16 remainders in rows 8-15.  One MMA then yields both partial products of a row in the SAME thread (the
+// accumulator registers of rows g and g + 8), for the scores and again for P V (probability heads feed rows 0-7 of the
+// operand, remainders rows 8-15), so that tile costs half the tensor instructions of a full one.  It serves 1..8 query
+// rows (MT = 1) and 17..24 (MT = 2: 20 rows at four query heads per KV head and k = 4).
+template <int HD, int MT, bool PK>
 __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
     constexpr int CK = A2_CK, GTB = MT * 16, NT = HD / 8, RB = HD * 2;       // RB: bytes of a tile row
+    constexpr int PB = (MT - 1) * 16;                                        // first row of the packed tile
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int G = a.qh / a.kvh, T = a.T, GT = G * T;
     const Attn2Layout L = attn2_layout(HD, MT);
@@ -954,10 +960,12 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                 if (qi < GT) {
                     const float2 cs = rope_s[(qi - (int)((qi * tinv) >> 16) * T) * HP + e];
                     __nv_bfloat16 h, l;
+                    // the remainder of a row of the packed tile lives eight rows further down the same array
+                    __nv_bfloat16 *lo_row = (PK && qi >= PB) ? Qh_s + (size_t)(qi + 8) * KSTR : Ql_s + (size_t)qi * KSTR;
                     split_bf16((x0[u] * cs.x - x1[u] * cs.y) * scale, h, l);
-                    Qh_s[qi * KSTR + e] = h; Ql_s[qi * KSTR + e] = l;
+                    Qh_s[qi * KSTR + e] = h; lo_row[e] = l;
                     split_bf16((x1[u] * cs.x + x0[u] * cs.y) * scale, h, l);
-                    Qh_s[qi * KSTR + e + HP] = h; Ql_s[qi * KSTR + e + HP] = l;
+                    Qh_s[qi * KSTR + e + HP] = h; lo_row[e + HP] = l;
                 }
             }
         }
@@ -1044,9 +1052,11 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                         uint32_t ah[4], al[4];
                         const size_t qo = (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KSTR + ks * 16 + (lane >> 4) * 8;
                         ldsm_x4(ah, Qh_s + qo);
-                        ldsm_x4(al, Ql_s + qo);
                         mma_bf16(Sp[0][mt][0], ah, bk[0], bk[1]); mma_bf16(Sp[0][mt][1], ah, bk[2], bk[3]);
-                        mma_bf16(Sp[1][mt][0], al, bk[0], bk[1]); mma_bf16(Sp[1][mt][1], al, bk[2], bk[3]);
+                        if (!(PK && mt == MT - 1)) {
+                            ldsm_x4(al, Ql_s + qo);
+                            mma_bf16(Sp[1][mt][0], al, bk[0], bk[1]); mma_bf16(Sp[1][mt][1], al, bk[2], bk[3]);
+                        }
                     }
                 }
 #pragma unroll
@@ -1055,6 +1065,9 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                     for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) S[mt][nt][e] = Sp[0][mt][nt][e] + Sp[1][mt][nt][e];
+                if (PK)                      // packed tile: head product in the registers of row g, remainder product in those of row g + 8
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) { S[MT - 1][nt][0] += S[MT - 1][nt][2]; S[MT - 1][nt][1] += S[MT - 1][nt][3]; }
             }
             // ---- masks, running softmax, probabilities as operand fragments
             const bool edge = newrows || kb + 16 > nkeys;
@@ -1078,6 +1091,8 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                     for (int e = 0; e < 4; ++e) mx[e >> 1] = fmaxf(mx[e >> 1], S[mt][nt][e]);
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
+                    const bool packed = PK && mt == MT - 1;
+                    if (packed && r == 1) { corr_all[mt][1] = corr_all[mt][0]; continue; }   // rows 8-15 carry remainders, not rows
                     mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
                     mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
                     const float mnew = fmaxf(m_run[mt][r], mx[r]);
@@ -1092,8 +1107,10 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
                         sum += p0 + p1;
                         // two probabilities at a time: bf16 heads packed by one conversion, remainders from the exact differences
                         const uint32_t hh = pack_bf16x2(p0, p1);
+                        const uint32_t ll = pack_bf16x2(p0 - __uint_as_float(hh << 16), p1 - __uint_as_float(hh & 0xffff0000u));
                         ph[mt][r + 2 * nt] = hh;
-                        pl[mt][r + 2 * nt] = pack_bf16x2(p0 - __uint_as_float(hh << 16), p1 - __uint_as_float(hh & 0xffff0000u));
+                        if (packed) ph[mt][1 + 2 * nt] = ll;     // operand rows 8-15 of the packed tile
+                        else pl[mt][r + 2 * nt] = ll;
                     }
                     l_run[mt][r] = fmaf(l_run[mt][r], corr, sum);
                 }
@@ -1122,7 +1139,9 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     mma_bf16(O[mt][2 * p], ph[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], ph[mt], bv[2], bv[3]);
-                    mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
+                    if (!(PK && mt == MT - 1)) {
+                        mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
+                    }
                 }
             }
         }
@@ -1136,6 +1155,11 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
+            const bool packed = PK && mt == MT - 1;
+            if (packed && r == 1) continue;
+            if (packed)                       // head and remainder halves of the packed tile's outputs
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) { O[mt][nt][0] += O[mt][nt][2]; O[mt][nt][1] += O[mt][nt][3]; }
             float l = l_run[mt][r];
             l += __shfl_xor_sync(0xffffffffu, l, 1);
             l += __shfl_xor_sync(0xffffffffu, l, 2);
@@ -1221,17 +1245,17 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     }
 }
 
-template <int HD, int MT>
+template <int HD, int MT, bool PK>
 cudaError_t launch_attn2_t(const AttnArgs &a, cudaStream_t s) {
     static bool configured = false;
     const size_t smem = attn2_layout(HD, MT).total;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn2_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn2_kernel<HD, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        cudaError_t e = cudaFuncSetAttribute(attn2_kernel<HD, MT, PK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn2_kernel<HD, MT, PK>, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_pdl(attn2_kernel<HD, MT>, dim3(a.nch, a.kvh, a.nb), dim3(A2_THREADS), smem, s, a);
+    return launch_pdl(attn2_kernel<HD, MT, PK>, dim3(a.nch, a.kvh, a.nb), dim3(A2_THREADS), smem, s, a);
 }
 
 template <int HD, int MT>
@@ -1333,8 +1357,11 @@ cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s) {
     }
     if (a.stream) {          // the streaming form: 128-key tiles, a.tiles of them per CTA, at most 32 query rows
         if (GT > 32 || a.chunk != A2_CK || a.tiles < 1) return cudaErrorInvalidValue;
-        if (a.hd == 128) return GT <= 16 ? launch_attn2_t<128, 1>(a, s) : launch_attn2_t<128, 2>(a, s);
-        if (a.hd == 64) return GT <= 16 ? launch_attn2_t<64, 1>(a, s) : launch_attn2_t<64, 2>(a, s);
+        // at most 8 rows in the last 16-row tile: the packed form of that tile (half its tensor instructions)
+#define A2(hd_) if (a.hd == hd_) return GT <= 8 ? launch_attn2_t<hd_, 1, true>(a, s) : GT <= 16 ? launch_attn2_t<hd_, 1, false>(a, s) \
+                                      : GT <= 24 ? launch_attn2_t<hd_, 2, true>(a, s) : launch_attn2_t<hd_, 2, false>(a, s)
+        A2(128); A2(64);
+#undef A2
         return cudaErrorInvalidValue;
     }
     if (GT > HS_MAX_GT || a.chunk < 16 || a.chunk > 128 || (a.chunk & 15) || a.tiles < 1) return cudaErrorInvalidValue;
