@@ -216,6 +216,7 @@ struct AttnGeom {
 // (the same for a verify pass; a draft that keeps attention appends one row per step, k in all)
 AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
     if (m->att_force_chunk) return AttnGeom{m->att_force_chunk, m->att_force_tiles < 0 ? -m->att_force_tiles : m->att_force_tiles, 0, m->att_force_tiles < 0 ? 1 : 0};
+    const bool have_maps = !m->kmaps.empty();        // the streaming form fetches its tiles with tensor copies
     int maxlen = 0;
     for (int b = b0; b < b0 + nb; ++b) if (m->kv_upper[b] > maxlen) maxlen = m->kv_upper[b];
     {
@@ -231,7 +232,7 @@ AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
     {
         const bool own_launch = m->c.arch == HS_ARCH_SEQUENTIAL || (int64_t)(m->c.P / 16) * m->c.H * nb > 4 * 148;
         const int64_t ctas128 = (int64_t)nb * m->c.kvh * ((maxlen + T + 127) / 128);
-        if (g_hs_attn_stream && own_launch && (m->c.qh / m->c.kvh) * Tq <= 32 && ctas128 >= 2 * 148) {
+        if (g_hs_attn_stream && have_maps && own_launch && (m->c.qh / m->c.kvh) * Tq <= 32 && ctas128 >= 2 * 148) {
             int tiles = (int)(ctas128 / (4 * 148));
             tiles = tiles < 1 ? 1 : tiles > 16 ? 16 : tiles;
             return AttnGeom{128, tiles, 0, 1};
@@ -368,6 +369,7 @@ int model_pass(hs_model *m, bool draft, int T, int step, int b0, int nb, bool fi
             aa.kv_len = m->ctrl.kv_len; aa.o = m->obuf;
             aa.part_acc = m->att_acc; aa.part_ml = m->att_ml; aa.counters = m->ctrl.counters; aa.status = m->ctrl.status;
             aa.chunk = at_geom.chunk; aa.tiles = at_geom.tiles; aa.small = at_geom.small; aa.stream = at_geom.stream;
+            if (!m->kmaps.empty()) { aa.kmap = m->kmaps[ly.al]; aa.vmap = m->vmaps[ly.al]; }
             aa.len_off = draft ? step : 0;
             aa.nch = (c.kv_capacity + at_geom.chunk * at_geom.tiles - 1) / (at_geom.chunk * at_geom.tiles); aa.T = T; aa.b0 = b0; aa.nb = nb;
             bool fused = false;
@@ -618,6 +620,16 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     CK(configure_gemv(), "configure gemv");
     CK(configure_attn(), "configure attention");
     if (configure_gemm_tc() != cudaSuccess) { g_hs_gemm_tc = false; cudaGetLastError(); }   // falls back to several 16-row launches
+    if (g_hs_tensor_maps && c.hd % 64 == 0) {     // tensor maps of every attention layer's cache (streaming attention form)
+        const size_t per_layer = (size_t)v.B * c.kvh * c.kv_capacity * c.hd;
+        m->kmaps.resize(v.n_al); m->vmaps.resize(v.n_al);
+        for (int al = 0; al < v.n_al; ++al)
+            if (hs_make_kv_tensor_map(&m->kmaps[al], m->Kc + al * per_layer, (uint64_t)v.B * c.kvh * c.kv_capacity, c.hd) != cudaSuccess ||
+                hs_make_kv_tensor_map(&m->vmaps[al], m->Vc + al * per_layer, (uint64_t)v.B * c.kvh * c.kv_capacity, c.hd) != cudaSuccess) {
+                m->kmaps.clear(); m->vmaps.clear(); cudaGetLastError();
+                break;
+            }
+    }
     // RoPE table (rotate-half pairing: pair (e, e + hd/2) turns by pos * theta^(-2e/hd)), computed in double
     std::vector<float2> tab((size_t)c.kv_capacity * (c.hd / 2));
     for (int e = 0; e < c.hd / 2; ++e) {
@@ -920,6 +932,7 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles) {
     if (tiles < 0) {        // the streaming form: 128-key tiles, -tiles of them per CTA
         if (chunk != 128 || tiles < -32 || (m->c.qh / m->c.kvh) * (m->c.max_k + 1) > 32)
             return fail(m, HS_ERR_INVALID_ARG, "streaming attention: chunk 128, 1..32 tiles, at most 32 query rows per KV head");
+        if (m->kmaps.empty()) return fail(m, HS_ERR_INVALID_ARG, "streaming attention needs the driver's tensor-map encoder and a head dimension that is a multiple of 64");
     } else if (chunk < 16 || chunk > 128 || (chunk & 15) || tiles < 1 || tiles > 32 || chunk * tiles < m->att_chunk)
         return fail(m, HS_ERR_INVALID_ARG, "attention geometry: chunk a multiple of 16 up to 128, tiles 1..32, chunk * tiles >= workspace chunk");
     m->att_force_chunk = chunk; m->att_force_tiles = tiles;

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libhs (host orchestration + kernels).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -74,6 +75,7 @@ struct hs_model {
     const float *u_draft, *u_accept, *u_final;   // DEVICE uniforms of the round: [B][max_k], [B][max_k], [B]
     float *att_acc, *att_ml;
     __nv_bfloat16 *xb; int64_t xb_rows;   // packed activation operand of the many-row projection kernel
+    std::vector<CUtensorMap> kmaps, vmaps;   // per attention layer (streaming attention form)
     int tc_min_rows_auto;                 // the automatic row threshold of the tcgen05 kernel for this model
     __nv_bfloat16 *xb_h, *xb_a; float *ssbuf;   // packed residual stream / MLP activations handed from projection to projection, row statistics
     void *am_part;             // argmax partials [B*Tm][HS_ARGMAX_CHUNKS] x 16 bytes
@@ -244,8 +246,13 @@ struct AttnArgs {
     int stream;                         // 1: the streaming form for long caches (stand-alone launches: chunk = 128, at most 32 query rows)
     int small;                          // 1: the latency-lean form (G*T <= 16 rows, every cache within one cluster of 8 CTAs x chunk keys)
     int T, b0, nb;
+    // streaming form: this layer's K and V cache as 2-D tensors [B * kvh * cap rows][hd] for tiled bulk copies
+    // (boxes of 64 columns x 128 rows, 128-byte swizzle); made once per layer by hs_make_kv_tensor_map
+    alignas(64) CUtensorMap kmap, vmap;
 };
 cudaError_t launch_attn(const AttnArgs &a, cudaStream_t s);
+extern bool g_hs_tensor_maps;   // the driver's tensor-map encoder was found (configure_gemm_tc)
+cudaError_t hs_make_kv_tensor_map(CUtensorMap *map, const void *base, uint64_t rows, int hd);
 // mixer + attention of a parallel block in one launch (verify pass); *fused = false: not applicable, nothing launched
 cudaError_t launch_ssm_attn(const SsmArgs &sa, const AttnArgs &a, cudaStream_t s, bool *fused);
 bool ssm_wide(const SsmArgs &a);    // the mixer runs a whole head per block (large batch)

@@ -846,16 +846,19 @@ __host__ __device__ inline Attn2Layout attn2_layout(int hd, int mt) {
     Attn2Layout L;
     L.kstr = hd + 8;                       // padded rows of the query and new-row buffers
     L.tile_bytes = (size_t)A2_CK * hd * 2;
-    size_t o = 128;
+    size_t o = 0;                          // offsets from the first 1024-byte boundary of the dynamic shared memory
     L.tile_off = o; o += 2 * A2_NBUF * L.tile_bytes;               // K0 V0 K1 V1 K2 V2; later the warp partials
     L.q_off = o; o += (size_t)2 * mt * 16 * L.kstr * 2;            // bf16 head | remainder
     L.new_off = o; o += (size_t)2 * 16 * L.kstr * 2;               // the new K | V rows as they are cached: a 16-key group of their own
     L.rope_off = o; o += (size_t)HS_MAX_T * (hd / 2) * 8;
     L.ml_off = o; o += (size_t)(A2_WARPS + 1) * mt * 16 * 2 * 4;   // per warp (max, sum) per row, then the merged pair
-    L.total = (o + 127) / 128 * 128;
+    L.total = (o + 127) / 128 * 128 + 1024;
     return L;
 }
-__device__ __forceinline__ void cp_async_wait_but_two() { asm volatile("cp.async.wait_group 2;" ::: "memory"); }
+__device__ __forceinline__ void tma_tile_2d(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
 
 // PK: the last 16-row query tile is "packed" - it holds at most 8 query rows, their bf16 heads in its rows 0-7 and
 // their bf16 remainders in rows 8-15.  One MMA then yields both partial products of a row in the SAME thread (the
@@ -863,24 +866,26 @@ __device__ __forceinline__ void cp_async_wait_but_two() { asm volatile("cp.async
 // operand, remainders rows 8-15), so that tile costs half the tensor instructions of a full one.  It serves 1..8 query
 // rows (MT = 1) and 17..24 (MT = 2: 20 rows at four query heads per KV head and k = 4).
 template <int HD, int MT, bool PK>
-__global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) {
-    extern __shared__ __align__(128) unsigned char smraw[];
+__global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_constant__ AttnArgs a) {
+    extern __shared__ __align__(1024) unsigned char smraw[];
     constexpr int CK = A2_CK, GTB = MT * 16, NT = HD / 8, RB = HD * 2;       // RB: bytes of a tile row
     constexpr int PB = (MT - 1) * 16;                                        // first row of the packed tile
     const int split = blockIdx.x, kh = blockIdx.y, lb = blockIdx.z, b = a.b0 + lb;
     const int G = a.qh / a.kvh, T = a.T, GT = G * T;
     const Attn2Layout L = attn2_layout(HD, MT);
     const int KSTR = L.kstr;
-    unsigned char *tile_s = smraw + L.tile_off;
+    unsigned char *sm = smraw + ((1024u - (smem_u32(smraw) & 1023u)) & 1023u);      // swizzled tiles need 1024-byte alignment
+    unsigned char *tile_s = sm + L.tile_off;
     auto Kbuf = [&](int i) { return tile_s + (size_t)(2 * i) * L.tile_bytes; };
     auto Vbuf = [&](int i) { return tile_s + (size_t)(2 * i + 1) * L.tile_bytes; };
-    __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.q_off);        // [GTB][KSTR]
+    __nv_bfloat16 *Qh_s = reinterpret_cast<__nv_bfloat16 *>(sm + L.q_off);        // [GTB][KSTR]
     __nv_bfloat16 *Ql_s = Qh_s + (size_t)GTB * KSTR;
-    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(smraw + L.new_off);      // [16][KSTR]
+    __nv_bfloat16 *Kn_s = reinterpret_cast<__nv_bfloat16 *>(sm + L.new_off);      // [16][KSTR]
     __nv_bfloat16 *Vn_s = Kn_s + (size_t)16 * KSTR;
-    float2 *rope_s = reinterpret_cast<float2 *>(smraw + L.rope_off);
-    float *wml_s = reinterpret_cast<float *>(smraw + L.ml_off);                      // [A2_WARPS + 1][GTB][2]
+    float2 *rope_s = reinterpret_cast<float2 *>(sm + L.rope_off);
+    float *wml_s = reinterpret_cast<float *>(sm + L.ml_off);                      // [A2_WARPS + 1][GTB][2]
     __shared__ int ticket_s;
+    __shared__ __align__(8) uint64_t tile_bar[A2_NBUF];                              // one per tile buffer pair: bytes of K and V landed
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t tinv = (65536u + T - 1) / T;
@@ -901,19 +906,28 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
     const int nitem = ntile + (last ? 1 : 0);      // the range that ends the cache also takes the new rows, as one more item
     __nv_bfloat16 *Kb = a.Kc + ((size_t)b * a.kvh + kh) * a.cap * HD;
     __nv_bfloat16 *Vb = a.Vc + ((size_t)b * a.kvh + kh) * a.cap * HD;
-    auto fetch = [&](int t) {              // cached rows of tile t into buffer t % 3: one commit group, possibly empty
-        const int n = t < ntile ? min(CK, rc - t * CK) : 0;
-        unsigned char *kd = Kbuf(t % A2_NBUF), *vd = Vbuf(t % A2_NBUF);
-        const __nv_bfloat16 *ks = Kb + (size_t)(c0 + t * CK) * HD, *vs = Vb + (size_t)(c0 + t * CK) * HD;
-#pragma unroll 4
-        for (int idx = tid; idx < n * (HD / 8); idx += A2_THREADS) {
-            const int j = idx / (HD / 8), c = idx - j * (HD / 8);
-            const int so = j * RB + ((c ^ (j & 7)) << 4);
-            cp_async16(kd + so, ks + (size_t)j * HD + 8 * c);
-            cp_async16(vd + so, vs + (size_t)j * HD + 8 * c);
+    // Cached rows of tile t into buffer pair t % 3: tensor copies of 64 columns x 128 rows (the two halves of a 128-wide
+    // head dimension land 16 KB apart), issued by one thread, completion counted in bytes on the pair's barrier.  A tile
+    // is fetched whole: rows beyond the cache length hold earlier contents or belong to the next head - they are masked
+    // (K) or cleared (V) below; rows beyond the tensor read as zero.
+    constexpr int HALVES = HD / 64, HS_ = CK * 128;      // HS_: bytes between the halves of a tile
+    const int row00 = (b * a.kvh + kh) * a.cap + c0;
+    auto fetch = [&](int t) {
+        if (tid != 0 || t >= ntile) return;
+        uint64_t *bar = &tile_bar[t % A2_NBUF];
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the buffer was last touched by ordinary loads / stores
+        mbar_expect_tx(bar, 2u * CK * RB);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) {
+            tma_tile_2d(Kbuf(t % A2_NBUF) + hf * HS_, &a.kmap, hf * 64, row00 + t * CK, bar);
+            tma_tile_2d(Vbuf(t % A2_NBUF) + hf * HS_, &a.vmap, hf * 64, row00 + t * CK, bar);
         }
-        cp_async_commit();
     };
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < A2_NBUF; ++i) mbar_init(&tile_bar[i], 1);
+        mbar_fence_init();
+    }
     fetch(0);
     fetch(1);
 #pragma unroll 1
@@ -1014,19 +1028,23 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
         const int nkeys = newrows ? T : min(CK, rc - t * CK);
         const int nkp = (nkeys + 15) & ~15;
         if (!newrows) {
-            cp_async_wait_but_one();        // this thread's copies of tile t have landed (tile t + 1 may be in flight)
+            // tile t has landed (tile t + 1 may be in flight); a wait that runs out is reported, the pass goes on
+            if (!mbar_wait(&tile_bar[t % A2_NBUF], (uint32_t)(t / A2_NBUF) & 1u) && tid == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
             if (nkp != nkeys) {             // a ragged tile (only the last can be): finite V rows for its padding keys
                 unsigned char *vd = Vbuf(t % A2_NBUF);
 #pragma unroll 1
-                for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS)
-                    *reinterpret_cast<uint4 *>(vd + (size_t)(nkeys + idx / (HD / 8)) * RB + ((idx % (HD / 8)) << 4)) = make_uint4(0, 0, 0, 0);
+                for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
+                    const int c = idx % (HD / 8);
+                    *reinterpret_cast<uint4 *>(vd + (c >> 3) * HS_ + (size_t)(nkeys + idx / (HD / 8)) * 128 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                }
             }
             __syncthreads();                // tile t complete for everybody; everybody is done with tile t - 1
             fetch(t + 2);                   // into the buffer tile t - 1 used (an empty group beyond the range)
         }
         const unsigned char *K_s = newrows ? reinterpret_cast<const unsigned char *>(Kn_s) : Kbuf(t % A2_NBUF);
         const unsigned char *V_s = newrows ? reinterpret_cast<const unsigned char *>(Vn_s) : Vbuf(t % A2_NBUF);
-        const int pitch = newrows ? KSTR * 2 : RB, swz = newrows ? 0 : 7;
+        // a tile: rows of 128 bytes per half, 16-byte chunks XOR-swizzled with the row; the new rows: padded rows, no swizzle
+        const int pitch = newrows ? KSTR * 2 : 128, swz = newrows ? 0 : 7, hstr = newrows ? 128 : HS_;
         // 16 keys per warp; the new rows are one group, given to the warp that a ragged last tile leaves idle most often
 #pragma unroll 1
         for (int kb = (newrows ? (warp == A2_WARPS - 1 ? 0 : nkp) : warp * 16); kb < nkp; kb += A2_WARPS * 16) {
@@ -1046,7 +1064,7 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
                     uint32_t bk[4];
-                    ldsm_x4(bk, krp + (((ks * 2 + kc0) ^ ksw) << 4));
+                    ldsm_x4(bk, krp + ((ks * 2 + kc0) >> 3) * hstr + (((((ks * 2 + kc0) & 7)) ^ ksw) << 4));
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         uint32_t ah[4], al[4];
@@ -1135,7 +1153,7 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
 #pragma unroll
             for (int p = 0; p < NT / 2; ++p) {
                 uint32_t bv[4];
-                ldsm_x4_t(bv, vrp + (((p * 2 + vc0) ^ vsw) << 4));
+                ldsm_x4_t(bv, vrp + ((p * 2 + vc0) >> 3) * hstr + ((((p * 2 + vc0) & 7) ^ vsw) << 4));
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     mma_bf16(O[mt][2 * p], ph[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], ph[mt], bv[2], bv[3]);
@@ -1146,11 +1164,10 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const AttnArgs a) 
             }
         }
     }
-    cp_async_wait_all();
-    __syncthreads();                        // everybody is done with the tile buffers
+    __syncthreads();                        // everybody is done with the tile buffers (every requested tile was waited for)
 
     // ---- merge the eight warp partials through shared memory (the tile buffers are free now)
-    float *wo_s = reinterpret_cast<float *>(smraw + L.tile_off);            // [A2_WARPS][GTB][HD]
+    float *wo_s = reinterpret_cast<float *>(sm + L.tile_off);            // [A2_WARPS][GTB][HD]
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll

@@ -478,6 +478,13 @@ cudaError_t launch_tc_epi(int epi, const CUtensorMap &mA0, const CUtensorMap &mA
 }  // namespace
 
 bool g_hs_gemm_tc = true;
+bool g_hs_tensor_maps = false;
+
+// K or V cache of one layer as a 2-D bf16 tensor [rows][hd]: boxes of 64 columns x 128 rows, 128-byte swizzle
+cudaError_t hs_make_kv_tensor_map(CUtensorMap *map, const void *base, uint64_t rows, int hd) {
+    if (hd % 64) return cudaErrorInvalidValue;
+    return make_map(map, base, rows, (uint64_t)hd, (uint64_t)hd, 128);
+}
 int g_hs_tc_min_rows = 17;
 
 cudaError_t configure_gemm_tc() {
@@ -487,6 +494,7 @@ cudaError_t configure_gemm_tc() {
     if (e != cudaSuccess) return e;
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    g_hs_tensor_maps = true;
     e = cudaFuncSetAttribute(pack_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(gemm_tc_kernel<32, EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_MAX);
