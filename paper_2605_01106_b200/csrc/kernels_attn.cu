@@ -886,6 +886,7 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_const
     float *wml_s = reinterpret_cast<float *>(sm + L.ml_off);                      // [A2_WARPS + 1][GTB][2]
     __shared__ int ticket_s;
     __shared__ __align__(8) uint64_t tile_bar[A2_NBUF];                              // one per tile buffer pair: bytes of K and V landed
+    __shared__ int tile_done[A2_NBUF];                                               // warps that have finished with the pair's current tile
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t tinv = (65536u + T - 1) / T;
@@ -912,8 +913,8 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_const
     // (K) or cleared (V) below; rows beyond the tensor read as zero.
     constexpr int HALVES = HD / 64, HS_ = CK * 128;      // HS_: bytes between the halves of a tile
     const int row00 = (b * a.kvh + kh) * a.cap + c0;
-    auto fetch = [&](int t) {
-        if (tid != 0 || t >= ntile) return;
+    auto fetch = [&](int t) {              // called by ONE thread
+        if (t >= ntile) return;
         uint64_t *bar = &tile_bar[t % A2_NBUF];
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the buffer was last touched by ordinary loads / stores
         mbar_expect_tx(bar, 2u * CK * RB);
@@ -925,11 +926,10 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_const
     };
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < A2_NBUF; ++i) mbar_init(&tile_bar[i], 1);
+        for (int i = 0; i < A2_NBUF; ++i) { mbar_init(&tile_bar[i], 1); tile_done[i] = 0; }
         mbar_fence_init();
     }
-    fetch(0);
-    fetch(1);
+    if (tid == 0) { fetch(0); fetch(1); fetch(2); }
 #pragma unroll 1
     for (int idx = tid; idx < T * (HD / 2); idx += A2_THREADS) {
         const int i = idx / (HD / 2), e = idx - i * (HD / 2);
@@ -1028,18 +1028,20 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_const
         const int nkeys = newrows ? T : min(CK, rc - t * CK);
         const int nkp = (nkeys + 15) & ~15;
         if (!newrows) {
-            // tile t has landed (tile t + 1 may be in flight); a wait that runs out is reported, the pass goes on
-            if (!mbar_wait(&tile_bar[t % A2_NBUF], (uint32_t)(t / A2_NBUF) & 1u) && tid == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
-            if (nkp != nkeys) {             // a ragged tile (only the last can be): finite V rows for its padding keys
+            // Tile t has landed (tiles t + 1 and t + 2 may be in flight); a wait that runs out is reported and the pass goes
+            // on.  There is no block-wide barrier per tile: a warp works on its 16 keys as soon as the tile is there and
+            // hands the buffers back when it is done (below), so the warps drift apart and fill each other's stalls.
+            if (!mbar_wait(&tile_bar[t % A2_NBUF], (uint32_t)(t / A2_NBUF) & 1u) && lane == 0) atomicCAS(a.status, 0, (int)HS_ERR_TIMEOUT);
+            if (nkp != nkeys && warp * 16 <= nkeys && nkeys < warp * 16 + 16) {
+                // a ragged tile (only the last can be): finite V rows for the padding keys of the group that holds them
                 unsigned char *vd = Vbuf(t % A2_NBUF);
 #pragma unroll 1
-                for (int idx = tid; idx < (nkp - nkeys) * (HD / 8); idx += A2_THREADS) {
+                for (int idx = lane; idx < (nkp - nkeys) * (HD / 8); idx += 32) {
                     const int c = idx % (HD / 8);
                     *reinterpret_cast<uint4 *>(vd + (c >> 3) * HS_ + (size_t)(nkeys + idx / (HD / 8)) * 128 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
                 }
+                __syncwarp();
             }
-            __syncthreads();                // tile t complete for everybody; everybody is done with tile t - 1
-            fetch(t + 2);                   // into the buffer tile t - 1 used (an empty group beyond the range)
         }
         const unsigned char *K_s = newrows ? reinterpret_cast<const unsigned char *>(Kn_s) : Kbuf(t % A2_NBUF);
         const unsigned char *V_s = newrows ? reinterpret_cast<const unsigned char *>(Vn_s) : Vbuf(t % A2_NBUF);
@@ -1161,6 +1163,14 @@ __global__ void __launch_bounds__(A2_THREADS, 1) attn2_kernel(const __grid_const
                         mma_bf16(O[mt][2 * p], pl[mt], bv[0], bv[1]); mma_bf16(O[mt][2 * p + 1], pl[mt], bv[2], bv[3]);
                     }
                 }
+            }
+        }
+        if (!newrows) {
+            // this warp is done with tile t: the last of the eight to say so refills the buffer pair with tile t + 3
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                if (atomicAdd(&tile_done[t % A2_NBUF], 1) == A2_WARPS - 1) { tile_done[t % A2_NBUF] = 0; fetch(t + A2_NBUF); }
             }
         }
     }
