@@ -855,9 +855,12 @@ __host__ __device__ inline Attn2Layout attn2_layout(int hd, int mt) {
     L.total = (o + 127) / 128 * 128 + 1024;
     return L;
 }
+// a tile of cached K or V rows: a long cache is read once per pass, so the copy is marked evict-first in L2
 __device__ __forceinline__ void tma_tile_2d(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 :: "r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 :: "r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol) : "memory");
 }
 
 // PK: the last 16-row query tile is "packed" - it holds at most 8 query rows, their bf16 heads in its rows 0-7 and

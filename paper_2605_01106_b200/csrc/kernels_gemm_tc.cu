@@ -140,6 +140,13 @@ __device__ __forceinline__ void tma_load_2d(void *dst_smem, const CUtensorMap *m
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  :: "r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// the same for a weight tile: streamed once per step, so marked evict-first in L2
+__device__ __forceinline__ void tma_load_2d_stream(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 :: "r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
 // shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | (1u << 16);
@@ -290,8 +297,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mA0, const __grid_constant__ 
         auto load_a = [&](int i) {                      // i: k block relative to kb0
             const int s = i % NS, kb = kb0 + i;
             mbar_expect_tx(&full_bar[s], STAGE);
-            if (kb < a.nk0) tma_load_2d(stages + (size_t)s * STAGE, &mA0, kb * TC_BK, m0, &full_bar[s]);
-            else tma_load_2d(stages + (size_t)s * STAGE, &mA1, (kb - a.nk0) * TC_BK, m0, &full_bar[s]);
+            if (kb < a.nk0) tma_load_2d_stream(stages + (size_t)s * STAGE, &mA0, kb * TC_BK, m0, &full_bar[s]);
+            else tma_load_2d_stream(stages + (size_t)s * STAGE, &mA1, (kb - a.nk0) * TC_BK, m0, &full_bar[s]);
         };
         auto load_b = [&](int i) {
             const int s = i % NS, kb = kb0 + i;
