@@ -259,7 +259,7 @@ int hs_set_attn_geometry(hs_model *m, int chunk, int tiles);
  *   HS_OPT_ATTN_STREAM     verify attention over long caches at large batch (a launch of its own, at most 32 query rows
  *                          per KV head) in its streaming form (default on; off: the general form)
  *   HS_OPT_TC_MIN_ROWS     not a switch: the smallest number of activation rows (2..17) whose projections run on
- *                          tcgen05; 0 restores the automatic choice (7; 5 for models whose weight matrices are large
+ *                          tcgen05; 0 restores the automatic choice (7; 4 for models whose weight matrices are large
  *                          enough that the kernel's fixed cost is small beside the time to stream them) */
 enum { HS_OPT_CLUSTER_REDUCE = 0, HS_OPT_GEMM_MMA = 1, HS_OPT_GEMM_TC = 2, HS_OPT_PDL = 3, HS_OPT_ATTN_SMALL = 4, HS_OPT_ATTN_STREAM = 5,
        HS_OPT_TC_MIN_ROWS = 6 };

@@ -604,8 +604,8 @@ static int init_model(hs_model *m, const hs_config *cfg, const hs_buffers *bufs,
     m->att_acc = (float *)(w + wl.att_acc); m->att_ml = (float *)(w + wl.att_ml); m->am_part = w + wl.am_part; m->xb = (__nv_bfloat16 *)(w + wl.xb); m->xb_rows = gemm_tc_rows(v.R);
     m->xb_h = (__nv_bfloat16 *)(w + wl.xb_h); m->xb_a = (__nv_bfloat16 *)(w + wl.xb_a); m->ssbuf = (float *)(w + wl.ssbuf);
     // the tcgen05 kernel's fixed cost (operand packing, tensor-memory set-up, epilogue out of tensor memory) pays from
-    // 7 activation rows on, from 5 where the weight matrices are large (measured: model widths 1024 and 2560)
-    m->tc_min_rows_auto = (int64_t)4 * c.ff * c.d >= ((int64_t)64 << 20) ? 5 : 7;
+    // 7 activation rows on, from 4 where the weight matrices are large (measured: model widths 1024 and 2560)
+    m->tc_min_rows_auto = (int64_t)4 * c.ff * c.d >= ((int64_t)64 << 20) ? 4 : 7;
     g_hs_tc_min_rows = m->tc_min_rows_auto;
     // conv buffer: committed windows | verify history | draft ping-pong
     float *cv = (float *)bufs->conv;
