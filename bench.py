@@ -34,7 +34,7 @@ ALPHA = 0.68
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection kernel from the ncu capture summarised in
 # profiles/gemv_kernel_cfg2.md: mean over the four projections of a layer of a verify pass, caches left alone (None: the
 # kernel changed after the counters were taken)
-GEMV_DRAM_BYTES_PER_LAUNCH = 11.97e6
+GEMV_DRAM_BYTES_PER_LAUNCH = 11.60e6
 
 
 # ------------------------------------------------------------------------------------------------
