@@ -558,7 +558,10 @@ cudaError_t launch_gemm_tc(const GemvArgs &a, int32_t *status, cudaStream_t s, i
         // stages with one CTA per SM beat two co-resident CTAs with two or three stages each).  Few activation rows
         // make the stages small: then two CTAs fit on an SM with four or more stages each, more CTAs than SMs still
         // run at once and the CTAs of the next projection can stream their weights while this one finishes.
-        const bool pair = TC_SMEM_PAIR >= 4 * stage + crx + TC_MISC_BYTES + 1024;
+        // More tiles than SMs would otherwise run in two rounds, the second nearly empty: there three stages are enough
+        // for a pair (measured: 4-6 % per verify pass on the batched workloads; with two stages it loses again).
+        const bool pair = TC_SMEM_PAIR >= 4 * stage + crx + TC_MISC_BYTES + 1024 ||
+                          (tiles * cand > 148 && TC_SMEM_PAIR >= 3 * stage + crx + TC_MISC_BYTES + 1024);
         if (cand > 1 && tiles > g_tc_clusters[pair ? 1 : 0][cand]) continue;
         if (cand > 1 && tiles * cand > 148) continue;
         S = cand; rb = crb; rx_bytes = crx; budget = pair ? TC_SMEM_PAIR : TC_SMEM_MAX;
