@@ -462,7 +462,7 @@ constexpr size_t tc_stage_bytes(int bn) { return (size_t)TC_BM * TC_BK * 2 + (si
 constexpr size_t TC_SMEM_MAX = 200 * 1024;
 constexpr size_t TC_SMEM_PAIR = 110 * 1024;   // up to this two CTAs fit on an SM
 constexpr size_t TC_MISC_BYTES = (128 + 128 + 4 * 128) * 4;
-int g_tc_clusters[2][9];     // clusters of S CTAs that run at once: [0] one CTA per SM, [1] two per SM
+int g_tc_clusters[2][9];     // clusters of S CTAs that run at once with one CTA per SM ([0]; [1]: the same query at the smaller footprint)
 
 template <int BN, int EPI>
 cudaError_t launch_tc(const CUtensorMap &mA0, const CUtensorMap &mA1, const CUtensorMap &mB, const TcArgs &t, dim3 grid, size_t smem, cudaStream_t s) {
@@ -562,8 +562,9 @@ cudaError_t launch_gemm_tc(const GemvArgs &a, int32_t *status, cudaStream_t s, i
         // for a pair (measured: 4-6 % per verify pass on the batched workloads; with two stages it loses again).
         const bool pair = TC_SMEM_PAIR >= 4 * stage + crx + TC_MISC_BYTES + 1024 ||
                           (tiles * cand > 148 && TC_SMEM_PAIR >= 3 * stage + crx + TC_MISC_BYTES + 1024);
-        if (cand > 1 && tiles > g_tc_clusters[pair ? 1 : 0][cand]) continue;
-        if (cand > 1 && tiles * cand > 148) continue;
+        // with two CTAs per SM twice as many clusters run at once (the occupancy query is made for one per SM)
+        if (cand > 1 && tiles > g_tc_clusters[0][cand] * (pair ? 2 : 1)) continue;
+        if (cand > 1 && tiles * cand > (pair ? 2 * 148 : 148)) continue;
         S = cand; rb = crb; rx_bytes = crx; budget = pair ? TC_SMEM_PAIR : TC_SMEM_MAX;
     }
     const int nkl = (nk + S - 1) / S;
