@@ -228,12 +228,14 @@ AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
     int want = 32;
     while (want < 128 && 8 * want < maxlen + T) want += 32;
     // Long caches at a batch that fills the GPU several times over, in a launch of its own (not fused with the mixer):
-    // the streaming form - 128-key tiles, as many per CTA (up to 16) as still leave every SM a few CTAs.
+    // the streaming form - 128-key tiles, up to 16 per CTA.
     {
         const bool own_launch = m->c.arch == HS_ARCH_SEQUENTIAL || (int64_t)(m->c.P / 16) * m->c.H * nb > 4 * 148;
         const int64_t ctas128 = (int64_t)nb * m->c.kvh * ((maxlen + T + 127) / 128);
         if (g_hs_attn_stream && have_maps && own_launch && (m->c.qh / m->c.kvh) * Tq <= 32 && ctas128 >= 2 * 148) {
-            int tiles = (int)(ctas128 / (4 * 148));
+            // tiles per CTA: up to 16, fewer only while that still leaves about half an SM count of CTAs (measured: 544 tiles
+            // of work run best as 8 per CTA - staging the queries and merging the ranges is paid per CTA)
+            int tiles = (int)((ctas128 + 73) / 74);
             tiles = tiles < 1 ? 1 : tiles > 16 ? 16 : tiles;
             return AttnGeom{128, tiles, 0, 1};
         }
