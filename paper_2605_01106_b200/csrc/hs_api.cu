@@ -246,6 +246,12 @@ AttnGeom attn_geom(const hs_model *m, int Tq, int T, int b0, int nb) {
     if (g.chunk == 128 && ctas64 >= 4 * fill) {
         g.chunk = 64;
         g.tiles = ctas64 / fill >= 16 ? 16 : ctas64 / fill >= 8 ? 8 : ctas64 / fill >= 4 ? 4 : 2;
+    } else if (g.chunk == 128 && maxlen + T > 8 * 128) {
+        // a cache beyond one cluster of 128-key ranges: as many tiles per CTA as keep it inside ONE cluster, which spares
+        // the merge of several clusters' partials through global memory (measured, 2048 keys: 2-3 % per verify pass)
+        int t = (maxlen + T + 8 * 128 - 1) / (8 * 128);
+        t = t < 4 ? (t < 2 ? 2 : 4) : t;              // measured: four tiles beat two and three at 2048 keys
+        g.tiles = t > 16 ? 16 : t;
     }
     return g;
 }
